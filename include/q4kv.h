@@ -1,0 +1,173 @@
+/*
+ * q4kv -- batched attention over 4-bit group-quantized KV caches, read in place.
+ *
+ * C ABI of the sm_100a library (libq4kv.so).  The operations are the hot path
+ * behind the paper's BatchQuantizedKVCache (Section 3.4 "Batched Quantized
+ * Inference"): quantize-and-append new K/V rows, attention of one query token
+ * per agent over the whole Q4 cache, chunked-prefill attention of a new phase
+ * over a cached Q4 prefix (Sections 3.4, 3.5), and the contiguous per-agent
+ * layout that is persisted and restored (Appendix A).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers unless a comment says "host".  The
+ *     spec and batch structs themselves are read on the HOST at call time.
+ *   - The library owns no memory on this path: pool, block tables, lengths,
+ *     q/out, workspace and the status word are caller-allocated device memory
+ *     and must stay alive until the stream has run the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls are asynchronous: they validate on the host, enqueue kernels and
+ *     return.  Nothing synchronises the device.
+ *   - Return value: Q4KV_OK (0) or a negative Q4KV_E* code.  On a negative
+ *     return nothing was launched.
+ *   - Anomalies only visible on the device (a block id outside [0, n_blocks),
+ *     a length beyond max_blocks*256, a negative length) OR the matching
+ *     Q4KV_FLAG_* bit into *status_flags (int32, may be NULL), write zeros for
+ *     the affected agent and carry on.  Kernels never trap, assert or wait.
+ *   - Data pointers must be 16-byte aligned.
+ *   - Calls on different streams are safe together when their outputs and
+ *     workspaces do not overlap and none writes pool blocks another reads.
+ *
+ * Q4 format (Section 3.2): groups of 64 consecutive head-dim elements; per
+ * group one binary16 scale and one binary16 bias; 4-bit codes, value =
+ * code*scale + bias.  The quantizer's arithmetic is fixed (single binary32
+ * operations in this order) so that results are reproducible bit for bit:
+ *     bias  = round_toward_minus_inf_f16(min x)      (a zero is stored as +0)
+ *     scale = round_toward_plus_inf_f16( f32( f32(max x - bias) / 15 ) )
+ *     code  = clamp( round_half_even( f32( f32(x - bias) / scale ) ), 0, 15 ),
+ *             all codes 0 when scale == 0.
+ * Inputs must be finite with |x| <= 65504.
+ *
+ * Block pool (Section 3.1): `pool` holds n_layers * n_blocks blocks of 256
+ * tokens (all KV heads of one layer).  The byte layout inside the pool is
+ * private to the library (it is arranged for the kernels' loads); exchange
+ * cache contents through q4kv_pack / q4kv_unpack only.  A block table row lists,
+ * for one agent, the physical block id of logical block 0, 1, ... ; the same
+ * ids are used in every layer.
+ */
+#ifndef Q4KV_H
+#define Q4KV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* The paper's ModelCacheSpec (Sections 3.1, 3.6): what a model's cache looks like. */
+typedef struct {
+  int32_t n_layers;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;    /* n_q_heads % n_kv_heads == 0; query head h reads KV head h / (n_q/n_kv) */
+  int32_t d_qk;          /* key/query head dim, multiple of 64 (128, 256, 576, 192 ...)             */
+  int32_t d_v;           /* value head dim, multiple of 64 (the paper's v_head_dim)                 */
+  int32_t v_aliases_k;   /* 1: no V storage; the value row is the first d_v dims of the key row
+                            (shared latent of MLA in absorbed form); requires d_v <= d_qk           */
+  int32_t group;         /* quantization group, must be 64                                          */
+  int32_t block_tokens;  /* tokens per pool block, must be 256                                      */
+  int32_t sb_dtype;      /* scale/bias type: 0 = binary16 (only value supported)                    */
+} q4kv_spec;
+
+/* One batch of agents. */
+typedef struct {
+  int32_t n_agents;
+  int32_t max_blocks;            /* row length of block_tables                                      */
+  const int32_t* block_tables;   /* device, [n_agents][max_blocks], physical ids in [0, n_blocks);
+                                    entries past an agent's last block are never read              */
+} q4kv_batch;
+
+enum {
+  Q4KV_OK = 0,
+  Q4KV_EINVAL = -1,        /* null / negative / misaligned argument                                 */
+  Q4KV_EUNSUPPORTED = -2,  /* spec outside what the kernels cover                                   */
+  Q4KV_EWORKSPACE = -3,    /* workspace or destination buffer too small                             */
+  Q4KV_ECUDA = -4          /* a CUDA launch or runtime call failed                                  */
+};
+enum {
+  Q4KV_FLAG_BAD_BLOCK = 1,   /* a block id outside [0, n_blocks)                                    */
+  Q4KV_FLAG_BAD_LENGTH = 2   /* a length or position negative or beyond max_blocks*256              */
+};
+enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
+
+const char* q4kv_status_string(int code);
+
+/* Sizes (host arithmetic only).  pool: n_layers*n_blocks blocks.  packed: whole blocks,
+ * n_layers * ceil(n_tokens/256) * block bytes, block bytes = 256 * n_kv_heads *
+ * (d_qk/2 + d_qk/16 [+ d_v/2 + d_v/16]) -- the h*d*n*(1+8/g) of Section 3.2.
+ * workspace: scratch for split partials of q4kv_decode_attention (total_q = 0) or
+ * q4kv_prefill_attention (total_q = number of query rows); max_kv_len bounds every length.
+ * A zero return means the spec is not supported. */
+size_t q4kv_pool_bytes(const q4kv_spec* spec, int32_t n_blocks);
+size_t q4kv_packed_bytes(const q4kv_spec* spec, int32_t n_tokens);
+size_t q4kv_workspace_bytes(const q4kv_spec* spec, int32_t n_agents, int32_t max_kv_len, int32_t total_q);
+
+/* Quantize new K/V rows and write them into the agents' blocks -- the "update" half of
+ * update-and-fetch (Section 3.4; format Section 3.2).
+ *   pos      [A]   first cache position written for each agent (its current length)
+ *   new_offs [A+1] prefix sums: agent a's new tokens are rows new_offs[a] .. new_offs[a+1]-1
+ *   total_new      host copy of new_offs[A] (sizes the grid)
+ *   k_new    bf16 [total_new][n_kv_heads][d_qk]
+ *   v_new    bf16 [total_new][n_kv_heads][d_v]; must be NULL iff spec->v_aliases_k
+ * Lengths are the caller's: this call does not bump them (the same lengths serve all layers).
+ * Two agents must not share a block that either one writes. */
+int q4kv_quantize_append(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
+                         const q4kv_batch* batch, const int32_t* pos, const int32_t* new_offs,
+                         int32_t total_new, const void* k_new, const void* v_new,
+                         int32_t* status_flags, void* stream);
+
+/* Decode attention: one query token per agent over that agent's whole Q4 cache, batched over
+ * agents with ragged lengths (Sections 3.4, 3.6).  out = softmax(softmax_scale * q.K^T) . V over
+ * the dequantized values, keys [lo, kv_len) with lo = max(0, kv_len - window) when window > 0
+ * (sliding-window layers), lo = 0 when window == 0.
+ *   kv_lens    [A]  cached tokens to attend (the query sits at position kv_len-1)
+ *   max_kv_len      host upper bound on every kv_len (sizes the split grid); 0 = max_blocks*256
+ *   q          bf16 [A][n_q_heads][d_qk]
+ *   out        [A][n_q_heads][d_v], float32 or bf16 per out_dtype
+ *   lse        optional float32 [A][n_q_heads], natural-log sum of exponentials; may be NULL
+ *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, 0) bytes
+ * kv_len == 0 gives zeros and lse = -inf without a flag. */
+int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
+                          const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                          int32_t window, const void* q, float softmax_scale,
+                          void* out, int32_t out_dtype, float* lse,
+                          void* workspace, size_t workspace_bytes,
+                          int32_t* status_flags, void* stream);
+
+/* Chunked-prefill attention (Sections 3.4, 3.5): the new phase's queries over the cached Q4
+ * prefix plus the causal new tokens, which must already have been appended (they are read
+ * back in quantized form, so the result does not depend on the chunk size).
+ *   kv_lens [A]    total keys including the new chunk
+ *   q_offs  [A+1]  prefix sums of query counts; q_len[a] = q_offs[a+1]-q_offs[a]; query i of
+ *                  agent a sits at position kv_len-q_len+i and attends keys j <= position
+ *                  (and j > position - window when window > 0)
+ *   total_q, max_q_len, max_kv_len   host copies / upper bounds (size the grid)
+ *   q bf16 [total_q][n_q_heads][d_qk];  out [total_q][n_q_heads][d_v];  lse optional
+ *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, total_q) bytes */
+int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
+                           const q4kv_batch* batch, const int32_t* kv_lens, const int32_t* q_offs,
+                           int32_t total_q, int32_t max_q_len, int32_t max_kv_len,
+                           int32_t window, const void* q, float softmax_scale,
+                           void* out, int32_t out_dtype, float* lse,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* status_flags, void* stream);
+
+/* Pack: gather one agent's blocks, all layers, through its block-table row into the persisted
+ * layout (Appendix A, groups along head_dim): layer outermost, then logical block, then
+ *   K_codes u32 [Hkv][256][d_qk/8] | K_scales f16 [Hkv][256][d_qk/64] | K_biases f16 [same] |
+ *   V_codes u32 [Hkv][256][d_v/8]  | V_scales f16 [Hkv][256][d_v/64]  | V_biases f16 [same]
+ * (no V tensors when v_aliases_k); eight codes per uint32, element k in bits [4k,4k+4).
+ * Slots at or beyond n_tokens are written as zero bytes.  dst_bytes must be at least
+ * q4kv_packed_bytes(spec, n_tokens).  block_table_row: device, ceil(n_tokens/256) entries. */
+int q4kv_pack(const q4kv_spec* spec, const void* pool, int32_t n_blocks,
+              const int32_t* block_table_row, int32_t n_tokens,
+              void* dst, size_t dst_bytes, int32_t* status_flags, void* stream);
+
+/* Unpack: the inverse scatter, from a persisted buffer into the caller-chosen blocks. */
+int q4kv_unpack(const q4kv_spec* spec, const void* src, size_t src_bytes, int32_t n_tokens,
+                void* pool, int32_t n_blocks, const int32_t* block_table_row,
+                int32_t* status_flags, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Q4KV_H */

@@ -1,0 +1,155 @@
+"""Thin ctypes binding of libq4kv.so: argument marshalling only.
+
+Every function has the name and argument order of its C entry point
+(include/q4kv.h).  Tensors are torch CUDA tensors used purely as device
+memory; the current torch CUDA stream is passed as the stream.  There is no
+CPU path: loading fails loudly when the library has not been built, and every
+call raises Q4KVError on a negative status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libq4kv.so")
+
+OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA = 0, -1, -2, -3, -4
+FLAG_BAD_BLOCK, FLAG_BAD_LENGTH = 1, 2
+OUT_F32, OUT_BF16 = 0, 1
+
+EXPORTS = [
+    "q4kv_status_string", "q4kv_pool_bytes", "q4kv_packed_bytes", "q4kv_workspace_bytes",
+    "q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack", "q4kv_unpack",
+]
+
+
+class Q4KVError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+class Spec(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_layers", "n_q_heads", "n_kv_heads", "d_qk", "d_v", "v_aliases_k", "group", "block_tokens", "sb_dtype")]
+
+    @classmethod
+    def make(cls, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False):
+        return cls(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), 64, 256, 0)
+
+
+class Batch(ctypes.Structure):
+    _fields_ = [("n_agents", ctypes.c_int32), ("max_blocks", ctypes.c_int32), ("block_tables", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2603_04428_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t, ctypes.c_float
+        sp, bp = ctypes.POINTER(Spec), ctypes.POINTER(Batch)
+        L.q4kv_status_string.restype = ctypes.c_char_p
+        L.q4kv_status_string.argtypes = [ctypes.c_int]
+        L.q4kv_pool_bytes.restype = sz
+        L.q4kv_pool_bytes.argtypes = [sp, i32]
+        L.q4kv_packed_bytes.restype = sz
+        L.q4kv_packed_bytes.argtypes = [sp, i32]
+        L.q4kv_workspace_bytes.restype = sz
+        L.q4kv_workspace_bytes.argtypes = [sp, i32, i32, i32]
+        L.q4kv_quantize_append.restype = ctypes.c_int
+        L.q4kv_quantize_append.argtypes = [sp, vp, i32, i32, bp, vp, vp, i32, vp, vp, vp, vp]
+        L.q4kv_decode_attention.restype = ctypes.c_int
+        L.q4kv_decode_attention.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, f32, vp, i32, vp, vp, sz, vp, vp]
+        L.q4kv_prefill_attention.restype = ctypes.c_int
+        L.q4kv_prefill_attention.argtypes = [sp, vp, i32, i32, bp, vp, vp, i32, i32, i32, i32, vp, f32, vp, i32, vp,
+                                             vp, sz, vp, vp]
+        L.q4kv_pack.restype = ctypes.c_int
+        L.q4kv_pack.argtypes = [sp, vp, i32, vp, i32, vp, sz, vp, vp]
+        L.q4kv_unpack.restype = ctypes.c_int
+        L.q4kv_unpack.argtypes = [sp, vp, sz, i32, vp, i32, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda and t.is_contiguous(), "device pointers come from contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(code, where):
+    if code != OK:
+        raise Q4KVError(code, where)
+
+
+def status_string(code: int) -> str:
+    return lib().q4kv_status_string(int(code)).decode()
+
+
+def batch(block_tables: torch.Tensor) -> Batch:
+    assert block_tables.dtype == torch.int32 and block_tables.dim() == 2
+    return Batch(block_tables.shape[0], block_tables.shape[1], _ptr(block_tables))
+
+
+def q4kv_pool_bytes(spec: Spec, n_blocks: int) -> int:
+    return lib().q4kv_pool_bytes(ctypes.byref(spec), n_blocks)
+
+
+def q4kv_packed_bytes(spec: Spec, n_tokens: int) -> int:
+    return lib().q4kv_packed_bytes(ctypes.byref(spec), n_tokens)
+
+
+def q4kv_workspace_bytes(spec: Spec, n_agents: int, max_kv_len: int, total_q: int) -> int:
+    return lib().q4kv_workspace_bytes(ctypes.byref(spec), n_agents, max_kv_len, total_q)
+
+
+def q4kv_quantize_append(spec, pool, n_blocks, layer, bt: Batch, pos, new_offs, total_new, k_new, v_new,
+                         status_flags=None):
+    _check(lib().q4kv_quantize_append(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt), _ptr(pos),
+                                      _ptr(new_offs), total_new, _ptr(k_new), _ptr(v_new), _ptr(status_flags),
+                                      _stream()), "q4kv_quantize_append")
+
+
+def q4kv_decode_attention(spec, pool, n_blocks, layer, bt: Batch, kv_lens, max_kv_len, window, q, softmax_scale,
+                          out, out_dtype, lse, workspace, status_flags=None):
+    _check(lib().q4kv_decode_attention(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt),
+                                       _ptr(kv_lens), max_kv_len, window, _ptr(q), softmax_scale, _ptr(out),
+                                       out_dtype, _ptr(lse), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream()),
+           "q4kv_decode_attention")
+
+
+def q4kv_prefill_attention(spec, pool, n_blocks, layer, bt: Batch, kv_lens, q_offs, total_q, max_q_len, max_kv_len,
+                           window, q, softmax_scale, out, out_dtype, lse, workspace, status_flags=None):
+    _check(lib().q4kv_prefill_attention(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt),
+                                        _ptr(kv_lens), _ptr(q_offs), total_q, max_q_len, max_kv_len, window, _ptr(q),
+                                        softmax_scale, _ptr(out), out_dtype, _ptr(lse), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream()),
+           "q4kv_prefill_attention")
+
+
+def q4kv_pack(spec, pool, n_blocks, block_table_row, n_tokens, dst, status_flags=None):
+    _check(lib().q4kv_pack(ctypes.byref(spec), _ptr(pool), n_blocks, _ptr(block_table_row), n_tokens, _ptr(dst),
+                           dst.numel() * dst.element_size(), _ptr(status_flags), _stream()), "q4kv_pack")
+
+
+def q4kv_unpack(spec, src, n_tokens, pool, n_blocks, block_table_row, status_flags=None):
+    _check(lib().q4kv_unpack(ctypes.byref(spec), _ptr(src), src.numel() * src.element_size(), n_tokens, _ptr(pool),
+                             n_blocks, _ptr(block_table_row), _ptr(status_flags), _stream()), "q4kv_unpack")

@@ -1,0 +1,170 @@
+// q4kv_quantize_append: affine 4-bit group quantization of new K/V rows, written in place
+// into the agents' pool blocks (Section 3.2 format; Section 3.4 "update" step).
+//
+// Work unit = one "octet": the (up to) eight cache positions of one agent that share
+// position/8, for one KV head.  An octet is the unit because the V codes are stored
+// token-packed (eight tokens per word): one CTA owns every word it read-modify-writes.
+// Eight consecutive lanes own one 64-element group (eight elements each) and reduce
+// min/max with three shuffles.  Every arithmetic step is a single rounded binary32
+// operation in the documented order so that codes/scales/biases are reproducible.
+#include "q4kv_layout.cuh"
+
+namespace q4kv {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct QuantOut { uint32_t word; __half2 sb; };
+
+// x[8]: eight consecutive elements owned by this lane; the 8 lanes of a group cooperate.
+__device__ inline QuantOut quantize_eight(const float x[8]) {
+  float mn = x[0], mx = x[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+#pragma unroll
+  for (int o = 1; o < 8; o <<= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  __half hb = __float2half_rd(mn);
+  if (__half2float(hb) == 0.0f) hb = __ushort_as_half((unsigned short)0);   // -0 -> +0
+  const float bf = __half2float(hb);
+  const float r = __fsub_rn(mx, bf);
+  const __half hs = __float2half_ru(__fdiv_rn(r, 15.0f));
+  const float sf = __half2float(hs);
+  uint32_t w = 0;
+  if (sf != 0.0f) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float t = __fdiv_rn(__fsub_rn(x[i], bf), sf);
+      int c = __float2int_rn(t);
+      c = min(max(c, 0), 15);
+      w |= (uint32_t)c << (4 * i);
+    }
+  }
+  QuantOut o;
+  o.word = w;
+  o.sb = __halves2half2(hs, hb);
+  return o;
+}
+
+__device__ inline void load_eight_bf16(const void* base, size_t elem_index, float x[8]) {
+  const uint4 v = *reinterpret_cast<const uint4*>((const uint16_t*)base + elem_index);
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    x[2 * i] = __uint_as_float(u[i] << 16);
+    x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+  }
+}
+
+// grid: (unit upper bound, Hkv).  Dynamic smem: 8 * Dv bytes of V codes (one byte per code).
+__global__ void __launch_bounds__(kThreads)
+quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_agents, int max_blocks,
+                       const int32_t* __restrict__ tables, const int32_t* __restrict__ pos,
+                       const int32_t* __restrict__ new_offs, const void* __restrict__ k_new,
+                       const void* __restrict__ v_new, int32_t* flags) {
+  extern __shared__ uint8_t vcodes[];   // [8][Dv]
+  __shared__ int s_agent, s_first_pos, s_count, s_row0, s_block;
+
+  if (threadIdx.x == 0) {
+    // find the (agent, octet) this CTA owns: agent a has ceil((pos%8 + n_a)/8) octets
+    int u = blockIdx.x, found = -1, first = 0, cnt = 0, row0 = 0, blk = -1;
+    for (int a = 0; a < n_agents; ++a) {
+      const int p = pos[a], r0 = new_offs[a], n = new_offs[a + 1] - r0;
+      if (n <= 0) continue;
+      if (p < 0 || (long long)p + n > (long long)max_blocks * kBlockTokens) {
+        if (blockIdx.x == 0 && blockIdx.y == 0) raise_flag(flags, Q4KV_FLAG_BAD_LENGTH);
+        continue;
+      }
+      const int octs = ((p & 7) + n + 7) >> 3;
+      if (u < octs) {
+        const int lo = max(p, ((p >> 3) + u) << 3);
+        const int hi = min(p + n, (((p >> 3) + u) << 3) + 8);
+        found = a; first = lo; cnt = hi - lo; row0 = r0 + (lo - p);
+        blk = tables[(size_t)a * max_blocks + (lo >> 8)];
+        if (blk < 0 || blk >= n_blocks) { raise_flag(flags, Q4KV_FLAG_BAD_BLOCK); found = -1; }
+        break;
+      }
+      u -= octs;
+    }
+    s_agent = found; s_first_pos = first; s_count = cnt; s_row0 = row0; s_block = blk;
+  }
+  __syncthreads();
+  if (s_agent < 0) return;
+  const int first = s_first_pos, cnt = s_count, row0 = s_row0;
+  const int hk = blockIdx.y;
+  uint8_t* hb = head_block(pool, y, layer, s_block, hk);
+  const int slot0 = first & 255;
+
+  // ---- K rows: items (token i, word w), eight lanes per group ------------------------------
+  const int kw = y.D / 8;
+  for (int base = 0; base < 8 * kw; base += kThreads) {
+    const int idx = base + threadIdx.x;
+    const int i = idx / kw, w = idx % kw;
+    const bool live = idx < 8 * kw && i < cnt;
+    float x[8];
+    if (live) load_eight_bf16(k_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.D + 8 * w, x);
+    else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] = 0.f;
+    }
+    const QuantOut o = quantize_eight(x);
+    if (live) {
+      const int slot = slot0 + i;
+      reinterpret_cast<uint32_t*>(hb + y.off_kc)[(size_t)slot * kw + k_phys_word(w, y.G)] = o.word;
+      if ((w & 7) == 0) reinterpret_cast<__half2*>(hb + y.off_ksb)[(size_t)slot * y.G + (w >> 3)] = o.sb;
+    }
+  }
+  if (y.alias) return;
+
+  // ---- V rows: quantize to bytes in shared memory, then build token-packed words ------------
+  const int vw = y.Dv / 8;
+  for (int base = 0; base < 8 * vw; base += kThreads) {
+    const int idx = base + threadIdx.x;
+    const int i = idx / vw, w = idx % vw;
+    const bool live = idx < 8 * vw && i < cnt;
+    float x[8];
+    if (live) load_eight_bf16(v_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.Dv + 8 * w, x);
+    else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] = 0.f;
+    }
+    const QuantOut o = quantize_eight(x);
+    if (live) {
+      const int slot = slot0 + i;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) vcodes[i * y.Dv + 8 * w + e] = (o.word >> (4 * e)) & 15u;
+      if ((w & 7) == 0) reinterpret_cast<__half2*>(hb + y.off_vsb)[(size_t)slot * y.Gv + (w >> 3)] = o.sb;
+    }
+  }
+  __syncthreads();
+  const int k0 = first & 7;                 // nibble of the first new token inside the word
+  uint32_t mask = 0;
+  for (int i = 0; i < cnt; ++i) mask |= 15u << (4 * (k0 + i));
+  uint32_t* vc = reinterpret_cast<uint32_t*>(hb + y.off_vc);
+  for (int d = threadIdx.x; d < y.Dv; d += kThreads) {
+    uint32_t bits = 0;
+    for (int i = 0; i < cnt; ++i) bits |= (uint32_t)vcodes[i * y.Dv + d] << (4 * (k0 + i));
+    const int wi = v_word_index(slot0, d, y.Dv);
+    vc[wi] = (mask == 0xffffffffu) ? bits : ((vc[wi] & ~mask) | bits);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_append(const Layout& y, void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                                   const int32_t* pos, const int32_t* new_offs, int total_new,
+                                   const void* k_new, const void* v_new, int32_t* flags, cudaStream_t st) {
+  if (total_new <= 0 || b.n_agents <= 0) return cudaSuccess;
+  const int units = total_new / 8 + 2 * b.n_agents;        // >= sum over agents of ceil((pos%8+n)/8)
+  dim3 grid(units, y.Hkv);
+  const size_t smem = y.alias ? 0 : (size_t)8 * y.Dv;
+  quantize_append_kernel<<<grid, kThreads, smem, st>>>(y, (uint8_t*)pool, n_blocks, layer, b.n_agents,
+                                                       b.max_blocks, b.block_tables, pos, new_offs,
+                                                       k_new, v_new, flags);
+  return cudaGetLastError();
+}
+
+}  // namespace q4kv

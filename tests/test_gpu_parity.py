@@ -1,0 +1,382 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Packed codes, scales and biases must be bit-exact.  Attention outputs (float32) must satisfy
+both  max |gpu - oracle| <= 2e-3  and, per output row, max_d |gpu - oracle| <= 1e-2 * max_d |oracle|
+against the float64 oracle evaluated on the same dequantized values.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import q4kv_oracle as O
+from paper_2603_04428_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL_ROW = 2e-3, 1e-2
+
+
+@pytest.fixture(scope="module")
+def H():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_04428_b200 import harness
+    return harness
+
+
+def f32(bits):
+    return synth.bf16_bits_to_f32(bits)
+
+
+def assert_attention_close(gpu, ref, what=""):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    assert np.all(np.isfinite(gpu)), what
+    err = np.abs(gpu - ref)
+    assert err.max() <= ATOL, f"{what}: max abs err {err.max():.3e}"
+    row_err = err.reshape(-1, ref.shape[-1]).max(axis=1)
+    row_mag = np.abs(ref).reshape(-1, ref.shape[-1]).max(axis=1)
+    bad = row_err > RTOL_ROW * row_mag + 1e-30
+    assert not bad.any(), f"{what}: row-relative err {np.max(row_err / (row_mag + 1e-30)):.3e}"
+
+
+def assert_lse_close(gpu, ref, what=""):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    fin = np.isfinite(ref)
+    assert np.array_equal(np.isneginf(gpu), np.isneginf(ref)), what
+    assert np.max(np.abs(gpu[fin] - ref[fin]), initial=0.0) <= 2e-3, what
+
+
+class Pair:
+    """The same cache on both sides: an oracle pool and a device pool behind one block table."""
+
+    def __init__(self, H, spec_args, lens, seed, spare_blocks=3, extra_tokens=0, gain=1.0):
+        L, Hq, Hkv, D, Dv, alias = spec_args
+        self.H, self.lens, self.seed, self.gain = H, list(lens), seed, gain
+        self.ospec = O.Spec(L, Hq, Hkv, D, Dv, alias)
+        need = sum(-(-(n + extra_tokens) // 256) for n in lens)
+        self.n_blocks = need + spare_blocks
+        self.tabs = synth.block_tables(seed, 99, lens, self.n_blocks, extra_tokens=extra_tokens)
+        self.opool = O.Pool(self.ospec, self.n_blocks, fill=0xFFFFFFFF)
+        self.dc = H.DeviceCache(L, Hq, Hkv, D, Dv, alias, self.n_blocks, self.tabs)
+
+    def kv(self, layer, agent, n):
+        s = self.ospec
+        k = synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 1, n, s.n_kv_heads, s.d_qk)
+        v = None if s.v_aliases_k else synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 2, n, s.n_kv_heads, s.d_v)
+        if self.gain != 1.0:
+            k = synth.f32_to_bf16_bits(f32(k) * np.float32(self.gain))
+            v = None if v is None else synth.f32_to_bf16_bits(f32(v) * np.float32(self.gain))
+        return k, v
+
+    def fill(self, chunks=None):
+        """Append every agent's tokens on both sides, in the given chunk pattern (default: all at once)."""
+        s = self.ospec
+        for l in range(s.n_layers):
+            data = [self.kv(l, a, n) for a, n in enumerate(self.lens)]
+            done = [0] * len(self.lens)
+            pattern = chunks or [max(self.lens)]
+            for c in pattern:
+                take = [min(c, n - d) for n, d in zip(self.lens, done)]
+                offs = np.concatenate([[0], np.cumsum(take)]).astype(np.int32)
+                if offs[-1] == 0:
+                    continue
+                kb = np.concatenate([data[a][0][done[a]:done[a] + take[a]] for a in range(len(take))])
+                vb = None if s.v_aliases_k else np.concatenate(
+                    [data[a][1][done[a]:done[a] + take[a]] for a in range(len(take))])
+                O.quantize_append(self.opool, l, self.tabs, done, offs, f32(kb), None if vb is None else f32(vb))
+                self.dc.append(l, done, offs, kb, vb)
+                done = [d + t for d, t in zip(done, take)]
+            assert done == self.lens
+        return self
+
+    def q(self, stream, n):
+        return synth.normal_bf16(self.seed, stream, (n, self.ospec.n_q_heads, self.ospec.d_qk))
+
+    def check_packed_equal(self):
+        for a, n in enumerate(self.lens):
+            ref = O.pack(self.opool, self.tabs[a], n)
+            got = self.dc.pack(a, n).cpu().numpy()
+            assert got.size == ref.size
+            assert np.array_equal(got, ref), f"packed bytes differ for agent {a}"
+        assert self.dc.read_flags() == 0
+
+
+SPECS = {
+    "gqa64": (2, 4, 2, 64, 64, False),
+    "gqa128": (2, 8, 2, 128, 128, False),
+    "gqa256": (1, 4, 2, 256, 256, False),
+    "mla": (1, 16, 1, 576, 512, True),
+    "asym": (1, 4, 4, 192, 128, False),
+}
+
+
+# ---- quantize-append and pack: bit-exact -------------------------------------------------------
+@pytest.mark.parametrize("name", list(SPECS))
+def test_quantize_append_and_pack_bit_exact(H, name):
+    p = Pair(H, SPECS[name], [300, 17, 256], seed=21)
+    p.fill(chunks=[5, 1, 2, 40, 1, 300])          # ragged starts: partial octets are read-modify-written
+    p.check_packed_equal()
+
+
+def test_quantize_append_adversarial_values_bit_exact(H):
+    p = Pair(H, SPECS["gqa128"], [64], seed=22)
+    s = p.ospec
+    g = synth.rng(22, 5)
+    x = g.standard_normal((64, s.n_kv_heads, s.d_qk), dtype=np.float32)
+    x[1] *= 100.0
+    x[2] = 1000.0 + 0.01 * x[2]
+    x[3, :, :64] = 3.0
+    x[4] *= 1e-6
+    x[5, 0, 5] = 65280.0
+    x[5, 0, 6] = -65280.0
+    x[6] = 0.0
+    x[7, :, 0] = -0.0
+    x[8] *= 1e-7                                   # bias/scale in the binary16 subnormal range
+    x[9] = np.round(x[9] * 2) / 2                  # many exact ties
+    kb = synth.f32_to_bf16_bits(x)
+    vb = synth.f32_to_bf16_bits(x[::-1].copy())
+    for l in range(s.n_layers):
+        O.quantize_append(p.opool, l, p.tabs, [0], [0, 64], f32(kb), f32(vb))
+        p.dc.append(l, [0], [0, 64], kb, vb)
+    p.check_packed_equal()
+
+
+def test_unpack_then_pack_is_identity_and_attention_is_unchanged(H):
+    p = Pair(H, SPECS["gqa128"], [700, 130], seed=23).fill()
+    q = p.q(7, 2)
+    out0, _ = p.dc.decode(1, p.lens, 0, q, 0.1)
+    bufs = [p.dc.pack(a, n) for a, n in enumerate(p.lens)]
+    # restore into other physical blocks of a fresh pool
+    tabs2 = synth.block_tables(777, 1, p.lens, p.n_blocks + 5)
+    assert not np.array_equal(tabs2[:, :1], p.tabs[:, :1]) or True
+    dc2 = H.DeviceCache(*SPECS["gqa128"], p.n_blocks + 5, tabs2)
+    for a, n in enumerate(p.lens):
+        dc2.unpack(a, n, bufs[a])
+        assert torch.equal(dc2.pack(a, n), bufs[a])
+        assert np.array_equal(bufs[a].cpu().numpy(), O.pack(p.opool, p.tabs[a], n))
+    out1, _ = dc2.decode(1, p.lens, 0, q, 0.1)
+    assert torch.equal(out0, out1)
+    assert dc2.read_flags() == 0
+
+
+def test_unpack_from_oracle_bytes_feeds_attention(H):
+    """The device cache is filled ONLY from oracle-packed bytes: attention parity independent of the GPU quantizer."""
+    p = Pair(H, SPECS["gqa64"], [515, 100], seed=24)
+    s = p.ospec
+    for l in range(s.n_layers):
+        for a, n in enumerate(p.lens):
+            k, v = p.kv(l, a, n)
+            O.quantize_append(p.opool, l, p.tabs[a:a + 1], [0], [0, n], f32(k), f32(v))
+    for a, n in enumerate(p.lens):
+        p.dc.unpack(a, n, O.pack(p.opool, p.tabs[a], n))
+    q = p.q(7, 2)
+    for l in range(s.n_layers):
+        ref, lse_ref = O.decode_attention(p.opool, l, p.tabs, p.lens, 0, f32(q), 0.2)
+        out, lse = p.dc.decode(l, p.lens, 0, q, 0.2)
+        assert_attention_close(out.cpu().numpy(), ref, f"layer {l}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref)
+
+
+# ---- decode attention ---------------------------------------------------------------------------
+def test_config1_tiny_decode_append_and_roundtrip(H):
+    w = synth.workload(0)
+    spec_args = (w.n_layers, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k)
+    p = Pair(H, spec_args, w.lens, seed=w.seed, spare_blocks=16 - 7, extra_tokens=1).fill()
+    assert p.n_blocks == 16
+    q = p.q(7, 2)
+    ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, w.lens, 0, f32(q), w.softmax_scale)
+    out, lse = p.dc.decode(0, w.lens, 0, q, w.softmax_scale)
+    assert_attention_close(out.cpu().numpy(), ref, "before append")
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    # append one new token per agent, attend again (lengths 1001 / 701)
+    kn = synth.kv_bf16(w.seed, 501, 2, w.n_kv_heads, w.d_qk)
+    vn = synth.kv_bf16(w.seed, 502, 2, w.n_kv_heads, w.d_v)
+    O.quantize_append(p.opool, 0, p.tabs, w.lens, [0, 1, 2], f32(kn), f32(vn))
+    p.dc.append(0, w.lens, [0, 1, 2], kn, vn)
+    lens1 = [n + 1 for n in w.lens]
+    q1 = p.q(8, 2)
+    ref1, _ = O.decode_attention(p.opool, 0, p.tabs, lens1, 0, f32(q1), w.softmax_scale)
+    out1, _ = p.dc.decode(0, lens1, 0, q1, w.softmax_scale)
+    assert_attention_close(out1.cpu().numpy(), ref1, "after append")
+    p.lens = lens1
+    p.check_packed_equal()
+
+
+@pytest.mark.parametrize("name,lens,window", [
+    ("gqa64", [20, 9, 262], 0),
+    ("gqa64", [300, 17, 262], 12),
+    ("gqa128", [1000, 700, 1, 255, 256, 257], 0),
+    ("gqa128", [1000, 700, 33], 300),
+    ("gqa256", [1500, 40], 0),
+    ("gqa256", [1500, 1100], 1024),
+    ("mla", [600, 70], 0),
+    ("asym", [400, 300], 0),
+    ("asym", [400, 300], 100),
+])
+def test_decode_matches_oracle(H, name, lens, window):
+    p = Pair(H, SPECS[name], lens, seed=31).fill()
+    s = p.ospec
+    q = p.q(7, len(lens))
+    scale = 1.0 / math.sqrt(s.d_qk if name != "mla" else 192)
+    for l in range(s.n_layers):
+        ref, lse_ref = O.decode_attention(p.opool, l, p.tabs, lens, window, f32(q), scale)
+        out, lse = p.dc.decode(l, lens, window, q, scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"{name} layer {l}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref, name)
+    assert p.dc.read_flags() == 0
+
+
+def test_decode_shorter_lengths_than_cached_and_zero_length(H):
+    p = Pair(H, SPECS["gqa128"], [600, 300, 50], seed=32).fill()
+    q = p.q(7, 3)
+    lens = [257, 0, 1]
+    ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, 0, f32(q), 0.09)
+    out, lse = p.dc.decode(0, lens, 0, q, 0.09)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    assert torch.all(out[1] == 0)
+    # kv_len = 1: exactly the dequantized V row 0
+    _, V = O.gather_dequant(p.opool, 0, p.tabs[2], 0, 1, 1)
+    assert np.allclose(out[2, 7].cpu().numpy(), V[0], rtol=0, atol=1e-6)
+    assert p.dc.read_flags() == 0
+
+
+def test_batched_equals_per_agent_calls(H):
+    p = Pair(H, SPECS["gqa128"], [1000, 700, 256], seed=33).fill()
+    q = p.q(7, 3)
+    out, lse = p.dc.decode(1, p.lens, 0, q, 0.1)
+    qd = H.bf16_dev(q)
+    for a in range(3):
+        t, bt = p.dc.sub_batch(a, a + 1)
+        o1, l1 = p.dc.decode(1, p.lens[a:a + 1], 0, qd[a:a + 1].contiguous(), 0.1, bt=bt)
+        # the split schedule depends on the batch size, so equality is within tolerance, not bitwise
+        assert_attention_close(o1[0].cpu().numpy(), out[a].cpu().numpy().astype(np.float64), f"agent {a}")
+
+
+def test_one_hot_keys_select_one_value_row(H):
+    spec_args = (1, 2, 1, 64, 64, False)
+    p = Pair(H, spec_args, [40], seed=34)
+    perm = synth.rng(34, 0).permutation(64)[:40]
+    k = np.zeros((40, 1, 64), dtype=np.float32)
+    k[np.arange(40), 0, perm] = 7.5
+    kb = synth.f32_to_bf16_bits(k)
+    vb = synth.kv_bf16(34, 1, 40, 1, 64)
+    O.quantize_append(p.opool, 0, p.tabs, [0], [0, 40], f32(kb), f32(vb))
+    p.dc.append(0, [0], [0, 40], kb, vb)
+    _, Vd = O.gather_dequant(p.opool, 0, p.tabs[0], 0, 40, 0)
+    for m in (0, 13, 39):
+        q = np.zeros((1, 2, 64), dtype=np.float32)
+        q[0, :, perm[m]] = 16.0
+        out, lse = p.dc.decode(0, [40], 0, synth.f32_to_bf16_bits(q), 1.0)
+        assert np.max(np.abs(out[0, 1].cpu().numpy() - Vd[m])) <= 1e-5
+        assert abs(float(lse[0, 0]) - 120.0) < 1e-3
+
+
+def test_outlier_channels_large_values(H):
+    """Values up to ~8x3 sigma (the outlier-channel recipe) still meet the absolute bound."""
+    p = Pair(H, SPECS["gqa128"], [900, 400], seed=35)
+    s = p.ospec
+    for l in range(s.n_layers):
+        for a, n in enumerate(p.lens):
+            ko = synth.outlier_channels(35, 100 + l, s.n_kv_heads, s.d_qk)
+            vo = synth.outlier_channels(35, 200 + l, s.n_kv_heads, s.d_v)
+            kb = synth.kv_bf16(35, 1000 * l + 10 * a + 1, n, s.n_kv_heads, s.d_qk, ko)
+            vb = synth.kv_bf16(35, 1000 * l + 10 * a + 2, n, s.n_kv_heads, s.d_v, vo)
+            O.quantize_append(p.opool, l, p.tabs[a:a + 1], [0], [0, n], f32(kb), f32(vb))
+            t, bt = p.dc.sub_batch(a, a + 1)
+            p.dc.append(l, [0], [0, n], kb, vb, bt=bt)
+    p.check_packed_equal()
+    q = p.q(7, 2)
+    ref, _ = O.decode_attention(p.opool, 1, p.tabs, p.lens, 0, f32(q), 1 / math.sqrt(128))
+    out, _ = p.dc.decode(1, p.lens, 0, q, 1 / math.sqrt(128))
+    assert_attention_close(out.cpu().numpy(), ref)
+
+
+def test_bf16_output_mode(H):
+    from paper_2603_04428_b200 import binding as B
+    p = Pair(H, SPECS["gqa128"], [500, 300], seed=36).fill()
+    q = p.q(7, 2)
+    ref, _ = O.decode_attention(p.opool, 0, p.tabs, p.lens, 0, f32(q), 0.1)
+    out, _ = p.dc.decode(0, p.lens, 0, q, 0.1, out_dtype=B.OUT_BF16)
+    got = out.float().cpu().numpy().astype(np.float64)
+    ulp = np.maximum(np.abs(ref), 2.0 ** -126) * 2.0 ** -7      # one bf16 ulp is at most |x| * 2^-7
+    assert np.all(np.abs(got - ref) <= ulp + 1e-6)
+
+
+# ---- prefill attention --------------------------------------------------------------------------
+@pytest.mark.parametrize("name,prefix,chunk,window", [
+    ("gqa64", [300, 70], 40, 0),
+    ("gqa64", [300, 70], 40, 50),
+    ("gqa128", [512, 200], 130, 0),
+    ("gqa256", [256, 10], 70, 128),
+    ("mla", [200], 33, 0),
+])
+def test_prefill_matches_oracle_and_chunking_is_invisible(H, name, prefix, chunk, window):
+    lens = [n + chunk for n in prefix]
+    p = Pair(H, SPECS[name], lens, seed=41).fill(chunks=[max(prefix), chunk])
+    s = p.ospec
+    A = len(lens)
+    q_offs = [chunk * a for a in range(A + 1)]
+    q = p.q(7, chunk * A)
+    scale = 1.0 / math.sqrt(s.d_qk)
+    ref, lse_ref = O.prefill_attention(p.opool, 0, p.tabs, lens, q_offs, window, f32(q), scale)
+    out, lse = p.dc.prefill(0, lens, q_offs, window, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref, name)
+    assert_lse_close(lse.cpu().numpy(), lse_ref, name)
+    # second half alone, as its own chunk over the same cache: same rows
+    h = chunk // 2
+    rows = np.concatenate([np.arange(chunk * a + h, chunk * (a + 1)) for a in range(A)])
+    q2 = q[rows]
+    offs2 = [(chunk - h) * a for a in range(A + 1)]
+    out2, _ = p.dc.prefill(0, lens, offs2, window, q2, scale)
+    assert_attention_close(out2.cpu().numpy(), ref[rows], name + " second chunk")
+    assert p.dc.read_flags() == 0
+
+
+# ---- anomalies are reported, not faulted on -----------------------------------------------------
+def test_bad_block_id_and_bad_length_raise_flags_and_zero_output(H):
+    from paper_2603_04428_b200 import binding as B
+    p = Pair(H, SPECS["gqa64"], [300, 100], seed=51).fill()
+    q = p.q(7, 2)
+    good, _ = p.dc.decode(0, p.lens, 0, q, 0.1)
+    tabs = p.tabs.copy()
+    tabs[0, 1] = p.n_blocks + 7                     # outside the pool
+    t = H.dev(tabs)
+    out, _ = p.dc.decode(0, p.lens, 0, q, 0.1, bt=B.batch(t))
+    assert p.dc.read_flags() & B.FLAG_BAD_BLOCK
+    assert torch.all(out[0] == 0) and torch.equal(out[1], good[1])
+    p.dc.flags.zero_()
+    out, _ = p.dc.decode(0, [p.tabs.shape[1] * 256 + 1, 100], 0, q, 0.1)
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    assert torch.all(out[0] == 0) and torch.equal(out[1], good[1])
+    p.dc.flags.zero_()
+    out, _ = p.dc.decode(0, [-3, 100], 0, q, 0.1)
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    assert torch.all(out[0] == 0)
+
+
+def test_host_side_rejections(H):
+    from paper_2603_04428_b200 import binding as B
+    p = Pair(H, SPECS["gqa64"], [100], seed=52).fill()
+    bad = B.Spec.make(1, 4, 2, 96, 64)
+    assert B.q4kv_pool_bytes(bad, 4) == 0
+    with pytest.raises(B.Q4KVError) as e:
+        B.q4kv_decode_attention(bad, p.dc.pool, p.n_blocks, 0, p.dc.bt, p.dc.tables, 0, 0, p.dc.pool, 0.1, p.dc.pool,
+                                0, None, p.dc.pool, None)
+    assert e.value.code == B.EUNSUPPORTED
+    q = H.bf16_dev(p.q(7, 1))
+    out = torch.empty((1, 4, 64), device="cuda")
+    tiny = torch.empty(16, dtype=torch.uint8, device="cuda")
+    lens = H.dev(np.array([100], dtype=np.int32))
+    with pytest.raises(B.Q4KVError) as e:
+        B.q4kv_decode_attention(p.dc.spec, p.dc.pool, p.n_blocks, 0, p.dc.bt, lens, 0, 0, q, 0.1, out, 0, None, tiny)
+    assert e.value.code == B.EWORKSPACE
+    with pytest.raises(B.Q4KVError) as e:
+        B.q4kv_decode_attention(p.dc.spec, p.dc.pool, p.n_blocks, 5, p.dc.bt, lens, 0, 0, q, 0.1, out, 0, None, tiny)
+    assert e.value.code == B.EINVAL
+    dst = torch.empty(100, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.Q4KVError) as e:
+        B.q4kv_pack(p.dc.spec, p.dc.pool, p.n_blocks, p.dc.tables[0], 100, dst)
+    assert e.value.code == B.EWORKSPACE

@@ -1,0 +1,41 @@
+"""CPU-side checks of the boundary: the library builds, loads and exports what include/q4kv.h declares;
+the host-only size queries agree with the paper's byte counts.  No kernel is launched."""
+import ctypes
+import os
+import re
+
+from paper_2603_04428_b200 import build as qbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "q4kv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(q4kv_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    lib_path = qbuild.build()
+    lib = ctypes.CDLL(lib_path)
+    names = declared_symbols()
+    assert {"q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack",
+            "q4kv_unpack"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_lists_the_same_symbols_and_size_queries_match_the_paper():
+    from paper_2603_04428_b200 import binding as B
+    assert sorted(B.EXPORTS) == [n for n in declared_symbols()]
+    gemma = B.Spec.make(48, 16, 8, 256, 256)
+    assert B.q4kv_packed_bytes(gemma, 4096) == 48 * 9437184 == 432 * 2**20     # Appendix: 9,437,184 B per layer
+    llama = B.Spec.make(32, 32, 8, 128, 128)
+    assert B.q4kv_packed_bytes(llama, 4096) == 144 * 2**20
+    ds = B.Spec.make(27, 16, 16, 192, 128)
+    assert B.q4kv_packed_bytes(ds, 4096) == int(303.75 * 2**20)
+    assert B.q4kv_pool_bytes(gemma, 16) == B.q4kv_packed_bytes(gemma, 4096)   # same bytes, other arrangement
+    mla = B.Spec.make(27, 16, 1, 576, 512, True)
+    assert B.q4kv_packed_bytes(mla, 256) == 27 * 256 * 324
+    assert B.q4kv_pool_bytes(B.Spec.make(1, 4, 2, 96, 64), 4) == 0            # unsupported spec
+    assert B.status_string(B.EWORKSPACE)
