@@ -1,0 +1,487 @@
+#!/usr/bin/env python
+"""Benchmark of the Q4 KV-cache hot path on B200.
+
+Default workload: the Llama-3.1-8B-shaped batched decode step (32 layers, 5 agents x 4096 cached
+tokens, Q4 group-64 K and V in 256-token blocks): per layer, quantize-append one new K/V token per
+agent, then decode attention of one query per agent over the whole Q4 cache.  One "step" is all
+layers.  The metric is the achieved HBM bandwidth over the algorithmic bytes of the step (each
+needed Q4 row read once + q + out + new rows); agent-steps/s rides along.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4] [--impl reference]
+
+N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no collective.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_04428_b200 import synth  # noqa: E402
+
+
+# ------------------------------------------------------------------------------------------------
+# workload arithmetic (bytes / flops the roofline is quoted on)
+# ------------------------------------------------------------------------------------------------
+def row_bytes(w: synth.Workload) -> int:
+    """Bytes of one token's K and V rows over all KV heads."""
+    k = w.d_qk // 2 + 4 * (w.d_qk // 64)
+    v = 0 if w.v_aliases_k else w.d_v // 2 + 4 * (w.d_v // 64)
+    return w.n_kv_heads * (k + v)
+
+
+def decode_layer_bytes(w: synth.Workload, layer: int) -> int:
+    win = w.layer_window(layer)
+    toks = sum(min(n + w.new_tokens, win) if win else n + w.new_tokens for n in w.lens)
+    cache = toks * row_bytes(w)
+    q = w.n_agents * w.n_q_heads * w.d_qk * 2
+    out = w.n_agents * w.n_q_heads * w.d_v * 4
+    new_in = w.n_agents * w.new_tokens * w.n_kv_heads * (w.d_qk + (0 if w.v_aliases_k else w.d_v)) * 2
+    new_out = w.n_agents * w.new_tokens * row_bytes(w)
+    return cache + q + out + new_in + new_out
+
+
+def prefill_layer_flops(w: synth.Workload) -> float:
+    """4 * D * Hq * sum_i (P + i + 1) per agent (QK^T and PV, causal pairs only; D = d_qk = d_v)."""
+    fl = 0.0
+    for P in w.lens:
+        C = w.new_tokens
+        pairs = C * P + C * (C + 1) / 2
+        fl += 2.0 * w.n_q_heads * pairs * (w.d_qk + w.d_v)
+    return fl
+
+
+def workload_name(w: synth.Workload) -> str:
+    return w.name
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampling
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, c[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# device-side workload
+# ------------------------------------------------------------------------------------------------
+class DeviceWorkload:
+    """All state of one workload resident on the GPU: the Q4 pool (filled by the library's own quantizer
+    from seeded on-device N(0,1) bf16 values), block tables, per-layer q / new K,V, outputs."""
+
+    def __init__(self, w: synth.Workload, device_index: int):
+        import torch
+        from paper_2603_04428_b200 import binding as B, harness as H
+        self.torch, self.B, self.w = torch, B, w
+        torch.cuda.set_device(device_index)
+        A, L = w.n_agents, w.n_layers
+        self.n_blocks = w.blocks_needed() + 4
+        tabs = synth.block_tables(w.seed, 99, w.lens, self.n_blocks, extra_tokens=w.new_tokens)
+        self.dc = H.DeviceCache(L, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k, self.n_blocks, tabs,
+                                fill_byte=None)
+        dc = self.dc
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed)
+        self.lens0 = H.dev(np.asarray(w.lens, dtype=np.int32))
+        self.lens1 = H.dev(np.asarray([n + w.new_tokens for n in w.lens], dtype=np.int32))
+        self.max_kv = max(w.lens) + w.new_tokens
+        # ---- fill the cache: per layer, per agent (bounded temporaries) ----
+        zero = H.dev(np.zeros(1, dtype=np.int32))
+        for l in range(L):
+            ko = vo = None
+            if w.outlier_frac > 0:
+                ko = torch.from_numpy(synth.outlier_channels(w.seed, 100 + l, w.n_kv_heads, w.d_qk, w.outlier_frac)).cuda()
+                vo = torch.from_numpy(synth.outlier_channels(w.seed, 200 + l, w.n_kv_heads, w.d_v, w.outlier_frac)).cuda()
+            for a, n in enumerate(w.lens):
+                t, bt = dc.sub_batch(a, a + 1)
+                for c0 in range(0, n, 8192):
+                    c = min(8192, n - c0)
+                    k = torch.randn((c, w.n_kv_heads * w.d_qk), generator=g, device="cuda", dtype=torch.float32)
+                    if ko is not None:
+                        k[:, ko] *= 8.0
+                    k = k.to(torch.bfloat16).view(c, w.n_kv_heads, w.d_qk)
+                    v = None
+                    if not w.v_aliases_k:
+                        v = torch.randn((c, w.n_kv_heads * w.d_v), generator=g, device="cuda", dtype=torch.float32)
+                        if vo is not None:
+                            v[:, vo] *= 8.0
+                        v = v.to(torch.bfloat16).view(c, w.n_kv_heads, w.d_v)
+                    offs = H.dev(np.asarray([0, c], dtype=np.int32))
+                    pos = H.dev(np.asarray([c0], dtype=np.int32))
+                    dc.append(l, pos, offs, k, v, bt=bt)
+        # ---- per-step inputs and outputs ----
+        nq = A if w.kind == "decode" else A * w.new_tokens
+        self.q = torch.randn((L, nq, w.n_q_heads, w.d_qk), generator=g, device="cuda").to(torch.bfloat16)
+        self.k_new = torch.randn((L, A * w.new_tokens, w.n_kv_heads, w.d_qk), generator=g, device="cuda").to(torch.bfloat16)
+        self.v_new = None if w.v_aliases_k else torch.randn(
+            (L, A * w.new_tokens, w.n_kv_heads, w.d_v), generator=g, device="cuda").to(torch.bfloat16)
+        self.out = torch.empty((L, nq, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
+        self.new_offs = H.dev(np.arange(A + 1, dtype=np.int32) * w.new_tokens)
+        self.q_offs = self.new_offs
+        self.ws = torch.empty(max(B.q4kv_workspace_bytes(dc.spec, A, self.max_kv, 0),
+                                  B.q4kv_workspace_bytes(dc.spec, A, self.max_kv, nq)), dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()
+        assert dc.read_flags() == 0
+        self.launches_per_step = 0
+
+    # one layer of the step ----------------------------------------------------------------------
+    def append_layer(self, l):
+        w, dc, B = self.w, self.dc, self.B
+        B.q4kv_quantize_append(dc.spec, dc.pool, dc.n_blocks, l, dc.bt, self.lens0, self.new_offs,
+                               w.n_agents * w.new_tokens, self.k_new[l], None if self.v_new is None else self.v_new[l],
+                               dc.flags)
+
+    def attend_layer(self, l):
+        w, dc, B = self.w, self.dc, self.B
+        if w.kind == "decode":
+            B.q4kv_decode_attention(dc.spec, dc.pool, dc.n_blocks, l, dc.bt, self.lens1, self.max_kv,
+                                    w.layer_window(l), self.q[l], w.softmax_scale, self.out[l], B.OUT_F32, None,
+                                    self.ws, dc.flags)
+        else:
+            B.q4kv_prefill_attention(dc.spec, dc.pool, dc.n_blocks, l, dc.bt, self.lens1, self.q_offs,
+                                     w.n_agents * w.new_tokens, w.new_tokens, self.max_kv, w.layer_window(l),
+                                     self.q[l], w.softmax_scale, self.out[l], B.OUT_F32, None, self.ws, dc.flags)
+
+    def step(self):
+        for l in range(self.w.n_layers):
+            self.append_layer(l)
+            self.attend_layer(l)
+
+
+def time_region(torch, fn, iters):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / 1e3
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w: synth.Workload, budget_s: float = 12.0):
+    """Time the oracle on ONE layer of the workload restricted to a sample of agents: quantize-append of the
+    new tokens plus attention.  Returns (seconds per sample-step, bytes or flops covered, description, threads)."""
+    from oracle import q4kv_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    f32 = synth.bf16_bits_to_f32
+    spec = O.Spec(1, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k)
+    if w.kind == "decode":
+        # sample: the first agents until at least 12000 cached tokens
+        agents, tot = [], 0
+        for a, n in enumerate(w.lens):
+            agents.append(a)
+            tot += n
+            if tot >= 12000:
+                break
+        lens = [w.lens[a] for a in agents]
+    else:
+        agents, lens = [0], [w.lens[0]]
+    n_blocks = sum(-(-(n + w.new_tokens) // 256) for n in lens)
+    tabs = synth.block_tables(w.seed, 99, lens, n_blocks, extra_tokens=w.new_tokens)
+    pool = O.Pool(spec, n_blocks)
+    for i, n in enumerate(lens):
+        k = f32(synth.kv_bf16(w.seed, 10 * i + 1, n, w.n_kv_heads, w.d_qk))
+        v = None if w.v_aliases_k else f32(synth.kv_bf16(w.seed, 10 * i + 2, n, w.n_kv_heads, w.d_v))
+        O.quantize_append(pool, 0, tabs[i:i + 1], [0], [0, n], k, v)
+    A = len(lens)
+    kn = f32(synth.kv_bf16(w.seed, 501, A * w.new_tokens, w.n_kv_heads, w.d_qk))
+    vn = None if w.v_aliases_k else f32(synth.kv_bf16(w.seed, 502, A * w.new_tokens, w.n_kv_heads, w.d_v))
+    offs = [i * w.new_tokens for i in range(A + 1)]
+    lens1 = [n + w.new_tokens for n in lens]
+    if w.kind == "decode":
+        q = f32(synth.normal_bf16(w.seed, 7, (A, w.n_q_heads, w.d_qk)))
+        win = w.layer_window(w.n_layers - 1)          # a global layer when the model has them
+
+        def one():
+            O.quantize_append(pool, 0, tabs, lens, offs, kn, vn)
+            O.decode_attention(pool, 0, tabs, lens1, win, q, w.softmax_scale)
+        units = sum(lens1) * row_bytes(w)
+        desc = f"1 layer, agents {agents} of {w.n_agents} ({sum(lens1)} cached tokens), append + decode attention"
+    else:
+        rows = list(range(0, w.new_tokens, max(1, w.new_tokens // 16)))[:16]
+        q = f32(synth.normal_bf16(w.seed, 7, (w.new_tokens, w.n_q_heads, w.d_qk)))
+
+        def one():
+            O.quantize_append(pool, 0, tabs, lens, offs, kn, vn)
+            O.prefill_attention(pool, 0, tabs, lens1, offs, 0, q, w.softmax_scale, rows=rows)
+        units = sum(2.0 * w.n_q_heads * (lens[0] + r + 1) * (w.d_qk + w.d_v) for r in rows)
+        desc = f"1 layer, agent 0, append {w.new_tokens} tokens + {len(rows)} of {w.new_tokens} query rows"
+    t0 = time.perf_counter()
+    one()
+    dt = time.perf_counter() - t0
+    reps = 1
+    while (time.perf_counter() - t0) < budget_s and reps < 50:
+        one()
+        reps += 1
+    dt = (time.perf_counter() - t0) / reps
+    return dt, units, desc, threads
+
+
+def metric_of(w):
+    if w.kind == "decode":
+        return "q4_decode_step_hbm_gbps", "GB/s", 1e9
+    return "q4_prefix_chunked_prefill_tflops", "TFLOP/s", 1e12
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    metric, unit, div = metric_of(w)
+    times = []
+    desc, threads, units = "", 1, 0
+    for i in range(args.warmup + args.steps):
+        dt, units, desc, threads = oracle_sample(w, budget_s=0.0)
+        if i >= args.warmup:
+            times.append(dt)
+    t = float(np.mean(times))
+    val = units / t / div
+    line = {"impl": "reference", "metric": metric, "value": val, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(w), "sample": desc},
+            "cpu_baseline": {"value": val, "unit": unit, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return d.get("hbm_gbs", 6650.0), d.get("bf16_tflops", 1590.0), d.get("bf16_tflops_sustained", 1400.0), "measured"
+    return 6650.0, 1590.0, 1400.0, "fallback"
+
+
+# ncu DRAM traffic (read + write) per launch of the dominant kernel, from the committed profile summary
+NCU_TRAFFIC_BYTES = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=1, help="index into the five configurations (0-based); default 1")
+    ap.add_argument("--impl", default="q4kv", choices=["q4kv", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
+    w = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dw = DeviceWorkload(w, local)
+    metric, unit, div = metric_of(w)
+    L = w.n_layers
+
+    # ---- the step: eager or one CUDA graph replay ----
+    use_graph = not args.no_graph
+    stream = torch.cuda.Stream()
+    graph = None
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            dw.step()
+        stream.synchronize()
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                dw.step()
+        run = graph.replay if graph is not None else dw.step
+        for _ in range(args.warmup):
+            run()
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        torch.cuda.synchronize()
+        dt = time_region(torch, run, args.steps)
+        t_step = dt / args.steps
+        # ---- dominant kernel: per-launch duration with events around every attention call ----
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(L)]
+        att_ms = []
+        app_ms = []
+        for _ in range(max(2, min(args.steps, 5))):
+            for l in range(L):
+                dw.append_layer(l)
+                evs[l][0].record()
+                dw.attend_layer(l)
+                evs[l][1].record()
+            torch.cuda.synchronize()
+            att_ms.append([a.elapsed_time(b) for a, b in evs])
+        for _ in range(2):
+            for l in range(L):
+                evs[l][0].record()
+                dw.append_layer(l)
+                evs[l][1].record()
+                dw.attend_layer(l)
+            torch.cuda.synchronize()
+            app_ms.append([a.elapsed_time(b) for a, b in evs])
+        clocks = sampler.stop()
+        # ---- end to end through the C ABI with host buffers ----
+        hq = dw.q.cpu().pin_memory()
+        hk = dw.k_new.cpu().pin_memory()
+        hv = None if dw.v_new is None else dw.v_new.cpu().pin_memory()
+        hout = torch.empty(dw.out.shape, dtype=dw.out.dtype).pin_memory()
+
+        def e2e_step():
+            dw.q.copy_(hq, non_blocking=True)
+            dw.k_new.copy_(hk, non_blocking=True)
+            if hv is not None:
+                dw.v_new.copy_(hv, non_blocking=True)
+            run()
+            hout.copy_(dw.out, non_blocking=True)
+            stream.synchronize()
+        for _ in range(2):
+            e2e_step()
+        e2e_iters = max(3, min(args.steps, 10))
+        t_e2e = time_region(torch, e2e_step, e2e_iters) / e2e_iters
+        h2d = hq.numel() * 2 + hk.numel() * 2 + (0 if hv is None else hv.numel() * 2)
+        d2h = hout.numel() * 4
+    assert dw.dc.read_flags() == 0, "device status flags set during the benchmark"
+
+    if dist is not None:
+        tt = torch.tensor([t_step, t_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_step, t_e2e = float(tt[0]), float(tt[1])
+
+    hbm_peak, tf_burst, tf_sust, peak_kind = peaks()
+    att = np.asarray(att_ms)[1:] if len(att_ms) > 1 else np.asarray(att_ms)
+    app = np.asarray(app_ms)[1:] if len(app_ms) > 1 else np.asarray(app_ms)
+    att_avg_s = float(att.mean()) / 1e3
+    if w.kind == "decode":
+        step_units = float(sum(decode_layer_bytes(w, l) for l in range(L)))
+        launch_units = step_units / L
+        roof = {"bound": "hbm", "kernel": "q4kv_decode_attention (per-layer call)",
+                "achieved": launch_units / att_avg_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": peak_kind}
+        if w.window:
+            # window and global layers differ by ~9x in bytes: quote the global layers, which dominate the step
+            gl = [l for l in range(L) if w.layer_window(l) == 0]
+            roof["achieved"] = float(np.mean([decode_layer_bytes(w, l) for l in gl])) / (float(att[:, gl].mean()) / 1e3) / 1e9
+            roof["kernel"] += ", global layers"
+    else:
+        step_units = prefill_layer_flops(w) * L
+        launch_units = step_units / L
+        roof = {"bound": "tensor", "kernel": "q4kv_prefill_attention (per-layer call)",
+                "achieved": launch_units / att_avg_s / 1e12, "peak": tf_sust, "unit": "TFLOP/s", "peak_kind": peak_kind + " sustained bf16"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
+    roof["avg_launch_us"] = att_avg_s * 1e6
+    value = world * step_units / t_step / div
+    e2e_val = world * step_units / t_e2e / div
+
+    line = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u4 codes x int8 / f32" if w.kind == "decode" else "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(w), "layers": L, "agents": w.n_agents, "kv_lens": w.lens if len(set(w.lens)) > 1 else w.lens[0],
+                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "d_qk": w.d_qk, "d_v": w.d_v,
+                   "new_tokens_per_agent": w.new_tokens, "window": w.window,
+                   "l2": "inputs larger than L2: every step streams the whole multi-layer cache",
+                   "launch": "cuda graph replay of the L-layer step" if graph is not None else "eager",
+                   "multi_gpu": "replicas only"},
+        "agent_steps_per_s": world * w.n_agents / t_step,
+        "step_bytes" if w.kind == "decode" else "step_flops": step_units,
+        "append_avg_us": float(app.mean()) * 1e3,
+        "roofline": roof,
+        "e2e": {"value": e2e_val, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": t_e2e * 1e3},
+        "gpu_launches": dw_launches(w) * args.steps,
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        dt_o, units_o, desc, threads = oracle_sample(w)
+        line["cpu_baseline"] = {"value": units_o / dt_o / div, "unit": unit, "cores": threads, "kind": "oracle",
+                                "sample": desc, "seconds_per_sample": dt_o}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def dw_launches(w):
+    """Kernels of this library launched per step: per layer one quantize-append, one attention kernel and,
+    when the keys are split across CTAs, one merge kernel."""
+    per_layer = 2 + (1 if w.kind == "decode" else 0)
+    return per_layer * w.n_layers
+
+
+if __name__ == "__main__":
+    main()
