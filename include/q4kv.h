@@ -85,7 +85,8 @@ enum {
 };
 enum {
   Q4KV_FLAG_BAD_BLOCK = 1,   /* a block id outside [0, n_blocks)                                    */
-  Q4KV_FLAG_BAD_LENGTH = 2   /* a length or position negative or beyond max_blocks*256              */
+  Q4KV_FLAG_BAD_LENGTH = 2,  /* a length or position negative or beyond max_blocks*256              */
+  Q4KV_FLAG_INTERNAL = 4     /* a bounded wait inside a kernel ran out (the output is not valid)    */
 };
 enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
 

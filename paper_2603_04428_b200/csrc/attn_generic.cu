@@ -96,24 +96,25 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
     // one octet [o0, o0+8) lies inside one block
     const int blk = tables[(size_t)it.agent * max_blocks + (o0 >> 8)];
     if (blk < 0 || blk >= n_blocks) { bad_block = true; break; }
-    const uint8_t* hb = head_block(pool, y, layer, blk, hk);
     const int slot0 = o0 & 255;
+    const uint8_t* chunk = head_block(pool, y, layer, blk, hk) + (size_t)(slot0 >> 5) * y.chunk_bytes;
+    const int tau0 = slot0 & 31;
     const int tok = o0 + k;
     const bool valid = tok >= it.lo && tok < t1;
     // ---- dequantize this lane's quarter of row k, score from registers ----
     float s = 0.f;
     {
-      const uint32_t* kc = reinterpret_cast<const uint32_t*>(hb + y.off_kc) + (size_t)(slot0 + k) * kw + t * 2 * G;
-      const __half2* ksb = reinterpret_cast<const __half2*>(hb + y.off_ksb) + (size_t)(slot0 + k) * G;
+      const uint32_t* kc = reinterpret_cast<const uint32_t*>(chunk + y.off_kc);
+      const __half2* ksb = reinterpret_cast<const __half2*>(chunk + y.off_ksb);
       for (int p = 0; p < 2 * G; ++p) {
         const int gi = p >> 1, i2 = p & 1;
         const int w = 8 * gi + 4 * i2 + t;
         float sc = 0.f, bi = 0.f;
         uint32_t word = 0;
         if (valid) {
-          const float2 f = __half22float2(ksb[gi]);
+          const float2 f = __half22float2(ksb[sb_offset(tau0 + k, gi, G)]);
           sc = f.x; bi = f.y;
-          word = kc[p];
+          word = kc[k_word_offset(tau0 + k, w, G)];
         }
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -158,18 +159,18 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
         acc[i] = a;
       }
     } else {
-      const uint32_t* vc = reinterpret_cast<const uint32_t*>(hb + y.off_vc);
-      const __half2* vsb = reinterpret_cast<const __half2*>(hb + y.off_vsb) + (size_t)slot0 * y.Gv;
+      const uint32_t* vc = reinterpret_cast<const uint32_t*>(chunk + y.off_vc);
+      const __half2* vsb = reinterpret_cast<const __half2*>(chunk + y.off_vsb);
 #pragma unroll
       for (int i = 0; i < kMaxDvPerLane; ++i) {
         if (i >= nd) break;
         const int d = lane + 32 * i, gi = d >> 6;
-        const uint32_t word = vc[v_word_index(slot0, d, Dv)];
+        const uint32_t word = vc[v_word_offset(tau0 >> 3, d)];
         float a = acc[i] * corr;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           if (p[kk] != 0.f) {     // invalid tokens may hold garbage scale bits
-            const float2 f = __half22float2(vsb[kk * y.Gv + gi]);
+            const float2 f = __half22float2(vsb[sb_offset(tau0 + kk, gi, y.Gv)]);
             a = fmaf(p[kk], fmaf((float)((word >> (4 * kk)) & 15u), f.x, f.y), a);
           }
         }

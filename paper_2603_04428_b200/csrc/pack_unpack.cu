@@ -3,7 +3,7 @@
 // through one block-table row.
 //
 // One CTA handles one (layer, logical block, KV head).  K words only change position
-// inside their row; scale/bias pairs are split into two tensors; V codes are transposed
+// inside their 32-token chunk; scale/bias pairs are split into two tensors; V codes are transposed
 // between the pool's token-packed words and the persisted head-dim-packed words through a
 // shared-memory tile of one byte per code, 32 tokens at a time.
 #include "q4kv_layout.cuh"
@@ -48,14 +48,15 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
   const PersistedOffsets po = persisted_offsets(y);
   const int kw = y.D / 8, vw = y.Dv / 8;
 
-  // K codes: word permutation inside each row
+  // K codes: word permutation inside each chunk
   {
     uint32_t* pk = reinterpret_cast<uint32_t*>(pb + po.kc) + (size_t)hk * kBlockTokens * kw;
-    uint32_t* dk = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + y.off_kc);
     for (int i = threadIdx.x; i < kBlockTokens * kw; i += kThreads) {
       const int slot = i / kw, w = i % kw;
-      if (kPack) pk[i] = (slot < valid && !bad) ? dk[(size_t)slot * kw + k_phys_word(w, y.G)] : 0u;
-      else dk[(size_t)slot * kw + k_phys_word(w, y.G)] = pk[i];
+      uint32_t* dk = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + (size_t)(slot >> 5) * y.chunk_bytes + y.off_kc) +
+                                         k_word_offset(slot & 31, w, y.G);
+      if (kPack) pk[i] = (slot < valid && !bad) ? *dk : 0u;
+      else *dk = pk[i];
     }
   }
   // K and V scale / bias
@@ -63,33 +64,34 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
     const int G = which ? y.Gv : y.G;
     __half* ps = reinterpret_cast<__half*>(pb + (which ? po.vs : po.ks)) + (size_t)hk * kBlockTokens * G;
     __half* pbias = reinterpret_cast<__half*>(pb + (which ? po.vb : po.kb)) + (size_t)hk * kBlockTokens * G;
-    __half2* dsb = bad ? nullptr : reinterpret_cast<__half2*>(hb + (which ? y.off_vsb : y.off_ksb));
     for (int i = threadIdx.x; i < kBlockTokens * G; i += kThreads) {
-      const int slot = i / G;
+      const int slot = i / G, gi = i % G;
+      __half2* dsb = bad ? nullptr : reinterpret_cast<__half2*>(hb + (size_t)(slot >> 5) * y.chunk_bytes +
+                                                                  (which ? y.off_vsb : y.off_ksb)) +
+                                         sb_offset(slot & 31, gi, G);
       if (kPack) {
         __half2 v = __halves2half2(__ushort_as_half((unsigned short)0), __ushort_as_half((unsigned short)0));
-        if (slot < valid && !bad) v = dsb[i];
+        if (slot < valid && !bad) v = *dsb;
         ps[i] = __low2half(v);
         pbias[i] = __high2half(v);
       } else {
-        dsb[i] = __halves2half2(ps[i], pbias[i]);
+        *dsb = __halves2half2(ps[i], pbias[i]);
       }
     }
   }
   if (y.alias) return;
   // V codes: transpose 32 tokens at a time
   uint32_t* pv = reinterpret_cast<uint32_t*>(pb + po.vc) + (size_t)hk * kBlockTokens * vw;
-  uint32_t* dv = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + y.off_vc);
   const int words = 4 * y.Dv;   // words of one 32-token chunk in either layout (32*Dv/8)
   for (int c = 0; c < 8; ++c) {
+    uint32_t* dv = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + (size_t)c * y.chunk_bytes + y.off_vc);
     if (kPack) {
-      // pool word (d, t) -> tile[8t+k][d]
+      // pool word (element d, token octet o) -> tile[8o+k][d]
       for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int j = i & 3, t = (i >> 2) & 3, g = (i >> 4) & 7, J = i >> 7;
-        const int d = 32 * J + 8 * j + g;
-        const uint32_t w = bad ? 0u : dv[(size_t)c * words + i];
+        const int d = i >> 2, o = i & 3;
+        const uint32_t w = bad ? 0u : dv[v_word_offset(o, d)];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) tile[(8 * t + k) * y.Dv + d] = (w >> (4 * k)) & 15u;
+        for (int k = 0; k < 8; ++k) tile[(8 * o + k) * y.Dv + d] = (w >> (4 * k)) & 15u;
       }
       __syncthreads();
       for (int i = threadIdx.x; i < words; i += kThreads) {
@@ -111,12 +113,11 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
       }
       __syncthreads();
       for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int j = i & 3, t = (i >> 2) & 3, g = (i >> 4) & 7, J = i >> 7;
-        const int d = 32 * J + 8 * j + g;
+        const int d = i >> 2, o = i & 3;
         uint32_t w = 0;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) w |= (uint32_t)tile[(8 * t + k) * y.Dv + d] << (4 * k);
-        dv[(size_t)c * words + i] = w;
+        for (int k = 0; k < 8; ++k) w |= (uint32_t)tile[(8 * o + k) * y.Dv + d] << (4 * k);
+        dv[v_word_offset(o, d)] = w;
       }
       __syncthreads();
     }

@@ -1,23 +1,33 @@
 // Device-side layout of the Q4 block pool and small shared helpers.
 //
-// The pool's byte layout is private to this library (include/q4kv.h): it is arranged so
-// that the attention kernels' warp-level loads are contiguous 16-byte accesses and feed
-// integer tensor-core fragments without shuffles.  The persisted layout of Appendix A is
-// produced/consumed only by the pack/unpack kernels.
+// The pool's byte layout is private to this library (include/q4kv.h): it is arranged so that
+// (a) any run of 32-token chunks of one KV head is ONE contiguous byte range (one bulk copy
+// into shared memory), and (b) inside a chunk every warp-wide 16-byte shared-memory load is a
+// contiguous 512-byte line whose words land directly in the register slots of the
+// m16n8k16 tensor-core fragments (no shuffles, no bank conflicts).  The persisted layout of
+// Appendix A is produced/consumed only by the pack/unpack kernels.
 //
-// pool = [n_layers][n_blocks][n_kv_heads] "head-blocks"; one head-block holds 256 tokens of
-// one KV head of one layer:
+// pool = [n_layers][n_blocks][n_kv_heads] "head-blocks"; one head-block = 8 chunks; one chunk
+// holds 32 consecutive tokens of one KV head of one layer:
 //
-//   Kc  : [256 tokens][D/8 words] uint32.  A logical word w of a row holds head-dim elements
-//         8w..8w+7 (element k in bits [4k,4k+4)), w = 8*gi + 4*i2 + t with gi the 64-element
-//         group, i2 in {0,1}, t in 0..3.  Physical position inside the row:
-//             phys(w) = t*(2G) + 2*gi + i2          (G = D/64)
-//         so the words one lane of a 4-lane quad needs (fixed t, all gi, i2) are contiguous.
-//   Ksb : [256 tokens][G] half2 (x = scale, y = bias).
-//   Vc  : [8 chunks of 32 tokens][Dv/32][8 g][4 t][4 j] uint32, token-packed ("V transposed"):
-//         the word at (chunk c, J, g, t, j) belongs to head-dim element d = 32J + 8j + g and
-//         holds tokens 32c + 8t + k, k = 0..7, in bits [4k,4k+4).   (absent when V aliases K)
-//   Vsb : [256 tokens][Gv] half2 (scale, bias); groups are still along head_dim.
+//   chunk = [ Kc | Ksb | Vc | Vsb ]                       (Vc, Vsb absent when V aliases K)
+//
+// Names: chunk token tau in 0..31; fragment coordinates g = lane/4 (0..7), tid = lane%4.
+//
+//   Kc  : D/8 uint32 per token.  Logical word w holds head-dim elements 8w..8w+7 (element k in
+//         bits [4k,4k+4)), w = 8*gi + 4*i2 + tid (gi = 64-element group, i2 in {0,1}).  Token
+//         tau = 4*g + i belongs to key tile i (the 8 tokens 4g+i, g = 0..7).  A lane's 2G words
+//         p = 2*gi + i2 are cut in pieces of 4 words (16 bytes):
+//             word offset = i*64G + (p/4)*128 + (g*4 + tid)*pw + p%4,   pw = min(4, 2G - 4*(p/4))
+//         so one 16-byte load per lane (g, tid) fetches a whole piece of tile i for the warp.
+//   Ksb : G half2 (x = scale, y = bias) per token; token tau = 8*tid + 4*e + i sits at
+//             half2 offset = ((i*4 + tid)*2 + e)*G + gi
+//         (the two tokens a lane owns in the score fragment of tile i are adjacent).
+//   Vc  : token-packed ("V transposed"): one uint32 holds the codes of ONE head-dim element d
+//         for the 8 tokens 8*tid..8*tid+7 (token 8*tid+k in bits [4k,4k+4)).  With d = 16*mt + r,
+//             word offset = (((mt/2)*8 + r%8)*4 + tid)*4 + (mt%2)*2 + r/8
+//         so one 16-byte load per lane fetches rows g and g+8 of two 16-row value tiles.
+//   Vsb : Gv half2 per token, arranged like Ksb; groups are still along head_dim.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
@@ -30,13 +40,15 @@ namespace q4kv {
 
 constexpr int kBlockTokens = 256;
 constexpr int kGroup = 64;
+constexpr int kChunkTokens = 32;
+constexpr int kChunksPerBlock = kBlockTokens / kChunkTokens;
 
 struct Layout {
   int L, Hq, Hkv, D, Dv, G, Gv, alias, n_rep;
-  // byte offsets inside a head-block
-  uint32_t off_kc, off_ksb, off_vc, off_vsb, head_block_bytes;
+  // byte offsets inside a chunk
+  uint32_t off_kc, off_ksb, off_vc, off_vsb, chunk_bytes, head_block_bytes;
   uint64_t block_bytes;   // all KV heads
-  uint64_t layer_bytes;   // n_blocks * block_bytes (filled by make_layout with n_blocks)
+  uint64_t layer_bytes;   // n_blocks * block_bytes
 };
 
 __host__ __device__ inline Layout make_layout(const q4kv_spec& s, int n_blocks) {
@@ -45,10 +57,11 @@ __host__ __device__ inline Layout make_layout(const q4kv_spec& s, int n_blocks) 
   y.G = s.d_qk / kGroup; y.Gv = s.d_v / kGroup; y.alias = s.v_aliases_k ? 1 : 0;
   y.n_rep = s.n_q_heads / s.n_kv_heads;
   y.off_kc = 0;
-  y.off_ksb = kBlockTokens * (y.D / 2);
-  y.off_vc = y.off_ksb + kBlockTokens * 4 * y.G;
-  y.off_vsb = y.off_vc + (y.alias ? 0 : kBlockTokens * (y.Dv / 2));
-  y.head_block_bytes = y.off_vsb + (y.alias ? 0 : kBlockTokens * 4 * y.Gv);
+  y.off_ksb = kChunkTokens * (y.D / 2);
+  y.off_vc = y.off_ksb + kChunkTokens * 4 * y.G;
+  y.off_vsb = y.off_vc + (y.alias ? 0 : kChunkTokens * (y.Dv / 2));
+  y.chunk_bytes = y.off_vsb + (y.alias ? 0 : kChunkTokens * 4 * y.Gv);
+  y.head_block_bytes = kChunksPerBlock * y.chunk_bytes;
   y.block_bytes = (uint64_t)y.Hkv * y.head_block_bytes;
   y.layer_bytes = (uint64_t)n_blocks * y.block_bytes;
   return y;
@@ -59,19 +72,23 @@ __host__ __device__ inline uint64_t persisted_block_bytes(const Layout& y) {
   return (uint64_t)kBlockTokens * y.Hkv * (y.D / 2 + 4 * y.G + (y.alias ? 0 : (y.Dv / 2 + 4 * y.Gv)));
 }
 
-__host__ __device__ inline int k_phys_word(int w, int G) {
-  const int gi = w >> 3, i2 = (w >> 2) & 1, t = w & 3;
-  return t * (2 * G) + 2 * gi + i2;
+// uint32 offset inside a chunk's Kc of logical word w (elements 8w..8w+7) of chunk token tau
+__host__ __device__ inline int k_word_offset(int tau, int w, int G) {
+  const int i = tau & 3, g = tau >> 2;
+  const int gi = w >> 3, i2 = (w >> 2) & 1, tid = w & 3;
+  const int p = 2 * gi + i2, j = p >> 2;
+  const int rest = 2 * G - 4 * j, pw = rest < 4 ? rest : 4;
+  return i * 64 * G + j * 128 + (g * 4 + tid) * pw + (p & 3);
 }
-__host__ __device__ inline int k_logical_word(int p, int G) {
-  const int t = p / (2 * G), r = p % (2 * G);
-  return 8 * (r >> 1) + 4 * (r & 1) + t;
+// half2 offset inside a chunk's Ksb / Vsb of (chunk token tau, group gi)
+__host__ __device__ inline int sb_offset(int tau, int gi, int G) {
+  const int i = tau & 3, e = (tau >> 2) & 1, tid = tau >> 3;
+  return ((i * 4 + tid) * 2 + e) * G + gi;
 }
-// word index inside Vc of (token slot in block, head-dim element d)
-__host__ __device__ inline int v_word_index(int slot, int d, int Dv) {
-  const int c = slot >> 5, t = (slot >> 3) & 3;
-  const int J = d >> 5, j = (d >> 3) & 3, g = d & 7;
-  return (((c * (Dv >> 5) + J) * 8 + g) * 4 + t) * 4 + j;
+// uint32 offset inside a chunk's Vc of the word holding element d for token octet o (tokens 8o..8o+7)
+__host__ __device__ inline int v_word_offset(int o, int d) {
+  const int mt = d >> 4, r = d & 15;
+  return ((((mt >> 1) * 8 + (r & 7)) * 4 + o) * 4) + (mt & 1) * 2 + (r >> 3);
 }
 
 __device__ inline const uint8_t* head_block(const void* pool, const Layout& y, int layer, int block, int kv_head) {
@@ -104,5 +121,12 @@ cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_bl
                                      const int32_t* kv_lens, const int32_t* q_offs, int total_q, int max_q_len,
                                      int max_kv_len, int window, const void* q, float scale, void* out,
                                      int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
+
+// tensor-core decode path (GQA shapes with d_qk = d_v in {128, 256}, at most 4 query heads per KV head)
+bool decode_mma_supported(const Layout& y);
+size_t decode_mma_workspace_bytes(const Layout& y, int n_agents);
+cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                              const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
+                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
 
 }  // namespace q4kv

@@ -95,8 +95,9 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
   if (s_agent < 0) return;
   const int first = s_first_pos, cnt = s_count, row0 = s_row0;
   const int hk = blockIdx.y;
-  uint8_t* hb = head_block(pool, y, layer, s_block, hk);
-  const int slot0 = first & 255;
+  const int slot0 = first & 255;                      // the octet lies inside one 32-token chunk
+  uint8_t* chunk = head_block(pool, y, layer, s_block, hk) + (size_t)(slot0 >> 5) * y.chunk_bytes;
+  const int tau0 = slot0 & 31;
 
   // ---- K rows: items (token i, word w), eight lanes per group ------------------------------
   const int kw = y.D / 8;
@@ -112,9 +113,9 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
     }
     const QuantOut o = quantize_eight(x);
     if (live) {
-      const int slot = slot0 + i;
-      reinterpret_cast<uint32_t*>(hb + y.off_kc)[(size_t)slot * kw + k_phys_word(w, y.G)] = o.word;
-      if ((w & 7) == 0) reinterpret_cast<__half2*>(hb + y.off_ksb)[(size_t)slot * y.G + (w >> 3)] = o.sb;
+      const int tau = tau0 + i;
+      reinterpret_cast<uint32_t*>(chunk + y.off_kc)[k_word_offset(tau, w, y.G)] = o.word;
+      if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_ksb)[sb_offset(tau, w >> 3, y.G)] = o.sb;
     }
   }
   if (y.alias) return;
@@ -133,21 +134,21 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
     }
     const QuantOut o = quantize_eight(x);
     if (live) {
-      const int slot = slot0 + i;
+      const int tau = tau0 + i;
 #pragma unroll
       for (int e = 0; e < 8; ++e) vcodes[i * y.Dv + 8 * w + e] = (o.word >> (4 * e)) & 15u;
-      if ((w & 7) == 0) reinterpret_cast<__half2*>(hb + y.off_vsb)[(size_t)slot * y.Gv + (w >> 3)] = o.sb;
+      if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_vsb)[sb_offset(tau, w >> 3, y.Gv)] = o.sb;
     }
   }
   __syncthreads();
   const int k0 = first & 7;                 // nibble of the first new token inside the word
   uint32_t mask = 0;
   for (int i = 0; i < cnt; ++i) mask |= 15u << (4 * (k0 + i));
-  uint32_t* vc = reinterpret_cast<uint32_t*>(hb + y.off_vc);
+  uint32_t* vc = reinterpret_cast<uint32_t*>(chunk + y.off_vc);
   for (int d = threadIdx.x; d < y.Dv; d += kThreads) {
     uint32_t bits = 0;
     for (int i = 0; i < cnt; ++i) bits |= (uint32_t)vcodes[i * y.Dv + d] << (4 * (k0 + i));
-    const int wi = v_word_index(slot0, d, y.Dv);
+    const int wi = v_word_offset(tau0 >> 3, d);
     vc[wi] = (mask == 0xffffffffu) ? bits : ((vc[wi] & ~mask) | bits);
   }
 }
