@@ -134,6 +134,30 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
                           void* workspace, size_t workspace_bytes,
                           int32_t* status_flags, void* stream);
 
+/* Decode attention without a caller-supplied workspace.  The paper has no counterpart: this entry
+ * point exists for hosts that cannot allocate device memory when they call -- a runtime that
+ * carved up all of its device memory at start-up, a plugin that must not touch its host's
+ * memory pool, code that runs where allocation calls are not allowed.  It computes exactly what
+ * q4kv_decode_attention computes (same arguments, minus workspace and workspace_bytes), with the
+ * split partials kept in a fixed array inside the library's device image instead.
+ *   - The array is Q4KV_STATIC_SCRATCH_BYTES long.  Every GPU on which the library is loaded
+ *     holds that much memory until the process exits, whether or not this entry point is used.
+ *   - A batch whose q4kv_workspace_bytes(spec, n_agents, max_kv_len, 0) exceeds the array is
+ *     rejected with Q4KV_EWORKSPACE and nothing is launched; use q4kv_decode_attention then.
+ *   - No call allocates or frees anything (no cudaMalloc, no cudaFree, no library that would).
+ *     The first call on each device looks up the array's device address (a host-side query, no
+ *     launch); make that first call before any stream capture begins on that device.
+ *   - All calls on one device share the one array, and it keeps whatever the last call left in
+ *     it (no call depends on those contents).  Two calls that overlap on the GPU -- different
+ *     streams, or one stream per thread -- race on it and give wrong results: order them on one
+ *     stream, or give the concurrent ones their own workspace through q4kv_decode_attention. */
+#define Q4KV_STATIC_SCRATCH_BYTES (8u << 20)
+int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
+                                 const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                                 int32_t window, const void* q, float softmax_scale,
+                                 void* out, int32_t out_dtype, float* lse,
+                                 int32_t* status_flags, void* stream);
+
 /* Chunked-prefill attention (Sections 3.4, 3.5): the new phase's queries over the cached Q4
  * prefix plus the causal new tokens, which must already have been appended (they are read
  * back in quantized form, so the result does not depend on the chunk size).
