@@ -125,7 +125,10 @@ int q4kv_quantize_append(const q4kv_spec* spec, void* pool, int32_t n_blocks, in
  *   q          bf16 [A][n_q_heads][d_qk]
  *   out        [A][n_q_heads][d_v], float32 or bf16 per out_dtype
  *   lse        optional float32 [A][n_q_heads], natural-log sum of exponentials; may be NULL
- *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, 0) bytes
+ *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, 0) bytes.  Fill it with zero bytes once
+ *              after allocating it: its head holds the arrival counters of the split merge, which
+ *              every call finds at zero and leaves at zero.  (If a call ever reports
+ *              Q4KV_FLAG_INTERNAL, zero it again.)  Nothing else in it carries over between calls.
  * kv_len == 0 gives zeros and lse = -inf without a flag. */
 int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                           const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,

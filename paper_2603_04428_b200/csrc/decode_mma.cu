@@ -5,39 +5,49 @@
 //
 // The kernel is bound by HBM bandwidth, so it is organised around the byte stream:
 //   * Work = the flattened list of 32-token chunks of all (agent, KV head) pairs inside their key
-//     range [lo, kv_len).  The list is cut into equal contiguous ranges, one per persistent CTA,
-//     so ragged lengths balance by construction.  A CTA's range may cover parts of several
-//     pairs ("segments"); per segment it writes one partial (m, l, acc) record and a small
-//     second kernel combines the records of each pair.
+//     range [lo, kv_len).  The list is cut into equal contiguous ranges, one per persistent CTA
+//     (one CTA per SM), so ragged lengths balance by construction.  A CTA's range may cover
+//     parts of several pairs ("segments").  A pair that lies inside one CTA is finished there;
+//     otherwise every CTA that holds a piece writes a partial (m, l, acc) record and takes a
+//     ticket, and the CTA that draws the last ticket combines the records -- one launch, no
+//     waiting on other CTAs.
 //   * A producer warp streams the CTA's chunks through a shared-memory ring with one bulk
 //     asynchronous copy per chunk (a chunk is one contiguous byte range of the pool) completing
-//     on an mbarrier; four consumer warps take chunks round-robin.
+//     on an mbarrier.  The consumer warps run independently of one another: each claims the next
+//     chunk from a shared counter, keeps its own online-softmax state, and on leaving a segment
+//     deposits that state in shared memory; the warp that makes the deposit count complete
+//     combines the deposits and does the segment's epilogue (output, or record + ticket) while
+//     the others are already working on the next segment.  No CTA-wide barrier after start-up.
 //   * Arithmetic runs on the 4-bit codes, not on dequantized values.  With x^ = c*s + b and one
 //     (s, b) per token and 64-element group,
 //         q.k_t   = sum_g [ s_tg * (sum_{d in g} q_d c_td) + b_tg * (sum_{d in g} q_d) ]
-//         (p.V)_d = sum_t (p_t s_tg(d)) c_td + sum_t p_t b_tg(d),
-//     so both contractions are mma.sync m16n8k16 (f16 in, f32 accumulate) whose code operand is
-//     produced by masking the packed word: a nibble in the low bits of a 16-bit lane is the
-//     binary16 subnormal c * 2^-24 (or 16c * 2^-24 one nibble higher; the 16 is folded into the
-//     other operand), which the tensor cores multiply exactly.  Cost: 5 logic ops per 8 codes.
-//   * Scores come out as [8 query rows x 8 tokens] fragments whose lane ownership is exactly the
-//     B-operand ownership of the P.V product, so probabilities never move between lanes.  Rows
-//     4..7 repeat the (at most four) query heads: they carry the low half of a two-term binary16
-//     split of p*s, which makes the value product accurate to ~2^-22 at no extra MMA.
+//         (p.V)_d = sum_t (p_t s_tg(d)) c_td + sum_t p_t b_tg(d).
+//     Both contractions run on the tensor cores with the code operand produced by masking the
+//     packed word in place:
+//       - q.K: mma.sync m16n8k32 e4m3.  A byte holding a code c in 0..15 IS the e4m3 number
+//         c * 2^-9 (the first normal binade continues the subnormal spacing), so two masks turn a
+//         word into the B operand.  The bf16 query is split exactly into two e4m3 terms
+//         (4 + 4 significant bits) that occupy different rows of the A operand.
+//       - p.V: mma.sync m16n8k16 f16.  A nibble in the low bits of a 16-bit lane is the binary16
+//         subnormal c * 2^-24 (16c * 2^-24 one nibble up; the 16 is folded into p).
+//     Both forms multiply exactly and at full rate on sm_100a.
+//   * Scores come out as [8 rows x 8 tokens] fragments whose lane ownership is the B-operand
+//     ownership of the P.V product, so probabilities never move between lanes.  Rows 0..3 are
+//     the query heads (first e4m3 term), rows 4..7 the same heads (second term); after one
+//     shuffle both hold the full score, and rows 4..7 go on to carry the low half of a two-term
+//     binary16 split of p*s, which makes the value product accurate to ~2^-22 at no extra MMA.
+#include <cstdlib>
+
 #include "q4kv_layout.cuh"
 
 namespace q4kv {
 
 namespace {
 
-constexpr int kConsumerWarps = 4;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;       // + one producer warp
-constexpr int kCtasPerSm = 2;
-constexpr int kRingBytes = 73728;                      // 16 chunks at d = 128, 8 at d = 256
+constexpr int kMaxCtas = 148;                          // one persistent CTA per SM
 constexpr uint32_t kSpinLimit = 1u << 22;              // bounded mbarrier waits (each try blocks a while in hardware)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u;
+constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u, kMaskB = 0x0F0F0F0Fu;
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -73,18 +83,32 @@ __device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* a
   *abort_flag = 1;
   return false;
 }
+// Bounded spin on a shared-memory word until it reaches `want`.
+__device__ inline bool spin_until_ge(volatile int* word, int want, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
+    if (*word >= want) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
 __device__ inline void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_u32(dst_smem)),
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-__device__ inline void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+__device__ inline void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-__device__ inline void mma16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+// D = A(16x32 e4m3, rows 8..15 zero) * B(32x8 e4m3) + C; only rows 0..7 of D are meaningful
+__device__ inline void mma_e4m3(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1, const float (&c)[4]) {
+  asm("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+__device__ inline void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -93,8 +117,24 @@ __device__ inline float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
-__device__ inline uint32_t h2_bits(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ inline float2 h2_to_f2(uint32_t u) { return __half22float2(*reinterpret_cast<__half2*>(&u)); }
+// half2(lo = a, hi = b), both rounded toward zero
+__device__ inline uint32_t f32x2_to_h2_rz(float a, float b) {
+  uint32_t r;
+  asm("cvt.rz.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+  return r;
+}
+// one float -> e4m3 byte (round to nearest, saturating)
+__device__ inline uint32_t f32_to_e4m3(float x) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(x));
+  return (uint32_t)(r & 0xffu);
+}
+__device__ inline float e4m3_to_f32(uint32_t b) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)b));
+  return __low2float(*reinterpret_cast<__half2*>(&h2));
+}
 
 // ---------------------------------------------------------------------------------------------
 // Work list: chunks of all (agent, KV head) pairs, agent-major, then head, then chunk
@@ -113,85 +153,124 @@ __device__ inline AgentRange agent_range(const int32_t* __restrict__ kv_lens, in
   return r;
 }
 
-// Warp-cooperative pass over the agents.  Returns the total number of units; when `want` >= 0
-// also locates the agent containing unit `want` (agent index, first unit of that agent).
-__device__ inline long long scan_units(const int32_t* __restrict__ kv_lens, int n_agents, int Hkv, int window,
-                                       int max_blocks, long long want, int& agent, long long& agent_start,
-                                       bool& any_bad) {
+// Equal partition of U units over n CTAs (all quantities fit 31 bits; the host checks):
+// the first U % n CTAs own U / n + 1 units, the others U / n.  Requires n <= U.
+struct Partition {
+  uint32_t U, n, q, r;
+  __device__ void init(uint32_t U_, uint32_t n_) { U = U_; n = n_; q = U_ / n_; r = U_ - q * n_; }
+  __device__ uint32_t begin(uint32_t c) const { return c * q + (c < r ? c : r); }
+  __device__ int cta_of(uint32_t u) const {
+    const uint32_t big = r * (q + 1);
+    return u < big ? (int)(u / (q + 1)) : (int)(r + (u - big) / q);
+  }
+};
+
+// Warp-cooperative: total number of units U, this CTA's range and the agent that contains its
+// first unit.  One pass over the agents when there are at most 32 of them.
+struct RangeStart { uint32_t U, u_begin, u_end, agent_start; int n_ctas, agent; bool any_bad; Partition part; };
+
+__device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int n_agents, int Hkv, int window,
+                                        int max_blocks, int cta, int grid) {
   const int lane = threadIdx.x & 31;
-  long long cum = 0;
-  agent = -1;
-  agent_start = 0;
-  any_bad = false;
+  RangeStart rs;
+  rs.any_bad = false;
+  rs.agent = -1;
+  rs.agent_start = 0;
+  uint32_t cum = 0, inc0 = 0, cnt0 = 0;
   for (int base = 0; base < n_agents; base += 32) {
     const int a = base + lane;
-    long long cnt = 0;
+    uint32_t cnt = 0;
     bool bad = false;
-    if (a < n_agents) cnt = (long long)agent_range(kv_lens, a, window, max_blocks, bad).nc * Hkv;
-    any_bad |= __any_sync(0xffffffffu, bad);
-    long long inc = cnt;
+    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, max_blocks, bad).nc * Hkv);
+    rs.any_bad |= __any_sync(0xffffffffu, bad);
+    uint32_t inc = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const long long v = __shfl_up_sync(0xffffffffu, inc, o);
+      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
       if (lane >= o) inc += v;
     }
-    const long long tot = __shfl_sync(0xffffffffu, inc, 31);
-    if (agent < 0 && want >= 0 && want < cum + tot) {
+    if (base == 0) { inc0 = inc; cnt0 = cnt; }
+    cum += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  rs.U = cum;
+  rs.n_ctas = (uint32_t)grid < cum ? grid : (int)cum;
+  rs.u_begin = rs.u_end = 0;
+  rs.part.U = 0; rs.part.n = 1; rs.part.q = 0; rs.part.r = 0;
+  if (cum == 0 || cta >= rs.n_ctas) return rs;
+  rs.part.init(cum, (uint32_t)rs.n_ctas);
+  rs.u_begin = rs.part.begin(cta);
+  rs.u_end = rs.part.begin(cta + 1);
+  const uint32_t want = rs.u_begin;
+  if (n_agents <= 32) {
+    const unsigned bal = __ballot_sync(0xffffffffu, inc0 > want);
+    const int l = __ffs(bal) - 1;
+    rs.agent = l;
+    rs.agent_start = __shfl_sync(0xffffffffu, inc0, l) - __shfl_sync(0xffffffffu, cnt0, l);
+    return rs;
+  }
+  cum = 0;
+  for (int base = 0; base < n_agents; base += 32) {
+    const int a = base + lane;
+    uint32_t cnt = 0;
+    bool bad = false;
+    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, max_blocks, bad).nc * Hkv);
+    uint32_t inc = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    const uint32_t tot = __shfl_sync(0xffffffffu, inc, 31);
+    if (want < cum + tot) {
       const unsigned bal = __ballot_sync(0xffffffffu, cum + inc > want);
       const int l = __ffs(bal) - 1;
-      agent = base + l;
-      agent_start = cum + __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, cnt, l);
+      rs.agent = base + l;
+      rs.agent_start = cum + __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, cnt, l);
+      return rs;
     }
     cum += tot;
   }
-  return cum;
-}
-
-__device__ inline long long range_begin(long long U, int c, int n_ctas) { return U * c / n_ctas; }
-__device__ inline int cta_of_unit(long long U, long long u, int n_ctas) {
-  int c = (int)(u * n_ctas / U);
-  while (c + 1 < n_ctas && range_begin(U, c + 1, n_ctas) <= u) ++c;
-  return c;
+  return rs;
 }
 
 // One segment: the part of pair (agent a, KV head hk) inside this CTA's unit range.
 struct Segment {
   int a, hk, c0, c1;      // logical chunk indices [c0, c1) of the agent
   int n, lo;              // key range of the agent
-  long long k0;           // running chunk counter of the CTA at c0
-  long long u0;           // global unit index at c0
-  bool first_of_pair;     // c0 is the pair's first chunk
+  int cf, nc;             // the pair's whole chunk range
+  int k0;                 // running chunk counter of the CTA at c0
+  uint32_t u0;            // global unit index at c0
 };
 
 struct Walker {
   const int32_t* kv_lens;
   int n_agents, Hkv, window, max_blocks;
-  long long u, u_end, k;
-  int a, hk, c;
+  uint32_t u, u_end;
+  int k, a, hk, c;
   AgentRange r;
 
-  __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int max_blocks_, long long u_begin,
-                       long long u_end_, int agent, long long agent_start) {
+  __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int max_blocks_,
+                       const RangeStart& rs) {
     kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; max_blocks = max_blocks_;
-    u = u_begin; u_end = u_end_; k = 0;
-    a = agent;
+    u = rs.u_begin; u_end = rs.u_end; k = 0;
+    a = rs.agent; hk = 0; c = 0;
+    r.n = 0; r.lo = 0; r.cf = 0; r.nc = 0;
     if (u < u_end && a >= 0) {
       bool bad;
       r = agent_range(kv_lens, a, window, max_blocks, bad);
-      const long long rem = u - agent_start;
-      hk = (int)(rem / r.nc);
-      c = r.cf + (int)(rem % r.nc);
+      const uint32_t rem = u - rs.agent_start;
+      hk = (int)(rem / (uint32_t)r.nc);
+      c = r.cf + (int)(rem - (uint32_t)hk * (uint32_t)r.nc);
     }
   }
   __device__ bool next(Segment& s) {
     if (u >= u_end || a < 0) return false;
     const int pair_end = r.cf + r.nc;
-    const long long left = u_end - u;
-    const int c1 = (long long)(pair_end - c) <= left ? pair_end : c + (int)left;
-    s.a = a; s.hk = hk; s.c0 = c; s.c1 = c1; s.n = r.n; s.lo = r.lo; s.k0 = k; s.u0 = u;
-    s.first_of_pair = (c == r.cf);
+    const uint32_t left = u_end - u;
+    const int c1 = (uint32_t)(pair_end - c) <= left ? pair_end : c + (int)left;
+    s.a = a; s.hk = hk; s.c0 = c; s.c1 = c1; s.n = r.n; s.lo = r.lo; s.cf = r.cf; s.nc = r.nc; s.k0 = k; s.u0 = u;
     const int cnt = c1 - c;
-    u += cnt; k += cnt;
+    u += (uint32_t)cnt; k += cnt;
     if (c1 == pair_end) {
       ++hk;
       if (hk == Hkv) {
@@ -223,32 +302,405 @@ struct DecodeParams {
   int window;
   const uint16_t* q;          // bf16 [A][Hq][D]
   float scale_log2;           // softmax_scale * log2(e)
-  int2* desc;                 // [A*Hkv] (first CTA, last CTA) of each non-empty pair
-  float* partials;            // [A*Hkv + n_ctas][n_rep][Dv + 2]
+  int32_t* tickets;           // [A*Hkv], zero between calls
+  float* partials;            // [A*Hkv + kMaxCtas][n_rep][Dv + 2]
+  void* out;
+  int out_dtype;
+  float* lse;
   int32_t* flags;
 };
 
-template <int G>
+constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
+constexpr int kMBufs = 2;      // deposit buffers
+
+template <int G, int NW>
 struct Smem {
   static constexpr int D = 64 * G;
   static constexpr int kChunkBytes = 32 * (D / 2 + 4 * G) * 2;
-  static constexpr int kSlots = kRingBytes / kChunkBytes;
+  static constexpr int kSlots = (G == 2 ? 147456 : 110592) / kChunkBytes;   // 32 chunks at d = 128, 12 at d = 256
   static constexpr int kMergeStride = D + 8;            // acc[Dv], m, l, bias[Gv], pad
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
+  alignas(16) float merge[kMBufs][NW][4][kMergeStride];
+  alignas(16) uint32_t qfrag[kQBufs][8][4][4 * G];      // [buffer][row][tid][A-operand registers of the lane]
+  float qsum[kQBufs][4][G];                             // scale_log2 * sum of the true q over each group
+  float kappa[kQBufs][4];                               // scale_log2 * 2^(ex + 2)
   alignas(8) uint64_t full[kSlots];
   uint64_t empty[kSlots];
   int bad[kSlots];
+  int q_tag[kQBufs];            // s + 1 once the query of segment s is staged in buffer s % kQBufs
+  int deposits[kMBufs];         // running count of deposits into each buffer
+  int epilogues[kMBufs];        // number of completed epilogues of each buffer
+  int next_chunk;               // claim counter
   int abort_flag;
-  alignas(16) __half qh[4][D];          // normalized query rows (odd dims pre-divided by 16)
-  float qsum[4][G];                     // scale_log2 * sum of the true q over each group
-  float kappa[4];                       // scale_log2 * 2^(24 + E - 10)
-  alignas(16) float merge[kConsumerWarps][4][kMergeStride];
 };
 
+// Online-softmax state of one warp for one segment (fragment layout, see the header comment).
 template <int G>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_mma_kernel(const DecodeParams P) {
+struct WarpState {
+  float m, l_e, l_o, bias_e[G], bias_o[G];
+  float o[4 * G][4];
+  __device__ void reset() {
+    m = -INFINITY; l_e = 0.f; l_o = 0.f;
+#pragma unroll
+    for (int i = 0; i < G; ++i) { bias_e[i] = 0.f; bias_o[i] = 0.f; }
+#pragma unroll
+    for (int i = 0; i < 4 * G; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
+  }
+};
+
+// Warp-level: stage the query rows of one pair as two e4m3 terms in A-fragment order, plus the
+// per-group sums of the true query and the per-head factor that undoes the normalisation.
+// Element d = 8w + n of a row, w = 8*gi + 4*i2 + t: register (2*gi + i2)*2 + (n & 1) of lane t, byte n >> 1.
+template <int G>
+__device__ __noinline__ void stage_query(uint32_t (*qfrag)[4][4 * G], float (*qsum)[G], float* kappa,
+                                         const uint16_t* __restrict__ q, int Hq, int n_rep, float scale_log2, int a,
+                                         int hk, int lane) {
+  constexpr int D = 64 * G;
+  for (int base = 0; base < n_rep * (D / 8); base += 32) {
+    const int idx = base + lane;
+    const bool valid = idx < n_rep * (D / 8);
+    const int h = valid ? idx / (D / 8) : 0, w = idx % (D / 8);
+    const uint16_t* qrow = q + ((size_t)a * Hq + (size_t)hk * n_rep + h) * D;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) v = *reinterpret_cast<const uint4*>(qrow + 8 * w);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(u[i] << 16); x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
+    // row maximum and group sums: the D/8 lanes of a row are consecutive (16 or 32)
+    float mx = 0.f, sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { mx = fmaxf(mx, fabsf(x[i])); sum += x[i]; }
+#pragma unroll
+    for (int o = D / 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);   // 8 words per group
+    if (!valid) continue;
+    int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
+    if (mx == 0.f) ex = 0;
+    ex = min(max(ex, -100), 100);
+    const float sf = __uint_as_float((uint32_t)(127 + 7 - ex) << 23);          // 2^(7 - ex): |q| * sf < 256
+    uint32_t r1a = 0u, r1b = 0u, r2a = 0u, r2b = 0u;    // even / odd elements -> two registers
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const float qn = x[n] * sf;
+      const uint32_t b1 = f32_to_e4m3(qn);
+      const uint32_t b2 = f32_to_e4m3(qn - e4m3_to_f32(b1));
+      if (n & 1) { r1b |= b1 << (8 * (n >> 1)); r2b |= b2 << (8 * (n >> 1)); }
+      else { r1a |= b1 << (8 * (n >> 1)); r2a |= b2 << (8 * (n >> 1)); }
+    }
+    const int gi = w >> 3, i2 = (w >> 2) & 1, t = w & 3;
+    const int reg = (2 * gi + i2) * 2;
+    *reinterpret_cast<uint2*>(&qfrag[h][t][reg]) = make_uint2(r1a, r1b);
+    *reinterpret_cast<uint2*>(&qfrag[h + 4][t][reg]) = make_uint2(r2a, r2b);
+    if ((w & 7) == 0) qsum[h][gi] = sum * scale_log2;
+    if (w == 0) kappa[h] = scale_log2 * __uint_as_float((uint32_t)(127 + 2 + ex) << 23);   // 2^(9 + ex - 7)
+  }
+}
+
+// One 32-token chunk against this warp's query fragments.
+template <int G>
+__device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
+                                              const uint32_t (&qa)[4 * G], const float (&qs)[G], float kap,
+                                              uint32_t split_mask, WarpState<G>& st) {
   constexpr int D = 64 * G, Dv = D, Gv = G;
-  using S = Smem<G>;
+  const uint4* kc4 = reinterpret_cast<const uint4*>(chunk);
+  const uint4* ksb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2));
+  const uint4* vc4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G);
+  const uint4* vsb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G + 32 * (Dv / 2));
+  const bool edge = pos0 < key_lo || pos0 + 32 > key_n;
+
+  // ---- scores of the 4 key tiles: s2[i][e] for token 8*tid + 4*e + i, in log2 units ----
+  float s2[4][2];
+  {
+    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+    float t[4][2];
+#pragma unroll
+    for (int half = 0; half < G / 2; ++half) {        // groups 2*half, 2*half+1
+      uint4 kw[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) kw[i] = kc4[((i * (G / 2) + half) * 8 + g) * 4 + tid];
+      float acc[4][2][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t w[4] = {kw[i].x, kw[i].y, kw[i].z, kw[i].w};
+#pragma unroll
+        for (int gg = 0; gg < 2; ++gg) {
+          const int r = (2 * (2 * half + gg)) * 2;      // registers of word (gi, i2 = 0)
+          mma_e4m3(acc[i][gg], qa[r], qa[r + 1], w[2 * gg] & kMaskB, (w[2 * gg] >> 4) & kMaskB, zero);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t w[4] = {kw[i].x, kw[i].y, kw[i].z, kw[i].w};
+#pragma unroll
+        for (int gg = 0; gg < 2; ++gg) {
+          const int r = (2 * (2 * half + gg) + 1) * 2;  // registers of word (gi, i2 = 1)
+          mma_e4m3(acc[i][gg], qa[r], qa[r + 1], w[2 * gg + 1] & kMaskB, (w[2 * gg + 1] >> 4) & kMaskB, acc[i][gg]);
+        }
+      }
+      // scale of the two tokens this lane owns in each tile
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (G == 2) {
+          const uint4 sb = ksb4[i * 4 + tid];
+          const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
+          t[i][0] = fmaf(acc[i][1][0], a1.x, acc[i][0][0] * a0.x);
+          t[i][1] = fmaf(acc[i][1][1], b1.x, acc[i][0][1] * b0.x);
+          s2[i][0] = fmaf(qs[1], a1.y, qs[0] * a0.y);
+          s2[i][1] = fmaf(qs[1], b1.y, qs[0] * b0.y);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const uint4 sb = ksb4[(i * 4 + tid) * 2 + e];
+            const float2 f0 = h2_to_f2(half == 0 ? sb.x : sb.z), f1 = h2_to_f2(half == 0 ? sb.y : sb.w);
+            const float tt = fmaf(acc[i][1][e], f1.x, acc[i][0][e] * f0.x);
+            const float uu = fmaf(qs[2 * half + 1], f1.y, qs[2 * half] * f0.y);
+            t[i][e] = half == 0 ? tt : t[i][e] + tt;
+            s2[i][e] = half == 0 ? uu : s2[i][e] + uu;
+          }
+        }
+      }
+    }
+    // rows g and g^4 hold the two e4m3 terms of the same head: add them, then both have the score
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float tt = t[i][e] + __shfl_xor_sync(0xffffffffu, t[i][e], 16);
+        s2[i][e] = fmaf(kap, tt, s2[i][e]);
+      }
+  }
+  if (edge) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int pos = pos0 + 8 * tid + 4 * e + i;
+        if (pos < key_lo || pos >= key_n) s2[i][e] = -INFINITY;
+      }
+  }
+  // ---- online softmax over the chunk ----
+  float cm = fmaxf(fmaxf(fmaxf(s2[0][0], s2[0][1]), fmaxf(s2[1][0], s2[1][1])),
+                   fmaxf(fmaxf(s2[2][0], s2[2][1]), fmaxf(s2[3][0], s2[3][1])));
+  cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+  cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+  float m_new = fmaxf(st.m, cm);
+  if (m_new == -INFINITY) m_new = 0.f;
+  const float corr = fast_exp2(st.m - m_new);
+  st.m = m_new;
+  float p[4][2];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float off = (i & 1) ? m_new + 4.f : m_new;     // odd tiles: p / 16 (their value codes carry a factor 16)
+    p[i][0] = fast_exp2(s2[i][0] - off);
+    p[i][1] = fast_exp2(s2[i][1] - off);
+  }
+  st.l_e = fmaf(st.l_e, corr, (p[0][0] + p[0][1]) + (p[2][0] + p[2][1]));
+  st.l_o = fmaf(st.l_o, corr, (p[1][0] + p[1][1]) + (p[3][0] + p[3][1]));
+  // rescale the accumulators when any head's running maximum moved
+  if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+    for (int gi = 0; gi < Gv; ++gi) { st.bias_e[gi] *= corr; st.bias_o[gi] *= corr; }
+    const float c0 = __shfl_sync(0xffffffffu, corr, ((2 * tid) & 3) * 4);
+    const float c1 = __shfl_sync(0xffffffffu, corr, ((2 * tid + 1) & 3) * 4);
+#pragma unroll
+    for (int mt = 0; mt < Dv / 16; ++mt) { st.o[mt][0] *= c0; st.o[mt][1] *= c1; st.o[mt][2] *= c0; st.o[mt][3] *= c1; }
+  }
+  // ---- p * s_v per group as two-term binary16 (rows 0..3: high part, rows 4..7: low part) ----
+  uint32_t bfr[Gv][4];                                  // [group][tile] = half2(token e=0, token e=1)
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float vs[2][Gv], vb[2][Gv];
+    if (G == 2) {
+      const uint4 sb = vsb4[i * 4 + tid];
+      const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
+      vs[0][0] = a0.x; vb[0][0] = a0.y; vs[0][1] = a1.x; vb[0][1] = a1.y;
+      vs[1][0] = b0.x; vb[1][0] = b0.y; vs[1][1] = b1.x; vb[1][1] = b1.y;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint4 sb = vsb4[(i * 4 + tid) * 2 + e];
+        const uint32_t v[4] = {sb.x, sb.y, sb.z, sb.w};
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(v[gi]); vs[e][gi] = f.x; vb[e][gi] = f.y; }
+      }
+    }
+    if (edge) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int pos = pos0 + 8 * tid + 4 * e + i;
+        if (pos < key_lo || pos >= key_n) {
+#pragma unroll
+          for (int gi = 0; gi < Gv; ++gi) { vs[e][gi] = 0.f; vb[e][gi] = 0.f; }
+        }
+      }
+    }
+#pragma unroll
+    for (int gi = 0; gi < Gv; ++gi) {
+      const float x0 = p[i][0] * vs[0][gi], x1 = p[i][1] * vs[1][gi];
+      // rows 0..3: trunc16(x); rows 4..7: trunc16(x - trunc11bits(x)) -- the binary16 conversion truncates
+      const float r0 = x0 - __uint_as_float(__float_as_uint(x0) & split_mask);
+      const float r1 = x1 - __uint_as_float(__float_as_uint(x1) & split_mask);
+      bfr[gi][i] = f32x2_to_h2_rz(r0, r1);
+      if (i & 1) st.bias_o[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], st.bias_o[gi]));
+      else st.bias_e[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], st.bias_e[gi]));
+    }
+  }
+  // ---- P.V on the codes: 16 value rows x 8 columns (heads hi|lo) x 32 tokens per tile pair ----
+#pragma unroll
+  for (int q4 = 0; q4 < Dv / 32; ++q4) {
+    const uint4 w4 = vc4[(q4 * 8 + g) * 4 + tid];
+    const int gi = q4 >> 1;
+    {
+      const uint32_t xh = w4.x >> 8, yh = w4.y >> 8;
+      mma_f16(st.o[2 * q4], w4.x & kMaskLo, w4.y & kMaskLo, w4.x & kMaskHi, w4.y & kMaskHi, bfr[gi][0], bfr[gi][1]);
+      mma_f16(st.o[2 * q4], xh & kMaskLo, yh & kMaskLo, xh & kMaskHi, yh & kMaskHi, bfr[gi][2], bfr[gi][3]);
+    }
+    {
+      const uint32_t xh = w4.z >> 8, yh = w4.w >> 8;
+      mma_f16(st.o[2 * q4 + 1], w4.z & kMaskLo, w4.w & kMaskLo, w4.z & kMaskHi, w4.w & kMaskHi, bfr[gi][0], bfr[gi][1]);
+      mma_f16(st.o[2 * q4 + 1], xh & kMaskLo, yh & kMaskLo, xh & kMaskHi, yh & kMaskHi, bfr[gi][2], bfr[gi][3]);
+    }
+  }
+}
+
+__device__ inline void store_out(const DecodeParams& P, size_t index, float v) {
+  if (P.out_dtype == Q4KV_OUT_BF16) reinterpret_cast<__nv_bfloat16*>(P.out)[index] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(P.out)[index] = v;
+}
+
+// Epilogue of one segment, run by the single warp that made the deposit count complete: combine
+// the NW deposits; a pair that lies wholly inside this CTA is normalised and written out, otherwise
+// the combination becomes this CTA's partial record and the warp takes a ticket -- the CTA whose
+// ticket is the pair's last combines all records of the pair.
+template <int G, int NW>
+__device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilogues_word, int use, const DecodeParams& P,
+                                              const Segment& seg, int cta, const Partition& part, int lane) {
+  constexpr int Dv = 64 * G, J = Dv / 32;
+  constexpr int kStride = Dv + 8;
+  const Layout& y = P.y;
+  const int n_rep = y.n_rep;
+  auto mrg = [&](int w, int h) { return merge_buf + ((size_t)w * 4 + h) * kStride; };
+  const int pair = seg.a * y.Hkv + seg.hk;
+  const bool whole = seg.c0 == seg.cf && seg.c1 == seg.cf + seg.nc;
+  const size_t row0 = (size_t)seg.a * y.Hq + (size_t)seg.hk * n_rep;
+  const size_t rstride = (size_t)n_rep * (Dv + 2);
+  float* rec = P.partials + (size_t)(pair + cta) * rstride;
+  for (int h = 0; h < n_rep; ++h) {
+    // weights of the NW deposits for head h
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) M = fmaxf(M, mrg(w, h)[Dv]);
+    float wgt[NW], Lsum = 0.f;
+    bool bad = false;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float mw = mrg(w, h)[Dv], lw = mrg(w, h)[Dv + 1];
+      if (lw < 0.f) bad = true;
+      wgt[w] = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
+      Lsum = fmaf(wgt[w], lw, Lsum);
+    }
+    if (bad) Lsum = 0.f;
+    const float inv = whole ? (Lsum > 0.f ? 1.f / Lsum : 0.f) : 1.f;
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int d = 32 * j + lane, gi = d >> 6;
+      float acc = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w)
+        if (wgt[w] != 0.f) acc = fmaf(wgt[w], mrg(w, h)[d] + mrg(w, h)[Dv + 2 + gi], acc);
+      acc *= inv;
+      if (whole) store_out(P, (row0 + h) * Dv + d, acc);
+      else rec[(size_t)h * (Dv + 2) + d] = acc;
+    }
+    if (lane == 0) {
+      if (whole) { if (P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY; }
+      else { rec[(size_t)h * (Dv + 2) + Dv] = M; rec[(size_t)h * (Dv + 2) + Dv + 1] = bad ? -1.f : Lsum; }
+    }
+  }
+  // the deposit buffer can be reused from here on
+  __threadfence_block();
+  __syncwarp();
+  if (lane == 0) *(volatile int*)epilogues_word = use + 1;
+  if (whole) return;
+
+  // ticket: the CTA whose record arrives last combines all records of the pair
+  const uint32_t pair_u0 = seg.u0 - (uint32_t)(seg.c0 - seg.cf);
+  const int c_first = part.cta_of(pair_u0), c_last = part.cta_of(pair_u0 + (uint32_t)seg.nc - 1u);
+  __threadfence();
+  __syncwarp();
+  int final_merge = 0;
+  if (lane == 0) {
+    final_merge = atomicAdd(&P.tickets[pair], 1) == c_last - c_first;
+    if (final_merge) P.tickets[pair] = 0;            // ready for the next call
+  }
+  final_merge = __shfl_sync(0xffffffffu, final_merge, 0);
+  if (!final_merge) return;
+  __threadfence();
+  // All loads of a batch of records are issued before any is used: one L2 round trip per batch.
+  const int R = c_last - c_first + 1;
+  constexpr int RB = G == 2 ? 4 : 2;                   // records per batch
+  const float* base = P.partials + (size_t)(pair + c_first) * rstride;
+  float M[4], L[4], acc[4][J];
+  bool bad = false;
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    M[h] = -INFINITY; L[h] = 0.f;
+#pragma unroll
+    for (int j = 0; j < J; ++j) acc[h][j] = 0.f;
+  }
+  for (int rb = 0; rb < R; rb += RB) {
+    float mw[RB][4], lw[RB][4], v[RB][4][J];
+#pragma unroll
+    for (int i = 0; i < RB; ++i) {
+      const int r = rb + i < R ? rb + i : R - 1;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const float* r0 = base + r * rstride + (size_t)(h < n_rep ? h : 0) * (Dv + 2);
+        mw[i][h] = __ldcg(r0 + Dv);
+        lw[i][h] = __ldcg(r0 + Dv + 1);
+#pragma unroll
+        for (int j = 0; j < J; ++j) v[i][h][j] = __ldcg(r0 + 32 * j + lane);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      float Mn = M[h];
+#pragma unroll
+      for (int i = 0; i < RB; ++i)
+        if (rb + i < R) Mn = fmaxf(Mn, mw[i][h]);
+      const float c0 = M[h] == -INFINITY ? 0.f : fast_exp2(M[h] - Mn);
+      L[h] *= c0;
+#pragma unroll
+      for (int j = 0; j < J; ++j) acc[h][j] *= c0;
+#pragma unroll
+      for (int i = 0; i < RB; ++i) {
+        if (rb + i >= R) continue;
+        if (lw[i][h] < 0.f && h < n_rep) bad = true;
+        const float e = mw[i][h] == -INFINITY ? 0.f : fast_exp2(mw[i][h] - Mn);
+        L[h] = fmaf(e, lw[i][h], L[h]);
+#pragma unroll
+        for (int j = 0; j < J; ++j) acc[h][j] = fmaf(e, v[i][h][j], acc[h][j]);
+      }
+      M[h] = Mn;
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    if (h >= n_rep) continue;
+    const float Lsum = bad ? 0.f : L[h];
+    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+#pragma unroll
+    for (int j = 0; j < J; ++j) store_out(P, (row0 + h) * Dv + 32 * j + lane, acc[h][j] * inv);
+    if (lane == 0 && P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M[h] + log2f(Lsum)) / kLog2e : -INFINITY;
+  }
+}
+
+template <int G, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __grid_constant__ DecodeParams P) {
+  constexpr int D = 64 * G, Dv = D, Gv = G;
+  using S = Smem<G, NW>;
   constexpr int kSlots = S::kSlots, kChunkBytes = S::kChunkBytes;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   S& sm = *reinterpret_cast<S*>(smem_raw);
@@ -258,48 +710,40 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_mma_kernel(const 
   const int cta = blockIdx.x;
   const int n_rep = y.n_rep;
 
+  grid_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); sm.bad[s] = 0; }
+    for (int i = 0; i < kQBufs; ++i) sm.q_tag[i] = 0;
+    for (int i = 0; i < kMBufs; ++i) { sm.deposits[i] = 0; sm.epilogues[i] = 0; }
+    sm.next_chunk = 0;
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
 
-  // ---- this CTA's unit range (every warp computes it for itself) ----
-  int agent0;
-  long long agent0_start;
-  bool any_bad;
-  const long long U = scan_units(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, -1, agent0, agent0_start, any_bad);
-  if (any_bad && cta == 0 && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
-  if (U == 0) return;
-  // never more ranges than units: every CTA below n_ctas then owns a non-empty range
-  const int n_ctas = (long long)gridDim.x < U ? (int)gridDim.x : (int)U;
-  if (cta >= n_ctas) return;
-  const long long u_begin = range_begin(U, cta, n_ctas), u_end = range_begin(U, cta + 1, n_ctas);
-  if (u_begin >= u_end) return;
-  scan_units(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, u_begin, agent0, agent0_start, any_bad);
+  // ---- this CTA's unit range (every warp computes it for itself; these inputs are not written by any kernel) ----
+  const RangeStart rs = find_range(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, cta, gridDim.x);
+  if (rs.any_bad && cta == 0 && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
+  const int n_chunks = (int)(rs.u_end - rs.u_begin);
   Walker wk;
-  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, u_begin, u_end, agent0, agent0_start);
+  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, rs);
   Segment seg;
 
   // =============================== producer warp ===============================================
-  if (warp == kConsumerWarps) {
-    if (lane != 0) return;
+  if (warp == NW) {
+    // every lane issues its own chunks: chunk c0 + lane, c0 + 32 + lane, ... of each segment
+    grid_dependency_wait();                 // the pool may still be being written by the preceding kernel
     while (wk.next(seg)) {
-      int cached_lb = -1, blk = -1;
-      for (int c = seg.c0; c < seg.c1; ++c) {
-        const long long k = seg.k0 + (c - seg.c0);
-        const int slot = (int)(k % kSlots);
+      for (int c = seg.c0 + lane; c < seg.c1; c += 32) {
+        const int k = seg.k0 + (c - seg.c0);
+        const int slot = k % kSlots;
         const uint32_t round = (uint32_t)(k / kSlots);
         if (round > 0 && !mbar_wait(&sm.empty[slot], (round - 1) & 1u, &sm.abort_flag)) {
           raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
           return;
         }
-        if ((c >> 3) != cached_lb) {
-          cached_lb = c >> 3;
-          blk = P.tables[(size_t)seg.a * P.max_blocks + cached_lb];
-        }
+        const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
         if (blk < 0 || blk >= P.n_blocks) {
           sm.bad[slot] = 1;
           raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
@@ -317,250 +761,65 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_mma_kernel(const 
   }
 
   // =============================== consumer warps ==============================================
+  // Everything the consumers write (output rows, partial records, tickets) may still be in use by
+  // the preceding kernels of the stream until they have completed.
+  grid_dependency_wait();
   const int g = lane >> 2, tid = lane & 3;
   const int hrow = g & 3;                              // query head (within the KV head) of this lane's score row
-  const float delta = g >= 4 ? 1.f : 0.f;              // rows 4..7 carry the low half of the p*s split
-  bool aborted = false;
+  const bool live = hrow < n_rep;
+  const uint32_t split_mask = g >= 4 ? 0xFFFFE000u : 0u;   // rows 4..7 carry p*s minus its binary16 truncation
 
-  while (wk.next(seg)) {
-    // ---- stage the query rows of this pair: normalize by a power of two, sums per group ----
-    if (warp < n_rep) {
-      const uint16_t* qrow = P.q + ((size_t)seg.a * y.Hq + (size_t)seg.hk * n_rep + warp) * D;
-      constexpr int E = D / 32;                        // elements per lane (4 or 8), all in one group
-      float x[E];
-      if (E == 4) {
-        const uint2 v = *reinterpret_cast<const uint2*>(qrow + lane * 4);
-        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
-        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
-      } else {
-        const uint4 v = *reinterpret_cast<const uint4*>(qrow + lane * 8);
-        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(u[i] << 16); x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
-      }
-      float mx = 0.f, sum = 0.f;
-#pragma unroll
-      for (int i = 0; i < E; ++i) { mx = fmaxf(mx, fabsf(x[i])); sum += x[i]; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      constexpr int kLanesPerGroup = 64 / E;           // 16 or 8
-#pragma unroll
-      for (int o = kLanesPerGroup / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
-      if (mx == 0.f) ex = 0;
-      ex = min(max(ex, -80), 80);
-      const float sf = __uint_as_float((uint32_t)(127 + 10 - ex) << 23);       // 2^(10 - ex)
-      __half* dst = &sm.qh[warp][lane * E];
-#pragma unroll
-      for (int i = 0; i < E; ++i) dst[i] = __float2half_rn(x[i] * sf * ((i & 1) ? 0.0625f : 1.f));
-      if ((lane % kLanesPerGroup) == 0) sm.qsum[warp][lane / kLanesPerGroup] = sum * P.scale_log2;
-      if (lane == 0) sm.kappa[warp] = P.scale_log2 * __uint_as_float((uint32_t)(127 + 14 + ex) << 23);   // 2^(24 + ex - 10)
-    }
-    consumer_bar();
-    uint32_t qa[8 * G][2];
-    float qs[G], kap = 0.f;
-    {
-      const bool live = hrow < n_rep;
-#pragma unroll
-      for (int ks = 0; ks < 8 * G; ++ks) {
-        const int gi = ks >> 2, i2 = (ks >> 1) & 1, e = ks & 1;
-        const int d0 = 8 * (8 * gi + 4 * i2 + tid) + 2 * e;
-        const __half* r = sm.qh[hrow];
-        qa[ks][0] = live ? h2_bits(__halves2half2(r[d0], r[d0 + 4])) : 0u;
-        qa[ks][1] = live ? h2_bits(__halves2half2(r[d0 + 1], r[d0 + 5])) : 0u;
-      }
-#pragma unroll
-      for (int gi = 0; gi < G; ++gi) qs[gi] = live ? sm.qsum[hrow][gi] : 0.f;
-      kap = live ? sm.kappa[hrow] : 0.f;
-    }
+  // agents without any key (kv_len == 0 or a rejected length): zeros, lse = -inf
+  for (int a = cta * NW + warp; a < P.n_agents; a += gridDim.x * NW) {
+    bool bad_len;
+    if (agent_range(P.kv_lens, a, P.window, P.max_blocks, bad_len).nc > 0) continue;
+    for (int i = lane; i < y.Hq * Dv; i += 32) store_out(P, (size_t)a * y.Hq * Dv + i, 0.f);
+    if (P.lse) for (int i = lane; i < y.Hq; i += 32) P.lse[(size_t)a * y.Hq + i] = -INFINITY;
+  }
+  if (n_chunks == 0) return;
 
-    // ---- running state of this warp for this segment ----
-    float m_run = -INFINITY, l_e = 0.f, l_o = 0.f, bias_e[Gv], bias_o[Gv];
-    float o[Dv / 16][4];
-#pragma unroll
-    for (int i = 0; i < Gv; ++i) { bias_e[i] = 0.f; bias_o[i] = 0.f; }
-#pragma unroll
-    for (int i = 0; i < Dv / 16; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
-    bool poisoned = false;
-
-    const int first = seg.c0 + (int)(((long long)warp - seg.k0 % kConsumerWarps + kConsumerWarps) % kConsumerWarps);
-    for (int c = first; c < seg.c1; c += kConsumerWarps) {
-      const long long k = seg.k0 + (c - seg.c0);
-      const int slot = (int)(k % kSlots);
-      const uint32_t round = (uint32_t)(k / kSlots);
-      if (aborted || !mbar_wait(&sm.full[slot], round & 1u, &sm.abort_flag)) { aborted = true; continue; }
-      if (sm.bad[slot]) {
-        poisoned = true;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[slot]);
-        continue;
-      }
-      const uint8_t* chunk = sm.ring + (size_t)slot * kChunkBytes;
-      const uint4* kc4 = reinterpret_cast<const uint4*>(chunk);
-      const uint4* ksb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2));
-      const uint4* vc4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G);
-      const uint4* vsb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G + 32 * (Dv / 2));
-      const int pos0 = c * 32;
-      const bool edge = pos0 < seg.lo || pos0 + 32 > seg.n;
-
-      // ---- scores of the 4 key tiles: s2[i][e] for token 8*tid + 4*e + i, in log2 units ----
-      float s2[4][2];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float acc[G][4];
-#pragma unroll
-        for (int gi = 0; gi < G; ++gi) { acc[gi][0] = 0.f; acc[gi][1] = 0.f; acc[gi][2] = 0.f; acc[gi][3] = 0.f; }
-#pragma unroll
-        for (int j = 0; j < G / 2; ++j) {
-          const uint4 w4 = kc4[((i * (G / 2) + j) * 8 + g) * 4 + tid];
-          const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const int gi = 2 * j + (x >> 1), i2 = x & 1;
-            const int ks = (gi * 2 + i2) * 2;
-            const uint32_t hi = w[x] >> 8;
-            mma16816(acc[gi], qa[ks][0], 0u, qa[ks][1], 0u, w[x] & kMaskLo, w[x] & kMaskHi);
-            mma16816(acc[gi], qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, hi & kMaskLo, hi & kMaskHi);
-          }
-        }
-        // scale and bias of the two tokens this lane owns in tile i
-        float t0 = 0.f, t1 = 0.f, u0 = 0.f, u1 = 0.f;
-        if (G == 2) {
-          const uint4 sb = ksb4[i * 4 + tid];
-          const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
-          t0 = acc[0][0] * a0.x; t0 = fmaf(acc[1][0], a1.x, t0);
-          u0 = qs[0] * a0.y; u0 = fmaf(qs[1], a1.y, u0);
-          t1 = acc[0][1] * b0.x; t1 = fmaf(acc[1][1], b1.x, t1);
-          u1 = qs[0] * b0.y; u1 = fmaf(qs[1], b1.y, u1);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const uint4 sb = ksb4[(i * 4 + tid) * 2 + e];
-            const uint32_t v[4] = {sb.x, sb.y, sb.z, sb.w};
-            float t = 0.f, u = 0.f;
-#pragma unroll
-            for (int gi = 0; gi < 4; ++gi) {
-              const float2 f = h2_to_f2(v[gi]);
-              t = fmaf(acc[gi][e], f.x, t);
-              u = fmaf(qs[gi], f.y, u);
-            }
-            if (e == 0) { t0 = t; u0 = u; } else { t1 = t; u1 = u; }
-          }
-        }
-        s2[i][0] = fmaf(kap, t0, u0);
-        s2[i][1] = fmaf(kap, t1, u1);
-      }
-      if (edge) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int pos = pos0 + 8 * tid + 4 * e + i;
-            if (pos < seg.lo || pos >= seg.n) s2[i][e] = -INFINITY;
-          }
-      }
-      // ---- online softmax over the chunk ----
-      float cm = fmaxf(fmaxf(fmaxf(s2[0][0], s2[0][1]), fmaxf(s2[1][0], s2[1][1])),
-                       fmaxf(fmaxf(s2[2][0], s2[2][1]), fmaxf(s2[3][0], s2[3][1])));
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-      float m_new = fmaxf(m_run, cm);
-      if (m_new == -INFINITY) m_new = 0.f;
-      const float corr = fast_exp2(m_run - m_new);
-      m_run = m_new;
-      float p[4][2];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float off = (i & 1) ? m_new + 4.f : m_new;     // odd tiles: p / 16 (their codes carry a factor 16)
-        p[i][0] = fast_exp2(s2[i][0] - off);
-        p[i][1] = fast_exp2(s2[i][1] - off);
-      }
-      l_e = fmaf(l_e, corr, (p[0][0] + p[0][1]) + (p[2][0] + p[2][1]));
-      l_o = fmaf(l_o, corr, (p[1][0] + p[1][1]) + (p[3][0] + p[3][1]));
-#pragma unroll
-      for (int gi = 0; gi < Gv; ++gi) { bias_e[gi] *= corr; bias_o[gi] *= corr; }
-      // rescale the value accumulators when any head's running maximum moved
-      if (__any_sync(0xffffffffu, corr != 1.f)) {
-        const float c0 = __shfl_sync(0xffffffffu, corr, ((2 * tid) & 3) * 4);
-        const float c1 = __shfl_sync(0xffffffffu, corr, ((2 * tid + 1) & 3) * 4);
-#pragma unroll
-        for (int mt = 0; mt < Dv / 16; ++mt) { o[mt][0] *= c0; o[mt][1] *= c1; o[mt][2] *= c0; o[mt][3] *= c1; }
-      }
-      // ---- p * s_v per group as two-term binary16 (rows 0..3: high part, rows 4..7: low part) ----
-      uint32_t bfr[Gv][4];                                  // [group][tile] = half2(token e=0, token e=1)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float vs[2][Gv], vb[2][Gv];
-        if (G == 2) {
-          const uint4 sb = vsb4[i * 4 + tid];
-          const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
-          vs[0][0] = a0.x; vb[0][0] = a0.y; vs[0][1] = a1.x; vb[0][1] = a1.y;
-          vs[1][0] = b0.x; vb[1][0] = b0.y; vs[1][1] = b1.x; vb[1][1] = b1.y;
-        } else {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const uint4 sb = vsb4[(i * 4 + tid) * 2 + e];
-            const uint32_t v[4] = {sb.x, sb.y, sb.z, sb.w};
-#pragma unroll
-            for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(v[gi]); vs[e][gi] = f.x; vb[e][gi] = f.y; }
-          }
-        }
-        if (edge) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int pos = pos0 + 8 * tid + 4 * e + i;
-            if (pos < seg.lo || pos >= seg.n) {
-#pragma unroll
-              for (int gi = 0; gi < Gv; ++gi) { vs[e][gi] = 0.f; vb[e][gi] = 0.f; }
-            }
-          }
-        }
-#pragma unroll
-        for (int gi = 0; gi < Gv; ++gi) {
-          const float x0 = p[i][0] * vs[0][gi], x1 = p[i][1] * vs[1][gi];
-          const __half2 h = __floats2half2_rn(x0, x1);
-          const float r0 = fmaf(-delta, __low2float(h), x0), r1 = fmaf(-delta, __high2float(h), x1);
-          bfr[gi][i] = h2_bits(__floats2half2_rn(r0, r1));
-          if (i & 1) bias_o[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], bias_o[gi]));
-          else bias_e[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], bias_e[gi]));
-        }
-      }
-      // ---- P.V on the codes: 16 value rows x 8 columns (heads hi|lo) x 32 tokens per tile pair ----
-#pragma unroll
-      for (int q4 = 0; q4 < Dv / 32; ++q4) {
-        const uint4 w4 = vc4[(q4 * 8 + g) * 4 + tid];
-        const int gi = q4 >> 1;
-        {
-          const uint32_t xh = w4.x >> 8, yh = w4.y >> 8;
-          mma16816(o[2 * q4], w4.x & kMaskLo, w4.y & kMaskLo, w4.x & kMaskHi, w4.y & kMaskHi, bfr[gi][0], bfr[gi][1]);
-          mma16816(o[2 * q4], xh & kMaskLo, yh & kMaskLo, xh & kMaskHi, yh & kMaskHi, bfr[gi][2], bfr[gi][3]);
-        }
-        {
-          const uint32_t xh = w4.z >> 8, yh = w4.w >> 8;
-          mma16816(o[2 * q4 + 1], w4.z & kMaskLo, w4.w & kMaskLo, w4.z & kMaskHi, w4.w & kMaskHi, bfr[gi][0], bfr[gi][1]);
-          mma16816(o[2 * q4 + 1], xh & kMaskLo, yh & kMaskLo, xh & kMaskHi, yh & kMaskHi, bfr[gi][2], bfr[gi][3]);
-        }
-      }
+  // ---- the first segments' queries are staged up front, one warp each ----
+  {
+    Walker w2 = wk;
+    Segment s2;
+    for (int s = 0; s < kQBufs && w2.next(s2); ++s) {
+      if (s % NW != warp) continue;
+      stage_query<G>(sm.qfrag[s], sm.qsum[s], sm.kappa[s], P.q, y.Hq, n_rep, P.scale_log2, s2.a, s2.hk, lane);
+      __threadfence_block();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.empty[slot]);
+      if (lane == 0) *(volatile int*)&sm.q_tag[s] = s + 1;
     }
+  }
 
-    // ---- flush this warp's state to shared memory ----
-    {
-      float l = l_e + 16.f * l_o;
+  bool aborted = false, poisoned = false;
+  int cur = -1;                 // index of the segment `seg` describes (-1: none yet)
+  bool have_seg = false;        // this warp holds state for segment `cur`
+  uint32_t qa[4 * G];
+  float qs[G], kap = 0.f;
+  WarpState<G> st;
+  st.reset();
+
+  // Deposit this warp's state for segment `cur` (described by `seg`); the warp that completes the
+  // count combines the deposits and runs the segment's epilogue.
+  auto deposit_and_maybe_finish = [&](bool real) {
+    const int b = cur % kMBufs, use = cur / kMBufs;
+    // the buffer is free once the epilogue of its previous use is done
+    if (!aborted && !spin_until_ge(&sm.epilogues[b], use, &sm.abort_flag)) aborted = true;
+    float (*mg)[S::kMergeStride] = sm.merge[b][warp];
+    if (real) {
+      float l = st.l_e + 16.f * st.l_o;
       l += __shfl_xor_sync(0xffffffffu, l, 1);
       l += __shfl_xor_sync(0xffffffffu, l, 2);
       float bias[Gv];
 #pragma unroll
       for (int gi = 0; gi < Gv; ++gi) {
-        float b = bias_e[gi] + 16.f * bias_o[gi];
-        b += __shfl_xor_sync(0xffffffffu, b, 1);
-        b += __shfl_xor_sync(0xffffffffu, b, 2);
-        bias[gi] = b;
+        float bb = st.bias_e[gi] + 16.f * st.bias_o[gi];
+        bb += __shfl_xor_sync(0xffffffffu, bb, 1);
+        bb += __shfl_xor_sync(0xffffffffu, bb, 2);
+        bias[gi] = bb;
       }
-      float (*mg)[S::kMergeStride] = sm.merge[warp];
       if (g < 4 && tid == 0) {
-        mg[g][Dv] = m_run;
+        mg[g][Dv] = st.m;
         mg[g][Dv + 1] = (poisoned || aborted) ? -1.f : l;
 #pragma unroll
         for (int gi = 0; gi < Gv; ++gi) mg[g][Dv + 2 + gi] = bias[gi];
@@ -570,121 +829,132 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_mma_kernel(const 
       for (int mt = 0; mt < Dv / 16; ++mt) {
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-          const float v = o[mt][r] + __shfl_xor_sync(0xffffffffu, o[mt][r], 2);
+          const float v = st.o[mt][r] + __shfl_xor_sync(0xffffffffu, st.o[mt][r], 2);
           if (tid < 2) mg[2 * tid + (r & 1)][16 * mt + g + 8 * (r >> 1)] = v * 16777216.f;
         }
       }
+    } else if (lane < 4) {
+      mg[lane][Dv] = -INFINITY;
+      mg[lane][Dv + 1] = aborted ? -1.f : 0.f;
     }
-    consumer_bar();
-    // ---- combine the four warps, write the segment's partial record ----
-    {
-      const int pair = seg.a * y.Hkv + seg.hk;
-      float* rec = P.partials + (size_t)(pair + cta) * n_rep * (Dv + 2);
-      const int t = threadIdx.x;
-      for (int idx = t; idx < n_rep * Dv; idx += kConsumerThreads) {
-        const int h = idx / Dv, d = idx % Dv, gi = d >> 6;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.merge[w][h][Dv]);
-        float a = 0.f;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
-          const float mw = sm.merge[w][h][Dv];
-          if (mw != -INFINITY) a += exp2f(mw - M) * (sm.merge[w][h][d] + sm.merge[w][h][Dv + 2 + gi]);
-        }
-        rec[(size_t)h * (Dv + 2) + d] = a;
-      }
-      if (t < n_rep) {
-        const int h = t;
-        float M = -INFINITY, Lsum = 0.f;
-        bool bad = false;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.merge[w][h][Dv]);
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
-          const float mw = sm.merge[w][h][Dv], lw = sm.merge[w][h][Dv + 1];
-          if (lw < 0.f) bad = true;
-          if (mw != -INFINITY) Lsum += exp2f(mw - M) * lw;
-        }
-        rec[(size_t)h * (Dv + 2) + Dv] = M;
-        rec[(size_t)h * (Dv + 2) + Dv + 1] = bad ? -1.f : Lsum;
-      }
-      if (seg.first_of_pair && t == 0) {
-        bool bad;
-        const AgentRange r = agent_range(P.kv_lens, seg.a, P.window, P.max_blocks, bad);
-        const long long pair_last = seg.u0 + (r.cf + r.nc - seg.c0) - 1;
-        P.desc[pair] = make_int2(cta, cta_of_unit(U, pair_last, n_ctas));
-      }
+    __threadfence_block();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = atomicAdd(&sm.deposits[b], 1) == (use + 1) * NW - 1;
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    __threadfence_block();
+    segment_epilogue<G, NW>(&sm.merge[b][0][0][0], &sm.epilogues[b], use, P, seg, cta, rs.part, lane);
+  };
+
+  bool out_of_chunks = false;
+  for (;;) {
+    int k = 0;
+    if (!out_of_chunks) {
+      if (lane == 0) k = atomicAdd(&sm.next_chunk, 1);
+      k = __shfl_sync(0xffffffffu, k, 0);
+      out_of_chunks = k >= n_chunks;
     }
-    consumer_bar();
+    // move to the segment that holds chunk k (to the end of the list when out of chunks), leaving a
+    // deposit in every segment passed
+    bool finished = false;
+    while (cur < 0 || out_of_chunks || k >= seg.k0 + (seg.c1 - seg.c0)) {
+      if (cur >= 0) deposit_and_maybe_finish(have_seg);
+      have_seg = false;
+      poisoned = false;
+      if (!wk.next(seg)) { finished = true; break; }
+      ++cur;
+    }
+    if (finished) break;
+    if (!have_seg) {
+      // entering segment `cur`: its query fragments
+      const int qb = cur % kQBufs;
+      if (cur >= kQBufs && k == seg.k0) {
+        // later segments are staged by whoever claims their first chunk, once the buffer's previous
+        // segment has been left by every warp (its epilogue is done)
+        const int prev = cur - kQBufs;
+        if (!aborted && !spin_until_ge(&sm.epilogues[prev % kMBufs], prev / kMBufs + 1, &sm.abort_flag)) aborted = true;
+        stage_query<G>(sm.qfrag[qb], sm.qsum[qb], sm.kappa[qb], P.q, y.Hq, n_rep, P.scale_log2, seg.a, seg.hk, lane);
+        __threadfence_block();
+        __syncwarp();
+        if (lane == 0) *(volatile int*)&sm.q_tag[qb] = cur + 1;
+      }
+      if (!aborted && !spin_until_ge(&sm.q_tag[qb], cur + 1, &sm.abort_flag)) aborted = true;
+      __threadfence_block();
+#pragma unroll
+      for (int i = 0; i < G; ++i) {
+        const uint4 v = *reinterpret_cast<const uint4*>(&sm.qfrag[qb][g][tid][4 * i]);
+        qa[4 * i] = live ? v.x : 0u; qa[4 * i + 1] = live ? v.y : 0u; qa[4 * i + 2] = live ? v.z : 0u; qa[4 * i + 3] = live ? v.w : 0u;
+      }
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) qs[gi] = live ? sm.qsum[qb][hrow][gi] : 0.f;
+      kap = live ? sm.kappa[qb][hrow] : 0.f;
+      st.reset();
+      have_seg = true;
+    }
+    const int slot = k % kSlots;
+    const uint32_t round = (uint32_t)(k / kSlots);
+    if (aborted || !mbar_wait(&sm.full[slot], round & 1u, &sm.abort_flag)) { aborted = true; continue; }
+    if (sm.bad[slot]) {
+      poisoned = true;
+    } else {
+      const int c = seg.c0 + (k - seg.k0);
+      process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, c * 32, seg.lo, seg.n, g, tid, qa, qs, kap, split_mask, st);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[slot]);
   }
   if (aborted && lane == 0) raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
 }
 
-// grid: (Hkv, A); combines the partial records of one (agent, KV head) pair and writes n_rep output rows
-__global__ void __launch_bounds__(128)
-decode_mma_merge_kernel(Layout y, int n_agents, int max_blocks, const int32_t* __restrict__ kv_lens, int window,
-                        const int2* __restrict__ desc, const float* __restrict__ partials, void* __restrict__ out,
-                        int out_dtype, float* __restrict__ lse) {
-  const int hk = blockIdx.x, a = blockIdx.y;
-  const int Dv = y.Dv, n_rep = y.n_rep;
-  bool bad_len;
-  const AgentRange r = agent_range(kv_lens, a, window, max_blocks, bad_len);
-  const int pair = a * y.Hkv + hk;
-  int c_first = 0, c_last = -1;
-  if (r.nc > 0) { const int2 d = desc[pair]; c_first = d.x; c_last = d.y; }
-  for (int h = 0; h < n_rep; ++h) {
-    float M = -INFINITY;
-    for (int c = c_first; c <= c_last; ++c)
-      M = fmaxf(M, partials[((size_t)(pair + c) * n_rep + h) * (Dv + 2) + Dv]);
-    float Lsum = 0.f;
-    bool poisoned = false;
-    for (int c = c_first; c <= c_last; ++c) {
-      const float* rec = partials + ((size_t)(pair + c) * n_rep + h) * (Dv + 2);
-      if (rec[Dv + 1] < 0.f) poisoned = true;
-      if (rec[Dv] != -INFINITY) Lsum += exp2f(rec[Dv] - M) * rec[Dv + 1];
-    }
-    if (poisoned) Lsum = 0.f;
-    const size_t row = (size_t)a * y.Hq + (size_t)hk * n_rep + h;
-    for (int d = threadIdx.x; d < Dv; d += blockDim.x) {
-      float acc = 0.f;
-      for (int c = c_first; c <= c_last; ++c) {
-        const float* rec = partials + ((size_t)(pair + c) * n_rep + h) * (Dv + 2);
-        if (rec[Dv] != -INFINITY) acc += exp2f(rec[Dv] - M) * rec[d];
-      }
-      const float v = Lsum > 0.f ? acc / Lsum : 0.f;
-      if (out_dtype == Q4KV_OUT_BF16) reinterpret_cast<__nv_bfloat16*>(out)[row * Dv + d] = __float2bfloat16_rn(v);
-      else reinterpret_cast<float*>(out)[row * Dv + d] = v;
-    }
-    if (threadIdx.x == 0 && lse) lse[row] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY;
-  }
-}
-
-int decode_grid(const Layout& y, int n_agents, int max_kv_len) {
-  const long long units = (long long)n_agents * y.Hkv * ((max_kv_len + 31) / 32 + 1);
-  const long long cap = 148 * kCtasPerSm;
-  return (int)(units < cap ? (units < 1 ? 1 : units) : cap);
-}
-
-template <int G>
-cudaError_t launch_g(const DecodeParams& P, int grid, cudaStream_t st) {
-  const size_t smem = sizeof(Smem<G>);
-  cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+template <int G, int NW>
+cudaError_t launch_g(const DecodeParams& P, int grid, bool pdl, cudaStream_t st) {
+  static bool configured[64] = {};     // the attribute is per function and device: set it once for each
+  const size_t smem = sizeof(Smem<G, NW>);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  decode_mma_kernel<G><<<grid, kThreads, smem, st>>>(P);
-  return cudaGetLastError();
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    e = cudaFuncSetAttribute(decode_mma_kernel<G, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3((NW + 1) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, NW>, P);
 }
 
 }  // namespace
+
+// Programmatic dependent launch lets a kernel's prologue overlap the tail of its predecessor in the
+// stream; every kernel of this library waits on its predecessors before it reads or writes shared
+// state.  Setting Q4KV_NO_PDL in the environment falls back to plain stream order.
+bool pdl_enabled() {
+  static const bool on = std::getenv("Q4KV_NO_PDL") == nullptr;
+  return on;
+}
 
 bool decode_mma_supported(const Layout& y) {
   return !y.alias && y.D == y.Dv && (y.D == 128 || y.D == 256) && y.n_rep <= 4;
 }
 
+// the kernel counts work units in 32 bits
+bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks) {
+  return (long long)n_agents * y.Hkv * (max_blocks * 8ll) < (1ll << 30);
+}
+
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents) {
   const size_t pairs = (size_t)n_agents * y.Hkv;
-  const size_t desc = (pairs * sizeof(int2) + 255) & ~(size_t)255;
-  return desc + (pairs + 148 * kCtasPerSm) * y.n_rep * (y.Dv + 2) * sizeof(float);
+  const size_t tickets = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
+  return tickets + (pairs + kMaxCtas) * y.n_rep * (y.Dv + 2) * sizeof(float);
 }
 
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
@@ -692,20 +962,18 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
                               void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st) {
   if (b.n_agents <= 0) return cudaSuccess;
   const size_t pairs = (size_t)b.n_agents * y.Hkv;
-  const size_t desc_bytes = (pairs * sizeof(int2) + 255) & ~(size_t)255;
+  const size_t ticket_bytes = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
   DecodeParams P;
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e;
-  P.desc = (int2*)ws; P.partials = (float*)((uint8_t*)ws + desc_bytes); P.flags = flags;
+  P.tickets = (int32_t*)ws; P.partials = (float*)((uint8_t*)ws + ticket_bytes);
+  P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
   const int span = (window > 0 && window + 32 < max_kv_len) ? window + 32 : max_kv_len;
-  const int grid = decode_grid(y, b.n_agents, span);
-  cudaError_t e = y.G == 2 ? launch_g<2>(P, grid, st) : launch_g<4>(P, grid, st);
-  if (e != cudaSuccess) return e;
-  dim3 mgrid(y.Hkv, b.n_agents);
-  decode_mma_merge_kernel<<<mgrid, 128, 0, st>>>(y, b.n_agents, b.max_blocks, kv_lens, window, P.desc, P.partials, out,
-                                                 out_dtype, lse);
-  return cudaGetLastError();
+  const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
+  const int grid = (int)(units < kMaxCtas ? (units < 1 ? 1 : units) : kMaxCtas);
+  const bool pdl = pdl_enabled();
+  return y.G == 2 ? launch_g<2, 7>(P, grid, pdl, st) : launch_g<4, 7>(P, grid, pdl, st);
 }
 
 }  // namespace q4kv

@@ -26,9 +26,11 @@ int check_batch(const q4kv_batch* b) {
 
 size_t workspace_need(const Layout& y, int n_agents, int max_kv_len, int total_q) {
   if (total_q > 0) return 16;   // the prefill path keeps no partials
-  if (decode_mma_supported(y)) return decode_mma_workspace_bytes(y, n_agents);
   const DecodePlan p = plan_decode(y, n_agents, max_kv_len, 0);
-  return (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
+  const size_t generic = (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
+  if (!decode_mma_supported(y)) return generic;
+  const size_t mma = decode_mma_workspace_bytes(y, n_agents);
+  return mma > generic ? mma : generic;
 }
 
 }  // namespace
@@ -102,7 +104,7 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
   const cudaError_t e =
-      decode_mma_supported(y)
+      (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
           ? launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out,
                               out_dtype, lse, workspace, status_flags, (cudaStream_t)stream)
           : launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, nullptr, 0, 1, max_kv_len, window, q,

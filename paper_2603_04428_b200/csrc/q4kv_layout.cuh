@@ -124,6 +124,8 @@ cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_bl
 
 // tensor-core decode path (GQA shapes with d_qk = d_v in {128, 256}, at most 4 query heads per KV head)
 bool decode_mma_supported(const Layout& y);
+bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks);
+bool pdl_enabled();
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents);
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,

@@ -44,7 +44,7 @@ class DeviceCache:
     def workspace(self, n_agents, max_kv_len, total_q=0):
         need = B.q4kv_workspace_bytes(self.spec, n_agents, max_kv_len, total_q)
         if self._ws is None or self._ws.numel() < need:
-            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+            self._ws = torch.zeros(need, dtype=torch.uint8, device="cuda")   # arrival counters start at zero
         return self._ws
 
     def read_flags(self) -> int:
