@@ -325,7 +325,7 @@ struct Smem {
   float qsum[kQBufs][4][G];                             // scale_log2 * sum of the true q over each group
   float kappa[kQBufs][4];                               // scale_log2 * 2^(ex + 2)
   alignas(8) uint64_t full[kSlots];
-  uint64_t empty[kSlots];
+  int released[kSlots];         // number of times each slot has been consumed (monotonic: no parity aliasing)
   int bad[kSlots];
   int q_tag[kQBufs];            // s + 1 once the query of segment s is staged in buffer s % kQBufs
   int deposits[kMBufs];         // running count of deposits into each buffer
@@ -712,7 +712,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
 
   grid_launch_dependents();
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); sm.bad[s] = 0; }
+    for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); sm.released[s] = 0; sm.bad[s] = 0; }
     for (int i = 0; i < kQBufs; ++i) sm.q_tag[i] = 0;
     for (int i = 0; i < kMBufs; ++i) { sm.deposits[i] = 0; sm.epilogues[i] = 0; }
     sm.next_chunk = 0;
@@ -732,28 +732,31 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
 
   // =============================== producer warp ===============================================
   if (warp == NW) {
-    // every lane issues its own chunks: chunk c0 + lane, c0 + 32 + lane, ... of each segment
+    // Lane s owns ring slot s (kSlots <= 32): it issues the chunks k = s, s + kSlots, ... in order, each
+    // once the slot's previous chunk has been consumed, so the copies of all slots are issued in parallel.
+    static_assert(kSlots <= 32, "one producer lane per ring slot");
+    if (lane >= kSlots) return;
     grid_dependency_wait();                 // the pool may still be being written by the preceding kernel
     while (wk.next(seg)) {
-      for (int c = seg.c0 + lane; c < seg.c1; c += 32) {
-        const int k = seg.k0 + (c - seg.c0);
-        const int slot = k % kSlots;
-        const uint32_t round = (uint32_t)(k / kSlots);
-        if (round > 0 && !mbar_wait(&sm.empty[slot], (round - 1) & 1u, &sm.abort_flag)) {
+      const int k_end = seg.k0 + (seg.c1 - seg.c0);
+      for (int k = seg.k0 + (lane - seg.k0 % kSlots + kSlots) % kSlots; k < k_end; k += kSlots) {
+        const int c = seg.c0 + (k - seg.k0);
+        const int round = k / kSlots;        // k % kSlots == lane
+        if (!spin_until_ge(&sm.released[lane], round, &sm.abort_flag)) {
           raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
           return;
         }
         const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
         if (blk < 0 || blk >= P.n_blocks) {
-          sm.bad[slot] = 1;
+          sm.bad[lane] = 1;
           raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
-          mbar_arrive(&sm.full[slot]);
+          mbar_arrive(&sm.full[lane]);
         } else {
-          sm.bad[slot] = 0;
-          mbar_arrive_expect_tx(&sm.full[slot], kChunkBytes);
-          bulk_load(sm.ring + (size_t)slot * kChunkBytes,
+          sm.bad[lane] = 0;
+          mbar_arrive_expect_tx(&sm.full[lane], kChunkBytes);
+          bulk_load(sm.ring + (size_t)lane * kChunkBytes,
                     head_block(P.pool, y, P.layer, blk, seg.hk) + (size_t)(c & 7) * kChunkBytes, kChunkBytes,
-                    &sm.full[slot]);
+                    &sm.full[lane]);
         }
       }
     }
@@ -893,8 +896,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       have_seg = true;
     }
     const int slot = k % kSlots;
-    const uint32_t round = (uint32_t)(k / kSlots);
-    if (aborted || !mbar_wait(&sm.full[slot], round & 1u, &sm.abort_flag)) { aborted = true; continue; }
+    const int round = k / kSlots;
+    // the slot's previous chunk must have been consumed (then its fill is complete and the parity wait is exact)
+    if (aborted || !spin_until_ge(&sm.released[slot], round, &sm.abort_flag) ||
+        !mbar_wait(&sm.full[slot], (uint32_t)round & 1u, &sm.abort_flag)) {
+      aborted = true;
+      continue;
+    }
     if (sm.bad[slot]) {
       poisoned = true;
     } else {
@@ -902,7 +910,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, c * 32, seg.lo, seg.n, g, tid, qa, qs, kap, split_mask, st);
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[slot]);
+    if (lane == 0) { __threadfence_block(); *(volatile int*)&sm.released[slot] = round + 1; }
   }
   if (aborted && lane == 0) raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
 }
