@@ -303,13 +303,14 @@ struct DecodeParams {
   const uint16_t* q;          // bf16 [A][Hq][D]
   float scale_log2;           // softmax_scale * log2(e)
   int32_t* tickets;           // [A*Hkv], zero between calls
-  float* partials;            // [A*Hkv + kMaxCtas][n_rep][Dv + 2]
+  float* partials;            // [A*Hkv + kMaxCtas][n_rep][Dv + 4]
   void* out;
   int out_dtype;
   float* lse;
   int32_t* flags;
 };
 
+__host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
 constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
 constexpr int kMBufs = 2;      // deposit buffers
 
@@ -573,11 +574,13 @@ __device__ inline void store_out(const DecodeParams& P, size_t index, float v) {
 // Epilogue of one segment, run by the single warp that made the deposit count complete: combine
 // the NW deposits; a pair that lies wholly inside this CTA is normalised and written out, otherwise
 // the combination becomes this CTA's partial record and the warp takes a ticket -- the CTA whose
-// ticket is the pair's last combines all records of the pair.
+// ticket is the pair's last combines all records of the pair.  Each lane owns 4 consecutive output
+// elements (per 128), so every access is a 16-byte one, and the loads of a step are all issued
+// before the first is used (the records sit in L2, a microsecond away).
 template <int G, int NW>
 __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilogues_word, int use, const DecodeParams& P,
                                               const Segment& seg, int cta, const Partition& part, int lane) {
-  constexpr int Dv = 64 * G, J = Dv / 32;
+  constexpr int Dv = 64 * G, V = Dv / 128;
   constexpr int kStride = Dv + 8;
   const Layout& y = P.y;
   const int n_rep = y.n_rep;
@@ -585,38 +588,62 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
   const int pair = seg.a * y.Hkv + seg.hk;
   const bool whole = seg.c0 == seg.cf && seg.c1 == seg.cf + seg.nc;
   const size_t row0 = (size_t)seg.a * y.Hq + (size_t)seg.hk * n_rep;
-  const size_t rstride = (size_t)n_rep * (Dv + 2);
+  const size_t rstride = (size_t)n_rep * kRecStride(Dv);
   float* rec = P.partials + (size_t)(pair + cta) * rstride;
+  auto store4 = [&](int h, int d, float4 v) {
+    if (P.out_dtype == Q4KV_OUT_BF16) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+      uint2 u = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(P.out) + (row0 + h) * Dv + d) = u;
+    } else {
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(P.out) + (row0 + h) * Dv + d) = v;
+    }
+  };
   for (int h = 0; h < n_rep; ++h) {
-    // weights of the NW deposits for head h
+    float mw[NW], lw[NW];
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { const float2 t = *reinterpret_cast<const float2*>(mrg(w, h) + Dv); mw[w] = t.x; lw[w] = t.y; }
+    float4 x[V][NW];
+    float bs[V][NW];
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        x[v][w] = *reinterpret_cast<const float4*>(mrg(w, h) + 128 * v + 4 * lane);
+        bs[v][w] = mrg(w, h)[Dv + 2 + ((128 * v + 4 * lane) >> 6)];
+      }
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) M = fmaxf(M, mrg(w, h)[Dv]);
+    for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
     float wgt[NW], Lsum = 0.f;
     bool bad = false;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
-      const float mw = mrg(w, h)[Dv], lw = mrg(w, h)[Dv + 1];
-      if (lw < 0.f) bad = true;
-      wgt[w] = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
-      Lsum = fmaf(wgt[w], lw, Lsum);
+      if (lw[w] < 0.f) bad = true;
+      wgt[w] = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);
+      Lsum = fmaf(wgt[w], lw[w], Lsum);
     }
     if (bad) Lsum = 0.f;
     const float inv = whole ? (Lsum > 0.f ? 1.f / Lsum : 0.f) : 1.f;
 #pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const int d = 32 * j + lane, gi = d >> 6;
-      float acc = 0.f;
+    for (int v = 0; v < V; ++v) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int w = 0; w < NW; ++w)
-        if (wgt[w] != 0.f) acc = fmaf(wgt[w], mrg(w, h)[d] + mrg(w, h)[Dv + 2 + gi], acc);
-      acc *= inv;
-      if (whole) store_out(P, (row0 + h) * Dv + d, acc);
-      else rec[(size_t)h * (Dv + 2) + d] = acc;
+      for (int w = 0; w < NW; ++w) {
+        const bool on = wgt[w] != 0.f;                 // an empty deposit holds stale bytes
+        acc.x = fmaf(wgt[w], on ? x[v][w].x + bs[v][w] : 0.f, acc.x);
+        acc.y = fmaf(wgt[w], on ? x[v][w].y + bs[v][w] : 0.f, acc.y);
+        acc.z = fmaf(wgt[w], on ? x[v][w].z + bs[v][w] : 0.f, acc.z);
+        acc.w = fmaf(wgt[w], on ? x[v][w].w + bs[v][w] : 0.f, acc.w);
+      }
+      acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      const int d = 128 * v + 4 * lane;
+      if (whole) store4(h, d, acc);
+      else *reinterpret_cast<float4*>(rec + (size_t)h * kRecStride(Dv) + d) = acc;
     }
     if (lane == 0) {
       if (whole) { if (P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY; }
-      else { rec[(size_t)h * (Dv + 2) + Dv] = M; rec[(size_t)h * (Dv + 2) + Dv + 1] = bad ? -1.f : Lsum; }
+      else *reinterpret_cast<float2*>(rec + (size_t)h * kRecStride(Dv) + Dv) = make_float2(M, bad ? -1.f : Lsum);
     }
   }
   // the deposit buffer can be reused from here on
@@ -638,62 +665,65 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
   final_merge = __shfl_sync(0xffffffffu, final_merge, 0);
   if (!final_merge) return;
   __threadfence();
-  // All loads of a batch of records are issued before any is used: one L2 round trip per batch.
   const int R = c_last - c_first + 1;
-  constexpr int RB = G == 2 ? 4 : 2;                   // records per batch
   const float* base = P.partials + (size_t)(pair + c_first) * rstride;
-  float M[4], L[4], acc[4][J];
-  bool bad = false;
-#pragma unroll
-  for (int h = 0; h < 4; ++h) {
-    M[h] = -INFINITY; L[h] = 0.f;
-#pragma unroll
-    for (int j = 0; j < J; ++j) acc[h][j] = 0.f;
-  }
-  for (int rb = 0; rb < R; rb += RB) {
-    float mw[RB][4], lw[RB][4], v[RB][4][J];
-#pragma unroll
-    for (int i = 0; i < RB; ++i) {
-      const int r = rb + i < R ? rb + i : R - 1;
-#pragma unroll
-      for (int h = 0; h < 4; ++h) {
-        const float* r0 = base + r * rstride + (size_t)(h < n_rep ? h : 0) * (Dv + 2);
-        mw[i][h] = __ldcg(r0 + Dv);
-        lw[i][h] = __ldcg(r0 + Dv + 1);
-#pragma unroll
-        for (int j = 0; j < J; ++j) v[i][h][j] = __ldcg(r0 + 32 * j + lane);
-      }
+  // pass 1: maximum and sum per head.  Lane l looks at (record, head) pairs l, l + 32, ...; its head is l % 4.
+  const int hl = lane & 3;
+  float Ml = -INFINITY, Ll = 0.f;
+  int badl = 0;
+  if (hl < n_rep) {
+    for (int r = lane >> 2; r < R; r += 8) {
+      const float2 t = __ldcg(reinterpret_cast<const float2*>(base + r * rstride + (size_t)hl * kRecStride(Dv) + Dv));
+      if (t.y < 0.f) badl = 1;
+      const float Mn = fmaxf(Ml, t.x);
+      if (Mn != -INFINITY) Ll = Ll * fast_exp2(Ml - Mn) + t.y * fast_exp2(t.x - Mn);
+      Ml = Mn;
     }
+  }
 #pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      float Mn = M[h];
+  for (int o = 4; o < 32; o <<= 1) {
+    const float Mo = __shfl_xor_sync(0xffffffffu, Ml, o), Lo = __shfl_xor_sync(0xffffffffu, Ll, o);
+    const float Mn = fmaxf(Ml, Mo);
+    if (Mn != -INFINITY) Ll = Ll * fast_exp2(Ml - Mn) + Lo * fast_exp2(Mo - Mn);
+    Ml = Mn;
+  }
+  const bool any_bad = __any_sync(0xffffffffu, badl);
+  // pass 2: weighted sum of the records, RB at a time
+  constexpr int RB = G == 2 ? 6 : 3;
+  for (int h = 0; h < n_rep; ++h) {
+    const float M = __shfl_sync(0xffffffffu, Ml, h);
+    const float Lsum = any_bad ? 0.f : __shfl_sync(0xffffffffu, Ll, h);
+    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+    float4 acc[V];
 #pragma unroll
-      for (int i = 0; i < RB; ++i)
-        if (rb + i < R) Mn = fmaxf(Mn, mw[i][h]);
-      const float c0 = M[h] == -INFINITY ? 0.f : fast_exp2(M[h] - Mn);
-      L[h] *= c0;
-#pragma unroll
-      for (int j = 0; j < J; ++j) acc[h][j] *= c0;
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float* rh = base + (size_t)h * kRecStride(Dv);
+    for (int rb = 0; rb < R; rb += RB) {
+      float mr[RB];
+      float4 xv[RB][V];
 #pragma unroll
       for (int i = 0; i < RB; ++i) {
-        if (rb + i >= R) continue;
-        if (lw[i][h] < 0.f && h < n_rep) bad = true;
-        const float e = mw[i][h] == -INFINITY ? 0.f : fast_exp2(mw[i][h] - Mn);
-        L[h] = fmaf(e, lw[i][h], L[h]);
+        const int r = rb + i < R ? rb + i : R - 1;
+        mr[i] = __ldcg(rh + r * rstride + Dv);
 #pragma unroll
-        for (int j = 0; j < J; ++j) acc[h][j] = fmaf(e, v[i][h][j], acc[h][j]);
+        for (int v = 0; v < V; ++v) xv[i][v] = __ldcg(reinterpret_cast<const float4*>(rh + r * rstride + 128 * v + 4 * lane));
       }
-      M[h] = Mn;
+#pragma unroll
+      for (int i = 0; i < RB; ++i) {
+        const float e = (rb + i >= R || mr[i] == -INFINITY) ? 0.f : fast_exp2(mr[i] - M);
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+          acc[v].x = fmaf(e, xv[i][v].x, acc[v].x); acc[v].y = fmaf(e, xv[i][v].y, acc[v].y);
+          acc[v].z = fmaf(e, xv[i][v].z, acc[v].z); acc[v].w = fmaf(e, xv[i][v].w, acc[v].w);
+        }
+      }
     }
-  }
 #pragma unroll
-  for (int h = 0; h < 4; ++h) {
-    if (h >= n_rep) continue;
-    const float Lsum = bad ? 0.f : L[h];
-    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-#pragma unroll
-    for (int j = 0; j < J; ++j) store_out(P, (row0 + h) * Dv + 32 * j + lane, acc[h][j] * inv);
-    if (lane == 0 && P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M[h] + log2f(Lsum)) / kLog2e : -INFINITY;
+    for (int v = 0; v < V; ++v) {
+      acc[v].x *= inv; acc[v].y *= inv; acc[v].z *= inv; acc[v].w *= inv;
+      store4(h, 128 * v + 4 * lane, acc[v]);
+    }
+    if (lane == 0 && P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY;
   }
 }
 
@@ -962,7 +992,7 @@ bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks) {
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents) {
   const size_t pairs = (size_t)n_agents * y.Hkv;
   const size_t tickets = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
-  return tickets + (pairs + kMaxCtas) * y.n_rep * (y.Dv + 2) * sizeof(float);
+  return tickets + (pairs + kMaxCtas) * y.n_rep * kRecStride(y.Dv) * sizeof(float);
 }
 
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
@@ -981,6 +1011,8 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
   const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
   const int grid = (int)(units < kMaxCtas ? (units < 1 ? 1 : units) : kMaxCtas);
   const bool pdl = pdl_enabled();
+  static const int nw = std::getenv("Q4KV_DECODE_NW") ? std::atoi(std::getenv("Q4KV_DECODE_NW")) : 7;
+  if (nw == 11) return y.G == 2 ? launch_g<2, 11>(P, grid, pdl, st) : launch_g<4, 11>(P, grid, pdl, st);
   return y.G == 2 ? launch_g<2, 7>(P, grid, pdl, st) : launch_g<4, 7>(P, grid, pdl, st);
 }
 
