@@ -667,6 +667,24 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
   __threadfence();
   const int R = c_last - c_first + 1;
   const float* base = P.partials + (size_t)(pair + c_first) * rstride;
+  // The first batch of record loads is issued before the (m, l) pass, so that both travel together.
+  constexpr int RB = G == 2 ? 6 : 3;
+  float mr[RB][4];
+  float4 xv[RB][4][V];
+  auto load_batch = [&](int rb) {
+#pragma unroll
+    for (int i = 0; i < RB; ++i) {
+      const int r = rb + i < R ? rb + i : R - 1;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const float* rh = base + r * rstride + (size_t)(h < n_rep ? h : 0) * kRecStride(Dv);
+        mr[i][h] = __ldcg(rh + Dv);
+#pragma unroll
+        for (int v = 0; v < V; ++v) xv[i][h][v] = __ldcg(reinterpret_cast<const float4*>(rh + 128 * v + 4 * lane));
+      }
+    }
+  };
+  load_batch(0);
   // pass 1: maximum and sum per head.  Lane l looks at (record, head) pairs l, l + 32, ...; its head is l % 4.
   const int hl = lane & 3;
   float Ml = -INFINITY, Ll = 0.f;
@@ -688,42 +706,43 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
     Ml = Mn;
   }
   const bool any_bad = __any_sync(0xffffffffu, badl);
-  // pass 2: weighted sum of the records, RB at a time
-  constexpr int RB = G == 2 ? 6 : 3;
-  for (int h = 0; h < n_rep; ++h) {
-    const float M = __shfl_sync(0xffffffffu, Ml, h);
-    const float Lsum = any_bad ? 0.f : __shfl_sync(0xffffffffu, Ll, h);
-    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-    float4 acc[V];
+  // pass 2: weighted sum of the records, RB at a time, all heads together (nothing is stored before the end)
+  float Mh[4], Lh[4];
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float* rh = base + (size_t)h * kRecStride(Dv);
-    for (int rb = 0; rb < R; rb += RB) {
-      float mr[RB];
-      float4 xv[RB][V];
+  for (int h = 0; h < 4; ++h) {
+    Mh[h] = __shfl_sync(0xffffffffu, Ml, h);
+    Lh[h] = any_bad ? 0.f : __shfl_sync(0xffffffffu, Ll, h);
+  }
+  float4 acc[4][V];
 #pragma unroll
-      for (int i = 0; i < RB; ++i) {
-        const int r = rb + i < R ? rb + i : R - 1;
-        mr[i] = __ldcg(rh + r * rstride + Dv);
+  for (int h = 0; h < 4; ++h)
 #pragma unroll
-        for (int v = 0; v < V; ++v) xv[i][v] = __ldcg(reinterpret_cast<const float4*>(rh + r * rstride + 128 * v + 4 * lane));
-      }
+    for (int v = 0; v < V; ++v) acc[h][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int rb = 0; rb < R; rb += RB) {
+    if (rb > 0) load_batch(rb);
 #pragma unroll
-      for (int i = 0; i < RB; ++i) {
-        const float e = (rb + i >= R || mr[i] == -INFINITY) ? 0.f : fast_exp2(mr[i] - M);
+    for (int i = 0; i < RB; ++i)
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const float e = (rb + i >= R || mr[i][h] == -INFINITY) ? 0.f : fast_exp2(mr[i][h] - Mh[h]);
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-          acc[v].x = fmaf(e, xv[i][v].x, acc[v].x); acc[v].y = fmaf(e, xv[i][v].y, acc[v].y);
-          acc[v].z = fmaf(e, xv[i][v].z, acc[v].z); acc[v].w = fmaf(e, xv[i][v].w, acc[v].w);
+          acc[h][v].x = fmaf(e, xv[i][h][v].x, acc[h][v].x); acc[h][v].y = fmaf(e, xv[i][h][v].y, acc[h][v].y);
+          acc[h][v].z = fmaf(e, xv[i][h][v].z, acc[h][v].z); acc[h][v].w = fmaf(e, xv[i][h][v].w, acc[h][v].w);
         }
       }
-    }
+  }
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    if (h >= n_rep) continue;
+    const float inv = Lh[h] > 0.f ? 1.f / Lh[h] : 0.f;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-      acc[v].x *= inv; acc[v].y *= inv; acc[v].z *= inv; acc[v].w *= inv;
-      store4(h, 128 * v + 4 * lane, acc[v]);
+      float4 o = acc[h][v];
+      o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+      store4(h, 128 * v + 4 * lane, o);
     }
-    if (lane == 0 && P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY;
+    if (lane == 0 && P.lse) P.lse[row0 + h] = Lh[h] > 0.f ? (Mh[h] + log2f(Lh[h])) / kLog2e : -INFINITY;
   }
 }
 

@@ -67,6 +67,9 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
                        const void* __restrict__ v_new, int32_t* flags) {
   extern __shared__ uint8_t vcodes[];   // [8][Dv]
   __shared__ int s_agent, s_first_pos, s_count, s_row0, s_block;
+  // let the next kernel of the stream start its prologue; wait for the preceding ones before touching the pool
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (threadIdx.x == 0) {
     // find the (agent, octet) this CTA owns: agent a has ceil((pos%8 + n_a)/8) octets
@@ -162,10 +165,18 @@ cudaError_t launch_quantize_append(const Layout& y, void* pool, int n_blocks, in
   const int units = total_new / 8 + 2 * b.n_agents;        // >= sum over agents of ceil((pos%8+n)/8)
   dim3 grid(units, y.Hkv);
   const size_t smem = y.alias ? 0 : (size_t)8 * y.Dv;
-  quantize_append_kernel<<<grid, kThreads, smem, st>>>(y, (uint8_t*)pool, n_blocks, layer, b.n_agents,
-                                                       b.max_blocks, b.block_tables, pos, new_offs,
-                                                       k_new, v_new, flags);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, quantize_append_kernel, y, (uint8_t*)pool, n_blocks, layer, b.n_agents, b.max_blocks,
+                            b.block_tables, pos, new_offs, k_new, v_new, flags);
 }
 
 }  // namespace q4kv
