@@ -135,9 +135,13 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (max_q_len == 0 || max_q_len > total_q) max_q_len = total_q;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
-  const cudaError_t e = launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, total_q, max_q_len,
-                                                 max_kv_len, window, q, softmax_scale, out, out_dtype, lse,
-                                                 workspace, status_flags, (cudaStream_t)stream);
+  const cudaError_t e =
+      prefill_mma_supported(y)
+          ? launch_prefill_mma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale,
+                               out, out_dtype, lse, status_flags, (cudaStream_t)stream)
+          : launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, total_q, max_q_len, max_kv_len,
+                                     window, q, softmax_scale, out, out_dtype, lse, workspace, status_flags,
+                                     (cudaStream_t)stream);
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 

@@ -131,4 +131,10 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
                               void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
 
+// tensor-core prefill path (d_qk = d_v = 128, at most 4 query heads per KV head)
+bool prefill_mma_supported(const Layout& y);
+cudaError_t launch_prefill_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                               const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
+                               float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
+
 }  // namespace q4kv

@@ -359,6 +359,34 @@ def test_prefill_matches_oracle_and_chunking_is_invisible(H, name, prefix, chunk
     assert p.dc.read_flags() == 0
 
 
+@pytest.mark.parametrize("spec_args,prefix,chunks,window", [
+    ((1, 8, 2, 128, 128, False), [700, 0, 33], [200, 77, 130], 0),       # several 64-query tiles, an empty prefix
+    ((1, 8, 2, 128, 128, False), [700, 300], [200, 150], 96),            # sliding window across chunk edges
+    ((1, 4, 4, 128, 128, False), [2500], [300], 0),                      # MHA (one query head per KV head)
+    ((2, 6, 2, 128, 128, False), [100, 40], [65, 1], 0),                 # three query heads per KV head, a 1-token phase
+])
+def test_prefill_tensor_core_path_ragged(H, spec_args, prefix, chunks, window):
+    """Ragged phases through the d=128 tensor-core prefill kernel: every row against the oracle."""
+    lens = [p0 + c for p0, c in zip(prefix, chunks)]
+    p = Pair(H, spec_args, lens, seed=43).fill()
+    s = p.ospec
+    q_offs = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
+    q = p.q(7, int(q_offs[-1]))
+    scale = 1.0 / math.sqrt(s.d_qk)
+    for l in range(s.n_layers):
+        ref, lse_ref = O.prefill_attention(p.opool, l, p.tabs, lens, q_offs, window, f32(q), scale)
+        out, lse = p.dc.prefill(l, lens, q_offs, window, q, scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"layer {l}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref)
+    # row i of the phase equals a decode call at kv_len = prefix + i + 1
+    a, i = 0, chunks[0] // 2
+    row = int(q_offs[a]) + i
+    ref_d, _ = O.decode_attention(p.opool, 0, p.tabs[a:a + 1], [prefix[a] + i + 1], window, f32(q[row:row + 1]), scale)
+    out0, _ = p.dc.prefill(0, lens, q_offs, window, q, scale)
+    assert_attention_close(out0[row:row + 1].cpu().numpy(), ref_d)
+    assert p.dc.read_flags() == 0
+
+
 # ---- anomalies are reported, not faulted on -----------------------------------------------------
 def test_bad_block_id_and_bad_length_raise_flags_and_zero_output(H):
     from paper_2603_04428_b200 import binding as B
