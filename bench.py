@@ -484,8 +484,12 @@ def main():
 
 
 def dw_launches(w):
-    """Kernels of this library launched per step: per layer one quantize-append and one attention kernel."""
-    return 2 * w.n_layers
+    """Kernels of this library launched per step: per layer one quantize-append and one attention kernel; the
+    shape-agnostic decode path (MLA latent caches, more than 4 query heads per KV head) adds a split-merge kernel."""
+    n_rep = w.n_q_heads // w.n_kv_heads
+    tensor_decode = (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
+    per_layer = 2 if (w.kind == "prefill" or tensor_decode) else 3
+    return per_layer * w.n_layers
 
 
 if __name__ == "__main__":
