@@ -319,7 +319,8 @@ def peaks():
 
 
 # ncu DRAM traffic (read + write) per launch of the dominant kernel, from the committed profile summary
-NCU_TRAFFIC_BYTES = {}
+# (profiles/decode_mma_llama31_8b.md, profiles/decode_mma_gemma3_12b_global_layer.md)
+NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23933355, "gemma3_12b_ragged_decode": 360373504}
 
 
 def main():
