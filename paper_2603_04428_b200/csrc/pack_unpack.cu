@@ -2,10 +2,10 @@
 // (Appendix A schema, groups along head_dim), gathered from / scattered into pool blocks
 // through one block-table row.
 //
-// One CTA handles one (layer, logical block, KV head).  K words only change position
-// inside their 32-token chunk; scale/bias pairs are split into two tensors; V codes are transposed
-// between the pool's token-packed words and the persisted head-dim-packed words through a
-// shared-memory tile of one byte per code, 32 tokens at a time.
+// One CTA handles one (layer, logical block, KV head), one warp per 32-token chunk.  K words only
+// change position inside their chunk; scale/bias pairs are split into two tensors; V codes are
+// transposed between the pool's token-packed words and the persisted head-dim-packed words as
+// 8x8 nibble blocks in registers.
 #include "q4kv_layout.cuh"
 
 namespace q4kv {
@@ -28,122 +28,158 @@ __device__ inline PersistedOffsets persisted_offsets(const Layout& y) {
   return o;
 }
 
-// grid: (n_logical_blocks * Hkv, L); dynamic smem 32 * Dv bytes (V transposition tile)
+// Transpose an 8x8 matrix of nibbles held as eight words (row r = a[r], column c in bits [4c, 4c+4)).
+__device__ inline void transpose_nibbles_8x8(uint32_t (&a)[8]) {
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const uint32_t t = ((a[r] >> 16) ^ a[r + 4]) & 0x0000FFFFu;
+    a[r + 4] ^= t; a[r] ^= t << 16;
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    if (r & 2) continue;
+    const uint32_t t = ((a[r] >> 8) ^ a[r + 2]) & 0x00FF00FFu;
+    a[r + 2] ^= t; a[r] ^= t << 8;
+  }
+#pragma unroll
+  for (int r = 0; r < 8; r += 2) {
+    const uint32_t t = ((a[r] >> 4) ^ a[r + 1]) & 0x0F0F0F0Fu;
+    a[r + 1] ^= t; a[r] ^= t << 4;
+  }
+}
+
+// grid: (n_logical_blocks * Hkv, L); 8 warps, warp c handles 32-token chunk c of the head-block through its own
+// shared-memory copy of the chunk (dynamic smem: 8 * chunk_bytes).  Every global access is a full 16- or 32-byte
+// piece of a contiguous run: the pool chunk is one contiguous range, and each persisted tensor's part of a chunk is too.
 template <bool kPack>
 __global__ void __launch_bounds__(kThreads)
 pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restrict__ row, int n_tokens,
                    uint8_t* buf, int32_t* flags) {
-  extern __shared__ uint8_t tile[];   // [32 tokens][Dv] codes
+  extern __shared__ __align__(16) uint8_t stage_all[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int lb = blockIdx.x / y.Hkv, hk = blockIdx.x % y.Hkv, layer = blockIdx.y;
   const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
   const int phys = row[lb];
-  if (phys < 0 || phys >= n_blocks) {
+  const bool bad = phys < 0 || phys >= n_blocks;
+  if (bad) {
     if (threadIdx.x == 0) raise_flag(flags, Q4KV_FLAG_BAD_BLOCK);
     if (!kPack) return;
   }
-  const bool bad = phys < 0 || phys >= n_blocks;
-  const int valid = min(kBlockTokens, n_tokens - lb * kBlockTokens);   // slots >= valid are zero bytes
-  uint8_t* hb = bad ? nullptr : head_block(pool, y, layer, phys, hk);
+  const int slot0 = warp * kChunkTokens;
+  const int nv = max(0, min(kChunkTokens, n_tokens - lb * kBlockTokens - slot0));   // tokens of this chunk that exist
+  uint8_t* chunk = bad ? nullptr : head_block(pool, y, layer, phys, hk) + (size_t)warp * y.chunk_bytes;
   uint8_t* pb = buf + ((uint64_t)layer * nblk + lb) * persisted_block_bytes(y);
   const PersistedOffsets po = persisted_offsets(y);
   const int kw = y.D / 8, vw = y.Dv / 8;
+  uint8_t* st = stage_all + (size_t)warp * y.chunk_bytes;
+  uint32_t* st_kc = reinterpret_cast<uint32_t*>(st + y.off_kc);
+  __half2* st_ksb = reinterpret_cast<__half2*>(st + y.off_ksb);
+  uint32_t* st_vc = reinterpret_cast<uint32_t*>(st + y.off_vc);
+  __half2* st_vsb = reinterpret_cast<__half2*>(st + y.off_vsb);
+  uint32_t* pk = reinterpret_cast<uint32_t*>(pb + po.kc) + ((size_t)hk * kBlockTokens + slot0) * kw;
+  uint32_t* pv = reinterpret_cast<uint32_t*>(pb + po.vc) + ((size_t)hk * kBlockTokens + slot0) * vw;
+  const __half hzero = __ushort_as_half((unsigned short)0);
 
-  // K codes: word permutation inside each chunk
-  {
-    uint32_t* pk = reinterpret_cast<uint32_t*>(pb + po.kc) + (size_t)hk * kBlockTokens * kw;
-    for (int i = threadIdx.x; i < kBlockTokens * kw; i += kThreads) {
-      const int slot = i / kw, w = i % kw;
-      uint32_t* dk = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + (size_t)(slot >> 5) * y.chunk_bytes + y.off_kc) +
-                                         k_word_offset(slot & 31, w, y.G);
-      if (kPack) pk[i] = (slot < valid && !bad) ? *dk : 0u;
-      else *dk = pk[i];
+  if (kPack) {
+    const int n16 = y.chunk_bytes / 16;
+    for (int u = lane; u < n16; u += 32)
+      reinterpret_cast<uint4*>(st)[u] = (bad || nv == 0) ? make_uint4(0u, 0u, 0u, 0u) : reinterpret_cast<const uint4*>(chunk)[u];
+    __syncwarp();
+    // K codes: one 16-byte piece of a persisted row per lane and step
+    for (int q = lane; q < kChunkTokens * kw / 4; q += 32) {
+      const int tau = q / (kw / 4), x0 = (q % (kw / 4)) * 4;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (tau < nv) {
+        v.x = st_kc[k_word_offset(tau, x0, y.G)]; v.y = st_kc[k_word_offset(tau, x0 + 1, y.G)];
+        v.z = st_kc[k_word_offset(tau, x0 + 2, y.G)]; v.w = st_kc[k_word_offset(tau, x0 + 3, y.G)];
+      }
+      reinterpret_cast<uint4*>(pk)[q] = v;
+    }
+  } else {
+    for (int q = lane; q < kChunkTokens * kw / 4; q += 32) {
+      const int tau = q / (kw / 4), x0 = (q % (kw / 4)) * 4;
+      const uint4 v = reinterpret_cast<const uint4*>(pk)[q];
+      st_kc[k_word_offset(tau, x0, y.G)] = v.x; st_kc[k_word_offset(tau, x0 + 1, y.G)] = v.y;
+      st_kc[k_word_offset(tau, x0 + 2, y.G)] = v.z; st_kc[k_word_offset(tau, x0 + 3, y.G)] = v.w;
     }
   }
-  // K and V scale / bias
+  // scales and biases: half2 (scale, bias) per token and group in the pool, two tensors when persisted
   for (int which = 0; which < (y.alias ? 1 : 2); ++which) {
     const int G = which ? y.Gv : y.G;
-    __half* ps = reinterpret_cast<__half*>(pb + (which ? po.vs : po.ks)) + (size_t)hk * kBlockTokens * G;
-    __half* pbias = reinterpret_cast<__half*>(pb + (which ? po.vb : po.kb)) + (size_t)hk * kBlockTokens * G;
-    for (int i = threadIdx.x; i < kBlockTokens * G; i += kThreads) {
-      const int slot = i / G, gi = i % G;
-      __half2* dsb = bad ? nullptr : reinterpret_cast<__half2*>(hb + (size_t)(slot >> 5) * y.chunk_bytes +
-                                                                  (which ? y.off_vsb : y.off_ksb)) +
-                                         sb_offset(slot & 31, gi, G);
+    __half* ps = reinterpret_cast<__half*>(pb + (which ? po.vs : po.ks)) + ((size_t)hk * kBlockTokens + slot0) * G;
+    __half* pbias = reinterpret_cast<__half*>(pb + (which ? po.vb : po.kb)) + ((size_t)hk * kBlockTokens + slot0) * G;
+    __half2* stsb = which ? st_vsb : st_ksb;
+    for (int i = lane; i < kChunkTokens * G; i += 32) {
+      const int tau = i / G, gi = i % G;
       if (kPack) {
-        __half2 v = __halves2half2(__ushort_as_half((unsigned short)0), __ushort_as_half((unsigned short)0));
-        if (slot < valid && !bad) v = *dsb;
+        const __half2 v = tau < nv ? stsb[sb_offset(tau, gi, G)] : __halves2half2(hzero, hzero);
         ps[i] = __low2half(v);
         pbias[i] = __high2half(v);
       } else {
-        *dsb = __halves2half2(ps[i], pbias[i]);
+        stsb[sb_offset(tau, gi, G)] = __halves2half2(ps[i], pbias[i]);
       }
     }
   }
-  if (y.alias) return;
-  // V codes: transpose 32 tokens at a time
-  uint32_t* pv = reinterpret_cast<uint32_t*>(pb + po.vc) + (size_t)hk * kBlockTokens * vw;
-  const int words = 4 * y.Dv;   // words of one 32-token chunk in either layout (32*Dv/8)
-  for (int c = 0; c < 8; ++c) {
-    uint32_t* dv = bad ? nullptr : reinterpret_cast<uint32_t*>(hb + (size_t)c * y.chunk_bytes + y.off_vc);
-    if (kPack) {
-      // pool word (element d, token octet o) -> tile[8o+k][d]
-      for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int d = i >> 2, o = i & 3;
-        const uint32_t w = bad ? 0u : dv[v_word_offset(o, d)];
+  // V codes: 8x8 nibble blocks (8 tokens x 8 head-dim elements) transposed in registers
+  if (!y.alias) {
+    const int o = lane >> 3;                      // token octet of the chunk
+    for (int w = lane & 7; w < vw; w += 8) {      // persisted word index inside a row
+      uint32_t a[8];
+      if (kPack) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) tile[(8 * o + k) * y.Dv + d] = (w >> (4 * k)) & 15u;
-      }
-      __syncthreads();
-      for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int tok = i / vw, w = i % vw;
-        uint32_t o = 0;
-        if (32 * c + tok < valid) {
+        for (int j = 0; j < 8; ++j) a[j] = st_vc[v_word_offset(o, 8 * w + j)];
+        transpose_nibbles_8x8(a);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) o |= (uint32_t)tile[tok * y.Dv + 8 * w + k] << (4 * k);
-        }
-        pv[(size_t)(32 * c + tok) * vw + w] = o;
-      }
-      __syncthreads();
-    } else {
-      for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int tok = i / vw, w = i % vw;
-        const uint32_t o = pv[(size_t)(32 * c + tok) * vw + w];
+        for (int k = 0; k < 8; ++k) pv[(size_t)(8 * o + k) * vw + w] = (8 * o + k < nv) ? a[k] : 0u;
+      } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) tile[tok * y.Dv + 8 * w + k] = (o >> (4 * k)) & 15u;
-      }
-      __syncthreads();
-      for (int i = threadIdx.x; i < words; i += kThreads) {
-        const int d = i >> 2, o = i & 3;
-        uint32_t w = 0;
+        for (int k = 0; k < 8; ++k) a[k] = pv[(size_t)(8 * o + k) * vw + w];
+        transpose_nibbles_8x8(a);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) w |= (uint32_t)tile[(8 * o + k) * y.Dv + d] << (4 * k);
-        dv[v_word_offset(o, d)] = w;
+        for (int j = 0; j < 8; ++j) st_vc[v_word_offset(o, 8 * w + j)] = a[j];
       }
-      __syncthreads();
     }
+  }
+  if (!kPack) {
+    __syncwarp();
+    const int n16 = y.chunk_bytes / 16;
+    for (int u = lane; u < n16; u += 32) reinterpret_cast<uint4*>(chunk)[u] = reinterpret_cast<const uint4*>(st)[u];
   }
 }
 
 }  // namespace
 
+namespace {
+template <bool kPack>
+cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_t* row, int n_tokens, uint8_t* buf,
+                      int32_t* flags, cudaStream_t st) {
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    e = cudaFuncSetAttribute(pack_unpack_kernel<kPack>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+  dim3 grid(nblk * y.Hkv, y.L);
+  pack_unpack_kernel<kPack><<<grid, kThreads, (size_t)kChunksPerBlock * y.chunk_bytes, st>>>(y, pool, n_blocks, row, n_tokens,
+                                                                                              buf, flags);
+  return cudaGetLastError();
+}
+}  // namespace
+
 cudaError_t launch_pack(const Layout& y, const void* pool, int n_blocks, const int32_t* row, int n_tokens,
                         void* dst, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-  dim3 grid(nblk * y.Hkv, y.L);
-  pack_unpack_kernel<true><<<grid, kThreads, y.alias ? 0 : 32 * y.Dv, st>>>(
-      y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags);
-  return cudaGetLastError();
+  return launch_pu<true>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags, st);
 }
 
 cudaError_t launch_unpack(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
                           const int32_t* row, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-  dim3 grid(nblk * y.Hkv, y.L);
-  pack_unpack_kernel<false><<<grid, kThreads, y.alias ? 0 : 32 * y.Dv, st>>>(
-      y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags);
-  return cudaGetLastError();
+  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st);
 }
 
 }  // namespace q4kv
