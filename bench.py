@@ -332,7 +332,12 @@ def main():
     ap.add_argument("--impl", default="q4kv", choices=["q4kv", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op", default="step", choices=["step", "pack"],
+                    help="step: the append + attention step of --workload; pack: q4kv_pack / q4kv_unpack / bulk append")
     args = ap.parse_args()
+    if args.op == "pack":
+        run_pack(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
     w = synth.workload(args.workload)
     if args.impl == "reference":
@@ -482,6 +487,52 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_pack(args):
+    """Persist / restore one Llama-3.1-8B-shaped agent (4096 tokens, 32 layers: 151 MB packed) and append a
+    1024-token phase for 8 agents: the copy-like kernels of the path, each against the measured copy rate."""
+    import torch
+    from paper_2603_04428_b200 import binding as B, harness as H
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    hbm_peak, _, _, peak_kind = peaks()
+    L, Hq, Hkv, D, n = 32, 32, 8, 128, 4096
+    nb = n // 256 + 2
+    dc = H.DeviceCache(L, Hq, Hkv, D, D, False, nb, synth.block_tables(synth.BASE_SEED, 99, [n], nb), fill_byte=7)
+    nbytes = B.q4kv_packed_bytes(dc.spec, n)
+    dst = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+
+    def timed(fn):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        return time_region(torch, fn, args.steps) / args.steps
+    t_pack = timed(lambda: B.q4kv_pack(dc.spec, dc.pool, dc.n_blocks, dc.tables[0], n, dst, dc.flags))
+    t_unpack = timed(lambda: B.q4kv_unpack(dc.spec, dst, n, dc.pool, dc.n_blocks, dc.tables[0], dc.flags))
+    A, new = 8, 1024
+    lens = [8192] * A
+    nb2 = sum(-(-(x + new) // 256) for x in lens) + 2
+    dc2 = H.DeviceCache(1, Hq, Hkv, D, D, False, nb2, synth.block_tables(synth.BASE_SEED, 98, lens, nb2, extra_tokens=new),
+                        fill_byte=None)
+    k = torch.randn((A * new, Hkv, D), device="cuda").to(torch.bfloat16)
+    v = torch.randn((A * new, Hkv, D), device="cuda").to(torch.bfloat16)
+    pos = H.dev(np.asarray(lens, dtype=np.int32))
+    offs = H.dev(np.arange(A + 1, dtype=np.int32) * new)
+    t_app = timed(lambda: B.q4kv_quantize_append(dc2.spec, dc2.pool, dc2.n_blocks, 0, dc2.bt, pos, offs, A * new, k, v,
+                                                 dc2.flags))
+    app_bytes = k.numel() * 2 * 2 + A * new * Hkv * 144
+    assert dc.read_flags() == 0 and dc2.read_flags() == 0
+    line = {"metric": "q4_pack_hbm_gbps", "value": 2 * nbytes / t_pack / 1e9, "unit": "GB/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_pack * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": "pack_unpack_append_llama31_8b_agent", "packed_bytes": nbytes,
+                       "l2": "packed buffer + pool (302 MB) larger than L2"},
+            "roofline": {"bound": "hbm", "kernel": "q4kv_pack", "achieved": 2 * nbytes / t_pack / 1e9, "peak": hbm_peak,
+                         "unit": "GB/s", "frac": 2 * nbytes / t_pack / 1e9 / hbm_peak, "peak_kind": peak_kind, "traffic": None},
+            "unpack": {"achieved": 2 * nbytes / t_unpack / 1e9, "frac": 2 * nbytes / t_unpack / 1e9 / hbm_peak, "us": t_unpack * 1e6},
+            "append_8x1024": {"achieved": app_bytes / t_app / 1e9, "frac": app_bytes / t_app / 1e9 / hbm_peak, "us": t_app * 1e6,
+                              "bytes": app_bytes},
+            "gpu_launches": args.steps}
+    print(json.dumps(line))
 
 
 def dw_launches(w):
