@@ -71,28 +71,49 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  if (threadIdx.x == 0) {
-    // find the (agent, octet) this CTA owns: agent a has ceil((pos%8 + n_a)/8) octets
-    int u = blockIdx.x, found = -1, first = 0, cnt = 0, row0 = 0, blk = -1;
-    for (int a = 0; a < n_agents; ++a) {
-      const int p = pos[a], r0 = new_offs[a], n = new_offs[a + 1] - r0;
-      if (n <= 0) continue;
-      if (p < 0 || (long long)p + n > (long long)max_blocks * kBlockTokens) {
-        if (blockIdx.x == 0 && blockIdx.y == 0) raise_flag(flags, Q4KV_FLAG_BAD_LENGTH);
-        continue;
+  if (threadIdx.x < 32) {
+    // Find the (agent, octet) this CTA owns: agent a has ceil((pos%8 + n_a)/8) octets.  The lanes of warp 0
+    // look at 32 agents at a time, so the lengths arrive in one round trip instead of one per agent.
+    const int lane = threadIdx.x;
+    const int u = blockIdx.x;
+    int cum = 0;
+    bool found = false;
+    for (int base = 0; base < n_agents && !found; base += 32) {
+      const int a = base + lane;
+      int p = 0, r0 = 0, n = 0, octs = 0;
+      bool bad_len = false;
+      if (a < n_agents) {
+        p = pos[a]; r0 = new_offs[a]; n = new_offs[a + 1] - r0;
+        if (n > 0) {
+          if (p < 0 || (long long)p + n > (long long)max_blocks * kBlockTokens) bad_len = true;
+          else octs = ((p & 7) + n + 7) >> 3;
+        }
       }
-      const int octs = ((p & 7) + n + 7) >> 3;
-      if (u < octs) {
-        const int lo = max(p, ((p >> 3) + u) << 3);
-        const int hi = min(p + n, (((p >> 3) + u) << 3) + 8);
-        found = a; first = lo; cnt = hi - lo; row0 = r0 + (lo - p);
-        blk = tables[(size_t)a * max_blocks + (lo >> 8)];
-        if (blk < 0 || blk >= n_blocks) { raise_flag(flags, Q4KV_FLAG_BAD_BLOCK); found = -1; }
-        break;
+      if (__any_sync(0xffffffffu, bad_len) && lane == 0 && blockIdx.x == 0 && blockIdx.y == 0)
+        raise_flag(flags, Q4KV_FLAG_BAD_LENGTH);
+      int inc = octs;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += v;
       }
-      u -= octs;
+      const int tot = __shfl_sync(0xffffffffu, inc, 31);
+      if (u < cum + tot) {
+        found = true;
+        const unsigned bal = __ballot_sync(0xffffffffu, cum + inc > u);
+        if (lane == __ffs(bal) - 1) {
+          const int uu = u - (cum + inc - octs);
+          const int lo = max(p, ((p >> 3) + uu) << 3);
+          const int hi = min(p + n, (((p >> 3) + uu) << 3) + 8);
+          int who = a;
+          const int blk = tables[(size_t)a * max_blocks + (lo >> 8)];
+          if (blk < 0 || blk >= n_blocks) { raise_flag(flags, Q4KV_FLAG_BAD_BLOCK); who = -1; }
+          s_agent = who; s_first_pos = lo; s_count = hi - lo; s_row0 = r0 + (lo - p); s_block = blk;
+        }
+      }
+      cum += tot;
     }
-    s_agent = found; s_first_pos = first; s_count = cnt; s_row0 = row0; s_block = blk;
+    if (!found && lane == 0) s_agent = -1;
   }
   __syncthreads();
   if (s_agent < 0) return;
@@ -102,47 +123,38 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
   uint8_t* chunk = head_block(pool, y, layer, s_block, hk) + (size_t)(slot0 >> 5) * y.chunk_bytes;
   const int tau0 = slot0 & 31;
 
-  // ---- K rows: items (token i, word w), eight lanes per group ------------------------------
-  const int kw = y.D / 8;
-  for (int base = 0; base < 8 * kw; base += kThreads) {
+  // ---- K and V rows in one sweep: items (tensor, token i, word w), eight lanes per group.  K words and
+  // scale/bias pairs go straight to the pool; V codes go to shared memory as bytes for the transposition. ----
+  const int kw = y.D / 8, vw = y.alias ? 0 : y.Dv / 8;
+  const int n_items = 8 * (kw + vw);
+  for (int base = 0; base < n_items; base += kThreads) {
     const int idx = base + threadIdx.x;
-    const int i = idx / kw, w = idx % kw;
-    const bool live = idx < 8 * kw && i < cnt;
+    const bool is_v = idx >= 8 * kw;
+    const int j = is_v ? idx - 8 * kw : idx, ww = is_v ? vw : kw;
+    const int i = j / (ww > 0 ? ww : 1), w = j % (ww > 0 ? ww : 1);
+    const bool live = idx < n_items && i < cnt;
     float x[8];
-    if (live) load_eight_bf16(k_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.D + 8 * w, x);
-    else {
+    if (live) {
+      if (is_v) load_eight_bf16(v_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.Dv + 8 * w, x);
+      else load_eight_bf16(k_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.D + 8 * w, x);
+    } else {
 #pragma unroll
       for (int e = 0; e < 8; ++e) x[e] = 0.f;
     }
     const QuantOut o = quantize_eight(x);
     if (live) {
       const int tau = tau0 + i;
-      reinterpret_cast<uint32_t*>(chunk + y.off_kc)[k_word_offset(tau, w, y.G)] = o.word;
-      if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_ksb)[sb_offset(tau, w >> 3, y.G)] = o.sb;
+      if (is_v) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vcodes[i * y.Dv + 8 * w + e] = (o.word >> (4 * e)) & 15u;
+        if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_vsb)[sb_offset(tau, w >> 3, y.Gv)] = o.sb;
+      } else {
+        reinterpret_cast<uint32_t*>(chunk + y.off_kc)[k_word_offset(tau, w, y.G)] = o.word;
+        if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_ksb)[sb_offset(tau, w >> 3, y.G)] = o.sb;
+      }
     }
   }
   if (y.alias) return;
-
-  // ---- V rows: quantize to bytes in shared memory, then build token-packed words ------------
-  const int vw = y.Dv / 8;
-  for (int base = 0; base < 8 * vw; base += kThreads) {
-    const int idx = base + threadIdx.x;
-    const int i = idx / vw, w = idx % vw;
-    const bool live = idx < 8 * vw && i < cnt;
-    float x[8];
-    if (live) load_eight_bf16(v_new, ((size_t)(row0 + i) * y.Hkv + hk) * y.Dv + 8 * w, x);
-    else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) x[e] = 0.f;
-    }
-    const QuantOut o = quantize_eight(x);
-    if (live) {
-      const int tau = tau0 + i;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) vcodes[i * y.Dv + 8 * w + e] = (o.word >> (4 * e)) & 15u;
-      if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_vsb)[sb_offset(tau, w >> 3, y.Gv)] = o.sb;
-    }
-  }
   __syncthreads();
   const int k0 = first & 7;                 // nibble of the first new token inside the word
   uint32_t mask = 0;
