@@ -462,7 +462,7 @@ def main():
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u4 codes x int8 / f32" if w.kind == "decode" else "bf16", "data": "synthetic",
+        "dtype": "e4m3+f16 on u4 codes, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_name(w), "layers": L, "agents": w.n_agents, "kv_lens": w.lens if len(set(w.lens)) > 1 else w.lens[0],
                    "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "d_qk": w.d_qk, "d_v": w.d_v,
                    "new_tokens_per_agent": w.new_tokens, "window": w.window,
