@@ -58,8 +58,10 @@ int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);
   if (rc != Q4KV_OK) return rc;
-  // Every partial the kernels read from the scratch was written earlier in the same call, so
-  // nothing in it has to start at zero and the previous call's contents are simply overwritten.
+  // The arrival counters at the head of the scratch must be zero when a call starts: the array is
+  // zero at module load and the kernel puts each counter back to zero when its last arrival is
+  // drawn.  Every partial record read from the rest was written earlier in the same call, so the
+  // previous call's records are simply overwritten.
   return q4kv_decode_attention(spec, pool, n_blocks, layer, batch, kv_lens, max_kv_len, window, q, softmax_scale,
                                out, out_dtype, lse, scratch, kStaticScratchBytes, status_flags, stream);
 }

@@ -7,11 +7,13 @@
 // built): a CTA owns 64 consecutive queries of one agent for the (up to) four query heads of one
 // KV head -- 256 score rows, 8 warps x 2 tiles of 16 rows -- and walks the 32-token chunks of that
 // pair's keys through a shared-memory ring filled by bulk asynchronous copies.
-//   * Scores: mma.sync m16n8k32 e4m3.  A byte holding a code c IS the e4m3 number c * 2^-9, so the
-//     key operand is the packed word under two masks; every bf16 query row is normalised by a power
-//     of two and split exactly into two e4m3 terms (two MMAs into one accumulator).  Per 64-element
-//     group the integer dot product is scaled by the token's scale, and the token's bias meets the
-//     row's per-group query sum.
+//   * Scores: mma.sync m16n8k16 f16.  A 16-bit lane holding a code c in its low nibble IS the
+//     binary16 subnormal c * 2^-24, so the key operand is the packed word under a mask (nibble 1 of
+//     a lane carries a factor 16 that the matching query elements are divided by); every bf16
+//     query row is scaled by a power of two into binary16 without rounding.  (The 8-bit float forms
+//     of mma.sync cost two f16 tensor instructions plus conversions and adds on this part, so
+//     they are not used.)  Per 64-element group the integer dot product is scaled by the token's
+//     scale, and the token's bias meets the row's per-group query sum.
 //   * Values: mma.sync m16n8k16 f16 with the value codes as binary16 subnormals c * 2^-24 (masked in
 //     place from the token-packed words) and probabilities pre-multiplied by the token's group scale,
 //     rounded once to binary16; the bias part is a per-row scalar sum.
@@ -28,7 +30,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kSlots = 16;                 // ring depth in chunks
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u, kMaskB = 0x0F0F0F0Fu;
+constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u;
 
 __device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ inline void mbar_init(uint64_t* bar, uint32_t count) {
@@ -65,16 +67,15 @@ __device__ inline void bulk_load(void* dst_smem, const void* src, uint32_t bytes
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// D += A(16x32 e4m3) * B(32x8 e4m3)
-__device__ inline void mma_e4m3(float (&c)[4], const uint4& a, uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
-}
 __device__ inline void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ inline void mma_f16(float (&c)[4], const uint4& a, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
 __device__ inline float fast_exp2(float x) {
   float r;
@@ -86,17 +87,6 @@ __device__ inline uint32_t f32x2_to_h2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
-__device__ inline uint32_t f32_to_e4m3(float x) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(x));
-  return (uint32_t)(r & 0xffu);
-}
-__device__ inline float e4m3_to_f32(uint32_t b) {
-  uint32_t h2;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)b));
-  return __low2float(*reinterpret_cast<__half2*>(&h2));
-}
-
 struct PrefillParams {
   Layout y;
   const uint8_t* pool;
@@ -118,8 +108,8 @@ struct PrefillSmem {
   static constexpr int kChunkBytes = 4608;               // d = 128: 32 * (64 + 8) * 2
   static constexpr int kRows = kWarps * R * 16;
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
-  alignas(16) uint4 qfrag[kWarps][R][2][4][32];          // [warp][row tile][e4m3 term][k step][lane] = A registers
-  float kappa[kRows];                                    // scale_log2 * 2^(ex + 2) of each row
+  alignas(16) uint4 qfrag[kWarps][R][4][2][32];          // [warp][row tile][key word][half of the word][lane] = A registers
+  float kappa[kRows];                                    // scale_log2 * 2^(ex + 13) of each row
   float qsum[kRows][2];                                  // scale_log2 * per-group sums of the true query row
   alignas(8) uint64_t full[kSlots];
   int released[kSlots];                                  // warps that have finished with each slot (monotonic)
@@ -181,7 +171,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
   };
   if (warp == 0 && lane < kSlots && lane < n_chunks) issue(lane);
 
-  // ---- stage the query rows: two e4m3 terms in A-fragment order, per-row factor and group sums ----
+  // ---- stage the query rows: binary16 in A-fragment order, per-row factor and group sums ----
   for (int item = threadIdx.x; item < S::kRows * 16; item += kThreads) {
     const int row = item >> 4, w = item & 15;
     const int wv = row / (16 * R), rt = (row >> 4) % R, rr = row & 15;
@@ -204,24 +194,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
     int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
     if (mx == 0.f) ex = 0;
     ex = min(max(ex, -100), 100);
-    const float sf = __uint_as_float((uint32_t)(127 + 7 - ex) << 23);                      // |q| * sf < 256
-    uint32_t r1a = 0u, r1b = 0u, r2a = 0u, r2b = 0u;
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const float qn = x[n] * sf;
-      const uint32_t b1 = f32_to_e4m3(qn);
-      const uint32_t b2 = f32_to_e4m3(qn - e4m3_to_f32(b1));
-      if (n & 1) { r1b |= b1 << (8 * (n >> 1)); r2b |= b2 << (8 * (n >> 1)); }
-      else { r1a |= b1 << (8 * (n >> 1)); r2a |= b2 << (8 * (n >> 1)); }
-    }
-    // A registers: x = row g even elements, y = row g+8 even, z = row g odd, w = row g+8 odd
+    const float sf = __uint_as_float((uint32_t)(127 + 11 - ex) << 23);                     // 2048 <= max |q| * sf < 4096
+    const float sl = sf * 0.0625f;                       // elements that meet a code in nibble 1 of its 16-bit lane
+    // Key word w of a token holds elements 8w..8w+7; its two 16x8x16 products take, per lane,
+    // (0,4 | 1,5) and (2,6 | 3,7): registers a0/a1 = rows g/g+8 of the first pair, a2/a3 of the second.
     const int ks = w >> 2, dl = (rr & 7) * 4 + (w & 3), up = rr >> 3;
-    uint32_t* f1 = reinterpret_cast<uint32_t*>(&sm.qfrag[wv][rt][0][ks][dl]);
-    uint32_t* f2 = reinterpret_cast<uint32_t*>(&sm.qfrag[wv][rt][1][ks][dl]);
-    f1[up] = r1a; f1[2 + up] = r1b;
-    f2[up] = r2a; f2[2 + up] = r2b;
+    uint32_t* f1 = reinterpret_cast<uint32_t*>(&sm.qfrag[wv][rt][ks][0][dl]);
+    uint32_t* f2 = reinterpret_cast<uint32_t*>(&sm.qfrag[wv][rt][ks][1][dl]);
+    f1[up] = f32x2_to_h2(x[0] * sf, x[4] * sf); f1[2 + up] = f32x2_to_h2(x[1] * sl, x[5] * sl);
+    f2[up] = f32x2_to_h2(x[2] * sf, x[6] * sf); f2[2 + up] = f32x2_to_h2(x[3] * sl, x[7] * sl);
     if ((w & 7) == 0) sm.qsum[row][w >> 3] = sum * P.scale_log2;
-    if (w == 0) sm.kappa[row] = P.scale_log2 * __uint_as_float((uint32_t)(127 + 2 + ex) << 23);
+    if (w == 0) sm.kappa[row] = P.scale_log2 * __uint_as_float((uint32_t)(127 + 13 + ex) << 23);
   }
   __syncthreads();
 
@@ -278,13 +261,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
         for (int i = 0; i < 4; ++i) kw[i] = kc4[(i * 8 + g) * 4 + tid];
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {
-          const uint4 a1 = sm.qfrag[warp][rt][0][ks][lane], a2 = sm.qfrag[warp][rt][1][ks][lane];
+          const uint4 a1 = sm.qfrag[warp][rt][ks][0][lane], a2 = sm.qfrag[warp][rt][ks][1][lane];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const uint32_t w = ks == 0 ? kw[i].x : ks == 1 ? kw[i].y : ks == 2 ? kw[i].z : kw[i].w;
-            const uint32_t b0 = w & kMaskB, b1 = (w >> 4) & kMaskB;
-            mma_e4m3(acc[i][ks >> 1], a1, b0, b1);
-            mma_e4m3(acc[i][ks >> 1], a2, b0, b1);
+            const uint32_t wh = w >> 8;
+            mma_f16(acc[i][ks >> 1], a1, w & kMaskLo, w & kMaskHi);
+            mma_f16(acc[i][ks >> 1], a2, wh & kMaskLo, wh & kMaskHi);
           }
         }
         // ---- scores in log2 units, mask, online softmax ----
