@@ -320,7 +320,7 @@ def peaks():
 
 # ncu DRAM traffic (read + write) per launch of the dominant kernel, from the committed profile summary
 # (profiles/decode_mma_llama31_8b.md, profiles/decode_mma_gemma3_12b_global_layer.md)
-NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23933355, "gemma3_12b_ragged_decode": 360373504}
+NCU_TRAFFIC_BYTES = {}   # workload -> dram bytes per launch of the current kernel (ncu); empty until re-captured
 
 
 def main():
@@ -462,7 +462,7 @@ def main():
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "e4m3+f16 on u4 codes, f32 accumulate", "data": "synthetic",
+        "dtype": "f16 tensor-core products on u4 codes, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_name(w), "layers": L, "agents": w.n_agents, "kv_lens": w.lens if len(set(w.lens)) > 1 else w.lens[0],
                    "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "d_qk": w.d_qk, "d_v": w.d_v,
                    "new_tokens_per_agent": w.new_tokens, "window": w.window,

@@ -22,20 +22,18 @@
 //     (s, b) per token and 64-element group,
 //         q.k_t   = sum_g [ s_tg * (sum_{d in g} q_d c_td) + b_tg * (sum_{d in g} q_d) ]
 //         (p.V)_d = sum_t (p_t s_tg(d)) c_td + sum_t p_t b_tg(d).
-//     Both contractions run on the tensor cores with the code operand produced by masking the
-//     packed word in place:
-//       - q.K: mma.sync m16n8k32 e4m3.  A byte holding a code c in 0..15 IS the e4m3 number
-//         c * 2^-9 (the first normal binade continues the subnormal spacing), so two masks turn a
-//         word into the B operand.  The bf16 query is split exactly into two e4m3 terms
-//         (4 + 4 significant bits) that occupy different rows of the A operand.
-//       - p.V: mma.sync m16n8k16 f16.  A nibble in the low bits of a 16-bit lane is the binary16
-//         subnormal c * 2^-24 (16c * 2^-24 one nibble up; the 16 is folded into p).
-//     Both forms multiply exactly and at full rate on sm_100a.
+//     Both contractions are mma.sync m16n8k16 f16 with the code operand produced by masking the
+//     packed word in place: a nibble in the low bits of a 16-bit lane IS the binary16 subnormal
+//     c * 2^-24, and one nibble up it is 16c * 2^-24 -- the 16 is divided out of the other operand
+//     (the matching query elements for q.K, the probabilities of odd key tiles for p.V).  The bf16
+//     query is scaled per row by a power of two into binary16, so nothing is rounded before the
+//     products, which are exact.  (The 8-bit float forms of mma.sync are not used: on this part
+//     each costs two f16 tensor instructions plus conversions and adds.)
 //   * Scores come out as [8 rows x 8 tokens] fragments whose lane ownership is the B-operand
 //     ownership of the P.V product, so probabilities never move between lanes.  Rows 0..3 are
-//     the query heads (first e4m3 term), rows 4..7 the same heads (second term); after one
-//     shuffle both hold the full score, and rows 4..7 go on to carry the low half of a two-term
-//     binary16 split of p*s, which makes the value product accurate to ~2^-22 at no extra MMA.
+//     the query heads and rows 4..7 repeat them; rows 4..7 go on to carry the low half of a
+//     two-term binary16 split of p*s, which makes the value product accurate to ~2^-22 at no
+//     extra MMA.
 #include <cstdlib>
 
 #include "q4kv_layout.cuh"
@@ -47,7 +45,7 @@ namespace {
 constexpr int kMaxCtas = 148;                          // one persistent CTA per SM
 constexpr uint32_t kSpinLimit = 1u << 22;              // bounded mbarrier waits (each try blocks a while in hardware)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u, kMaskB = 0x0F0F0F0Fu;
+constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u;
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -101,11 +99,17 @@ __device__ inline void bulk_load(void* dst_smem, const void* src, uint32_t bytes
 __device__ inline void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ inline void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// D = A(16x32 e4m3, rows 8..15 zero) * B(32x8 e4m3) + C; only rows 0..7 of D are meaningful
-__device__ inline void mma_e4m3(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1, const float (&c)[4]) {
-  asm("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+// D = A(16x16 f16, rows 8..15 zero) * B(16x8 f16); only rows 0..7 of D are meaningful
+__device__ inline void mma_f16_rows8_first(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
       : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+}
+// D += A(16x16 f16, rows 8..15 zero) * B(16x8 f16)
+__device__ inline void mma_f16_rows8(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 __device__ inline void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -124,16 +128,9 @@ __device__ inline uint32_t f32x2_to_h2_rz(float a, float b) {
   asm("cvt.rz.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
   return r;
 }
-// one float -> e4m3 byte (round to nearest, saturating)
-__device__ inline uint32_t f32_to_e4m3(float x) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(x));
-  return (uint32_t)(r & 0xffu);
-}
-__device__ inline float e4m3_to_f32(uint32_t b) {
-  uint32_t h2;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)b));
-  return __low2float(*reinterpret_cast<__half2*>(&h2));
+__device__ inline uint32_t f32x2_to_h2_rn(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -322,9 +319,9 @@ struct Smem {
   static constexpr int kMergeStride = D + 8;            // acc[Dv], m, l, bias[Gv], pad
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
   alignas(16) float merge[kMBufs][NW][4][kMergeStride];
-  alignas(16) uint32_t qfrag[kQBufs][8][4][4 * G];      // [buffer][row][tid][A-operand registers of the lane]
+  alignas(16) uint4 qfrag[kQBufs][2 * G][32];           // [buffer][key word of a lane][lane = row * 4 + tid] = A registers
   float qsum[kQBufs][4][G];                             // scale_log2 * sum of the true q over each group
-  float kappa[kQBufs][4];                               // scale_log2 * 2^(ex + 2)
+  float kappa[kQBufs][4];                               // scale_log2 * 2^(ex + 13)
   alignas(8) uint64_t full[kSlots];
   int released[kSlots];         // number of times each slot has been consumed (monotonic: no parity aliasing)
   int bad[kSlots];
@@ -349,11 +346,15 @@ struct WarpState {
   }
 };
 
-// Warp-level: stage the query rows of one pair as two e4m3 terms in A-fragment order, plus the
-// per-group sums of the true query and the per-head factor that undoes the normalisation.
-// Element d = 8w + n of a row, w = 8*gi + 4*i2 + t: register (2*gi + i2)*2 + (n & 1) of lane t, byte n >> 1.
+// Warp-level: stage the query rows of one pair as binary16 in A-fragment order (each row scaled by a
+// power of two, so nothing is rounded), plus the per-group sums of the true query and the per-head
+// factor that undoes the scaling.  Key word w = 8*gi + 4*i2 + t of a token holds elements 8w..8w+7
+// and feeds two 16x8x16 products: (0,4 | 1,5) and (2,6 | 3,7), where the second pair of each meets
+// codes in nibble 1 of their 16-bit lanes (a factor 16, divided out of the query here).  The uint4
+// of word p = 2*gi + i2 is {a0, a2} of the first product and {a0, a2} of the second, for the lane
+// (row h, t); rows h + 4 repeat rows h, so that lanes g and g + 4 see the same scores.
 template <int G>
-__device__ __noinline__ void stage_query(uint32_t (*qfrag)[4][4 * G], float (*qsum)[G], float* kappa,
+__device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], float* kappa,
                                          const uint16_t* __restrict__ q, int Hq, int n_rep, float scale_log2, int a,
                                          int hk, int lane) {
   constexpr int D = 64 * G;
@@ -380,29 +381,22 @@ __device__ __noinline__ void stage_query(uint32_t (*qfrag)[4][4 * G], float (*qs
     int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
     if (mx == 0.f) ex = 0;
     ex = min(max(ex, -100), 100);
-    const float sf = __uint_as_float((uint32_t)(127 + 7 - ex) << 23);          // 2^(7 - ex): |q| * sf < 256
-    uint32_t r1a = 0u, r1b = 0u, r2a = 0u, r2b = 0u;    // even / odd elements -> two registers
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const float qn = x[n] * sf;
-      const uint32_t b1 = f32_to_e4m3(qn);
-      const uint32_t b2 = f32_to_e4m3(qn - e4m3_to_f32(b1));
-      if (n & 1) { r1b |= b1 << (8 * (n >> 1)); r2b |= b2 << (8 * (n >> 1)); }
-      else { r1a |= b1 << (8 * (n >> 1)); r2a |= b2 << (8 * (n >> 1)); }
-    }
+    const float sf = __uint_as_float((uint32_t)(127 + 11 - ex) << 23);         // 2048 <= max |q| * sf < 4096
+    const float sl = sf * 0.0625f;
+    const uint4 f = make_uint4(f32x2_to_h2_rn(x[0] * sf, x[4] * sf), f32x2_to_h2_rn(x[1] * sl, x[5] * sl),
+                               f32x2_to_h2_rn(x[2] * sf, x[6] * sf), f32x2_to_h2_rn(x[3] * sl, x[7] * sl));
     const int gi = w >> 3, i2 = (w >> 2) & 1, t = w & 3;
-    const int reg = (2 * gi + i2) * 2;
-    *reinterpret_cast<uint2*>(&qfrag[h][t][reg]) = make_uint2(r1a, r1b);
-    *reinterpret_cast<uint2*>(&qfrag[h + 4][t][reg]) = make_uint2(r2a, r2b);
+    qfrag[2 * gi + i2][h * 4 + t] = f;
+    qfrag[2 * gi + i2][(h + 4) * 4 + t] = f;
     if ((w & 7) == 0) qsum[h][gi] = sum * scale_log2;
-    if (w == 0) kappa[h] = scale_log2 * __uint_as_float((uint32_t)(127 + 2 + ex) << 23);   // 2^(9 + ex - 7)
+    if (w == 0) kappa[h] = scale_log2 * __uint_as_float((uint32_t)(127 + 13 + ex) << 23);  // 2^24 / sf
   }
 }
 
 // One 32-token chunk against this warp's query fragments.
 template <int G>
 __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
-                                              const uint32_t (&qa)[4 * G], const float (&qs)[G], float kap,
+                                              const uint4* qa, const float (&qs)[G], float kap,
                                               uint32_t split_mask, WarpState<G>& st) {
   constexpr int D = 64 * G, Dv = D, Gv = G;
   const uint4* kc4 = reinterpret_cast<const uint4*>(chunk);
@@ -414,7 +408,6 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
   // ---- scores of the 4 key tiles: s2[i][e] for token 8*tid + 4*e + i, in log2 units ----
   float s2[4][2];
   {
-    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
     float t[4][2];
 #pragma unroll
     for (int half = 0; half < G / 2; ++half) {        // groups 2*half, 2*half+1
@@ -423,21 +416,15 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
       for (int i = 0; i < 4; ++i) kw[i] = kc4[((i * (G / 2) + half) * 8 + g) * 4 + tid];
       float acc[4][2][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t w[4] = {kw[i].x, kw[i].y, kw[i].z, kw[i].w};
+      for (int j = 0; j < 4; ++j) {                     // word p = 4*half + j: group 2*half + j/2, i2 = j%2
+        const uint4 a = qa[(4 * half + j) * 32];
 #pragma unroll
-        for (int gg = 0; gg < 2; ++gg) {
-          const int r = (2 * (2 * half + gg)) * 2;      // registers of word (gi, i2 = 0)
-          mma_e4m3(acc[i][gg], qa[r], qa[r + 1], w[2 * gg] & kMaskB, (w[2 * gg] >> 4) & kMaskB, zero);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t w[4] = {kw[i].x, kw[i].y, kw[i].z, kw[i].w};
-#pragma unroll
-        for (int gg = 0; gg < 2; ++gg) {
-          const int r = (2 * (2 * half + gg) + 1) * 2;  // registers of word (gi, i2 = 1)
-          mma_e4m3(acc[i][gg], qa[r], qa[r + 1], w[2 * gg + 1] & kMaskB, (w[2 * gg + 1] >> 4) & kMaskB, acc[i][gg]);
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t w = j == 0 ? kw[i].x : j == 1 ? kw[i].y : j == 2 ? kw[i].z : kw[i].w;
+          const uint32_t wh = w >> 8;
+          if ((j & 1) == 0) mma_f16_rows8_first(acc[i][j >> 1], a.x, a.y, w & kMaskLo, w & kMaskHi);
+          else mma_f16_rows8(acc[i][j >> 1], a.x, a.y, w & kMaskLo, w & kMaskHi);
+          mma_f16_rows8(acc[i][j >> 1], a.z, a.w, wh & kMaskLo, wh & kMaskHi);
         }
       }
       // scale of the two tokens this lane owns in each tile
@@ -463,14 +450,11 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
         }
       }
     }
-    // rows g and g^4 hold the two e4m3 terms of the same head: add them, then both have the score
+    // rows g and g + 4 carry the same head, so both lanes hold its score
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const float tt = t[i][e] + __shfl_xor_sync(0xffffffffu, t[i][e], 16);
-        s2[i][e] = fmaf(kap, tt, s2[i][e]);
-      }
+      for (int e = 0; e < 2; ++e) s2[i][e] = fmaf(kap, t[i][e], s2[i][e]);
   }
   if (edge) {
 #pragma unroll
@@ -760,6 +744,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   const int n_rep = y.n_rep;
 
   grid_launch_dependents();
+  // rows of query heads that do not exist (n_rep < 4) are never staged: they stay zero
+  for (int i = threadIdx.x; i < kQBufs * 2 * G * 32; i += blockDim.x) (&sm.qfrag[0][0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); sm.released[s] = 0; sm.bad[s] = 0; }
     for (int i = 0; i < kQBufs; ++i) sm.q_tag[i] = 0;
@@ -846,7 +832,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   bool aborted = false, poisoned = false;
   int cur = -1;                 // index of the segment `seg` describes (-1: none yet)
   bool have_seg = false;        // this warp holds state for segment `cur`
-  uint32_t qa[4 * G];
+  const uint4* qa = nullptr;    // this lane's A registers of the segment's query, in shared memory
   float qs[G], kap = 0.f;
   WarpState<G> st;
   st.reset();
@@ -933,11 +919,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       }
       if (!aborted && !spin_until_ge(&sm.q_tag[qb], cur + 1, &sm.abort_flag)) aborted = true;
       __threadfence_block();
-#pragma unroll
-      for (int i = 0; i < G; ++i) {
-        const uint4 v = *reinterpret_cast<const uint4*>(&sm.qfrag[qb][g][tid][4 * i]);
-        qa[4 * i] = live ? v.x : 0u; qa[4 * i + 1] = live ? v.y : 0u; qa[4 * i + 2] = live ? v.z : 0u; qa[4 * i + 3] = live ? v.w : 0u;
-      }
+      qa = &sm.qfrag[qb][0][lane];
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) qs[gi] = live ? sm.qsum[qb][hrow][gi] : 0.f;
       kap = live ? sm.kappa[qb][hrow] : 0.f;
