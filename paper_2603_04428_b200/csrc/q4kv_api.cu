@@ -1,5 +1,7 @@
 // C ABI of libq4kv.so: host-side validation, sizing and dispatch.  See include/q4kv.h for
 // the contract of every entry point.
+#include <cstdlib>
+
 #include "q4kv_layout.cuh"
 
 using namespace q4kv;
@@ -135,13 +137,19 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (max_q_len == 0 || max_q_len > total_q) max_q_len = total_q;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
-  const cudaError_t e =
-      prefill_mma_supported(y)
-          ? launch_prefill_mma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale,
-                               out, out_dtype, lse, status_flags, (cudaStream_t)stream)
-          : launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, total_q, max_q_len, max_kv_len,
-                                     window, q, softmax_scale, out, out_dtype, lse, workspace, status_flags,
-                                     (cudaStream_t)stream);
+  // Q4KV_PREFILL_PATH=mma in the environment keeps the register-level mma.sync kernel for shapes both cover.
+  static const bool force_mma = [] { const char* v = std::getenv("Q4KV_PREFILL_PATH"); return v && v[0] == 'm'; }();
+  cudaError_t e;
+  if (prefill_umma_supported(y) && softmax_scale > 0.f && !force_mma)
+    e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
+                            out_dtype, lse, status_flags, (cudaStream_t)stream);
+  else if (prefill_mma_supported(y))
+    e = launch_prefill_mma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
+                           out_dtype, lse, status_flags, (cudaStream_t)stream);
+  else
+    e = launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, total_q, max_q_len, max_kv_len,
+                                 window, q, softmax_scale, out, out_dtype, lse, workspace, status_flags,
+                                 (cudaStream_t)stream);
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 

@@ -137,4 +137,11 @@ cudaError_t launch_prefill_mma(const Layout& y, const void* pool, int n_blocks, 
                                const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
                                float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
 
+
+// tcgen05 prefill path (d_qk = d_v = 128; 1, 2 or 4 query heads per KV head)
+bool prefill_umma_supported(const Layout& y);
+cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                                const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
+                                float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
+
 }  // namespace q4kv
