@@ -139,8 +139,12 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
   // Q4KV_PREFILL_PATH=mma in the environment keeps the register-level mma.sync kernel for shapes both cover.
   static const bool force_mma = [] { const char* v = std::getenv("Q4KV_PREFILL_PATH"); return v && v[0] == 'm'; }();
+  // The tcgen05 kernel rounds each dequantized key and value once to binary16 (11 significant bits); the error that
+  // leaves in a score grows with the softmax scale, and stays well inside the library's 2e-3 output bound up to twice
+  // the usual 1/sqrt(d).  Sharper scales take the kernel that multiplies the codes exactly.
+  const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
   cudaError_t e;
-  if (prefill_umma_supported(y) && softmax_scale > 0.f && !force_mma)
+  if (prefill_umma_supported(y) && usual_scale && !force_mma)
     e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                             out_dtype, lse, status_flags, (cudaStream_t)stream);
   else if (prefill_mma_supported(y))

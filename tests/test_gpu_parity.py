@@ -387,6 +387,64 @@ def test_prefill_tensor_core_path_ragged(H, spec_args, prefix, chunks, window):
     assert p.dc.read_flags() == 0
 
 
+class QuietStartPair(Pair):
+    """The first 300 keys of every agent are tiny, so every row's running maximum jumps far when the walk leaves them."""
+
+    def kv(self, layer, agent, n):
+        k, v = super().kv(layer, agent, n)
+        kf = f32(k).copy()
+        kf[:300] *= np.float32(0.02)
+        return synth.f32_to_bf16_bits(kf), v
+
+
+@pytest.mark.parametrize("spec_args,prefix,chunks,window,scale_mul", [
+    ((1, 4, 2, 128, 128, False), [900, 5], [140, 70], 0, 1.0),           # two query heads per KV head: 64-query tiles
+    ((1, 8, 2, 128, 128, False), [3000], [200], 700, 1.0),               # the window starts many 64-key blocks in
+    ((1, 8, 2, 128, 128, False), [1500, 64], [129, 64], 0, 2.0),         # the row maximum jumps by more than 2^8, late
+    ((1, 8, 2, 128, 128, False), [1500, 64], [129, 64], 0, 8.0),         # a sharp scale is routed to the exact-code kernel
+    ((1, 4, 4, 128, 128, False), [0], [257], 0, 1.0),                    # no prefix at all: purely causal
+])
+def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
+    """The tensor-memory prefill kernel: tile shapes for 1, 2 and 4 heads per KV head, key ranges that start
+    inside the cache, wrap the shared-memory stages many times, and scores whose maximum grows in steps both
+    smaller and larger than the lazy-rescale threshold."""
+    lens = [p0 + c for p0, c in zip(prefix, chunks)]
+    p = QuietStartPair(H, spec_args, lens, seed=47).fill()
+    s = p.ospec
+    q_offs = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
+    q = p.q(9, int(q_offs[-1]))
+    scale = scale_mul / math.sqrt(s.d_qk)
+    ref, lse_ref = O.prefill_attention(p.opool, 0, p.tabs, lens, q_offs, window, f32(q), scale)
+    out, lse = p.dc.prefill(0, lens, q_offs, window, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    from paper_2603_04428_b200 import binding as B
+    out16, _ = p.dc.prefill(0, lens, q_offs, window, q, scale, out_dtype=B.OUT_BF16)
+    assert torch.allclose(out16.float(), out.to(torch.bfloat16).float(), atol=1e-5, rtol=2.0 ** -7)
+    assert p.dc.read_flags() == 0
+
+
+def test_prefill_bad_block_and_bad_length(H):
+    from paper_2603_04428_b200 import binding as B
+    lens = [600, 200]
+    p = Pair(H, (1, 8, 2, 128, 128, False), lens, seed=53).fill()
+    q_offs = [0, 100, 180]
+    q = p.q(7, 180)
+    good, _ = p.dc.prefill(0, lens, q_offs, 0, q, 0.1)
+    tabs = p.tabs.copy()
+    tabs[0, 1] = -5
+    t = H.dev(tabs)
+    out, lse = p.dc.prefill(0, lens, q_offs, 0, q, 0.1, bt=B.batch(t))
+    assert p.dc.read_flags() & B.FLAG_BAD_BLOCK
+    assert torch.all(out[:100] == 0) and torch.equal(out[100:], good[100:])
+    assert torch.all(torch.isneginf(lse[:100]))
+    p.dc.flags.zero_()
+    out, _ = p.dc.prefill(0, [50, 200], q_offs, 0, q, 0.1)          # more new tokens than cached tokens
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    assert torch.all(out[:100] == 0) and torch.equal(out[100:], good[100:])
+    p.dc.flags.zero_()
+
+
 # ---- anomalies are reported, not faulted on -----------------------------------------------------
 def test_bad_block_id_and_bad_length_raise_flags_and_zero_output(H):
     from paper_2603_04428_b200 import binding as B
