@@ -29,7 +29,11 @@ int check_batch(const q4kv_batch* b) {
 size_t workspace_need(const Layout& y, int n_agents, int max_kv_len, int total_q) {
   if (total_q > 0) return 16;   // the prefill path keeps no partials
   const DecodePlan p = plan_decode(y, n_agents, max_kv_len, 0);
-  const size_t generic = (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
+  size_t generic = (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
+  if (decode_mla_supported(y)) {
+    const size_t mla = decode_mla_workspace_bytes(y, n_agents, max_kv_len);
+    if (mla > generic) generic = mla;
+  }
   if (!decode_mma_supported(y)) return generic;
   const size_t mma = decode_mma_workspace_bytes(y, n_agents);
   return mma > generic ? mma : generic;
@@ -105,13 +109,20 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
-  const cudaError_t e =
-      (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
-          ? launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out,
-                              out_dtype, lse, workspace, status_flags, (cudaStream_t)stream)
-          : launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, nullptr, 0, 1, max_kv_len, window, q,
-                                     softmax_scale, out, out_dtype, lse, workspace, status_flags,
-                                     (cudaStream_t)stream);
+  // The tcgen05 kernels round each dequantized element once to binary16; the error that leaves in a score grows with
+  // the softmax scale and stays well inside the library's 2e-3 output bound up to 2 / sqrt(d_qk).  Sharper scales
+  // take the kernels that multiply the codes exactly.
+  const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
+  cudaError_t e;
+  if (decode_mla_supported(y) && usual_scale)
+    e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out, out_dtype,
+                          lse, workspace, status_flags, (cudaStream_t)stream);
+  else if (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
+    e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out,
+                          out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
+  else
+    e = launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, nullptr, 0, 1, max_kv_len, window, q,
+                                 softmax_scale, out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 
@@ -139,9 +150,7 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
   // Q4KV_PREFILL_PATH=mma in the environment keeps the register-level mma.sync kernel for shapes both cover.
   static const bool force_mma = [] { const char* v = std::getenv("Q4KV_PREFILL_PATH"); return v && v[0] == 'm'; }();
-  // The tcgen05 kernel rounds each dequantized key and value once to binary16 (11 significant bits); the error that
-  // leaves in a score grows with the softmax scale, and stays well inside the library's 2e-3 output bound up to twice
-  // the usual 1/sqrt(d).  Sharper scales take the kernel that multiplies the codes exactly.
+  // same rule as in q4kv_decode_attention: sharp softmax scales take the kernel that multiplies the codes exactly
   const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
   cudaError_t e;
   if (prefill_umma_supported(y) && usual_scale && !force_mma)

@@ -144,4 +144,11 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
                                 const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
                                 float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
 
+// tcgen05 decode path for the MLA-latent cache (d_qk 576, d_v 512 aliasing K, one KV head, at most 16 query heads)
+bool decode_mla_supported(const Layout& y);
+size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len);
+cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                              const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale, void* out,
+                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
+
 }  // namespace q4kv

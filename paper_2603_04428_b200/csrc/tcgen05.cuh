@@ -78,7 +78,29 @@ __device__ inline void mma_f16_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32
       "r"(a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ inline void mma_f16_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // lane l of the warp <-> tensor-memory lane (taddr.lane + l); register j <-> column taddr.column + j
+__device__ inline void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ inline void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ inline void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -102,14 +124,18 @@ __device__ inline void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[31])
       : "memory");
 }
-// Shared-memory operand, K-major, no swizzle: element (n, k) of a 16-bit tile sits at byte
-//   (n % 8) * 16 + (n / 8) * sbo + (k / 8) * lbo + (k % 8) * 2.
+// Shared-memory operand without swizzle, 16-bit elements, built from 8 x 16-byte core matrices.
+//   K-major:  element (n, k) sits at byte (n % 8) * 16 + (n / 8) * sbo + (k / 8) * lbo + (k % 8) * 2;
+//   MN-major: element (n, k) sits at byte (k % 8) * 16 + (k / 8) * lbo + (n / 8) * sbo + (n % 8) * 2.
+// A [row][column] tile whose 16-byte pieces hold 8 consecutive columns is therefore K-major when the
+// columns are the contraction index and MN-major when the rows are.
 __device__ inline uint64_t smem_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
   return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
 }
-// f16 x f16 -> f32, both operands K-major, M x N tile
-__host__ __device__ constexpr uint32_t idesc_f16(int M, int N) {
-  return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// f16 x f16 -> f32, M x N tile; a_mn / b_mn = 1 for an MN-major operand (0: K-major)
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N, int a_mn = 0, int b_mn = 0) {
+  return (1u << 4) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
 }
 
 }  // namespace tc

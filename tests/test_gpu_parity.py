@@ -329,6 +329,41 @@ def test_bf16_output_mode(H):
     assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -8 + ATOL)      # half a bf16 ulp + the float32 bound
 
 
+@pytest.mark.parametrize("spec_args,lens,window", [
+    ((1, 16, 1, 576, 512, True), [5000, 700, 0, 63, 64, 65], 0),     # many key shares per agent, an empty agent, block edges
+    ((1, 16, 1, 576, 512, True), [9000, 300], 1000),                 # a window that starts inside a 64-key block
+    ((2, 8, 1, 576, 512, True), [2100], 0),                          # fewer than 16 heads, two layers
+])
+def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
+    """The MLA-latent decode kernel: one binary16 tile per 64 keys serves as key and as value operand."""
+    from paper_2603_04428_b200 import binding as B
+    p = Pair(H, spec_args, lens, seed=37).fill()
+    s = p.ospec
+    q = p.q(7, len(lens))
+    scale = 1.0 / math.sqrt(192)
+    for l in range(s.n_layers):
+        ref, lse_ref = O.decode_attention(p.opool, l, p.tabs, lens, window, f32(q), scale)
+        out, lse = p.dc.decode(l, lens, window, q, scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"layer {l}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref)
+    out16, _ = p.dc.decode(0, lens, window, q, scale, out_dtype=B.OUT_BF16)
+    out32, _ = p.dc.decode(0, lens, window, q, scale)
+    assert torch.allclose(out16.float(), out32.to(torch.bfloat16).float(), atol=1e-5, rtol=2.0 ** -7)
+    assert p.dc.read_flags() == 0
+    # a block id outside the pool poisons that agent only
+    if lens[0] > 256:
+        tabs = p.tabs.copy()
+        tabs[0, 1] = p.n_blocks + 3
+        t = H.dev(tabs)
+        bad, lse_bad = p.dc.decode(0, lens, window, q, scale, bt=B.batch(t))
+        hit = window == 0 or lens[0] - window < 512
+        if hit:
+            assert p.dc.read_flags() & B.FLAG_BAD_BLOCK
+            assert torch.all(bad[0] == 0) and torch.isneginf(lse_bad[0]).all()
+        assert torch.allclose(bad[1:], out32[1:], atol=1e-5)
+        p.dc.flags.zero_()
+
+
 # ---- prefill attention --------------------------------------------------------------------------
 @pytest.mark.parametrize("name,prefix,chunk,window", [
     ("gqa64", [300, 70], 40, 0),
