@@ -247,25 +247,31 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
       if (lane == 0) { mbar_arrive(&sm.v_full[s]); mbar_arrive(&sm.raw_free[r]); }
     }
   } else if (warp == kMmaWarp) {
-    // =============================== MMA issue (one thread) ====================================
-    if (lane == 0 && n_iter > 0) {
+    // =============================== MMA issue ==================================================
+    // The whole warp runs this code, so that operands are computed once for the warp, and one elected
+    // lane (always the same) issues the MMAs and the commits.
+    if (n_iter > 0) {
       constexpr uint32_t kIdescS = idesc_f16(128, 64), kIdescO = idesc_f16(128, 128);
       auto issue_qk = [&](int t, int s) {                // S_t = Q_t K^T
         const uint32_t kb = smem_u32(sm.khat[s]);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_f16_ts(tb + kColS + 64 * t, tb + kColQ + 64 * t + 8 * k, smem_desc(kb + 256 * k, 128, 2048), kIdescS, k > 0);
-        commit(&sm.s_full[t]);
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t bd = smem_desc(kb + 256 * k, 128, 2048);
+          if (elect_one()) mma_f16_ts(tb + kColS + 64 * t, tb + kColQ + 64 * t + 8 * k, bd, kIdescS, k > 0);
+        }
+        if (elect_one()) commit(&sm.s_full[t]);
       };
       auto issue_pv = [&](int t, int s, bool first) {    // O_t (+)= P_t V^
         const uint32_t vb = smem_u32(sm.vhat[s]);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          mma_f16_ts(tb + kColO + 128 * t, tb + kColS + 64 * t + 8 * k, smem_desc(vb + 256 * k, 128, 1024), kIdescO,
-                     (!first || k > 0) ? 1u : 0u);
-        commit(&sm.o_done[t]);
+        for (int k = 0; k < 4; ++k) {
+          const uint64_t bd = smem_desc(vb + 256 * k, 128, 1024);
+          if (elect_one()) mma_f16_ts(tb + kColO + 128 * t, tb + kColS + 64 * t + 8 * k, bd, kIdescO, (!first || k > 0) ? 1u : 0u);
+        }
+        if (elect_one()) commit(&sm.o_done[t]);
       };
       bool ok = mbar_wait(&sm.q_ready, 0, abort_flag) && mbar_wait(&sm.k_full[0], 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         fence_after_sync();
         issue_qk(0, 0);
@@ -276,12 +282,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         for (int t = 0; t < 2 && ok; ++t) {
           ok = mbar_wait(&sm.p_full[t], (uint32_t)j, abort_flag);
           if (ok && t == 0) ok = mbar_wait(&sm.v_full[s], (uint32_t)(j / kStages), abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           fence_after_sync();
           issue_pv(t, s, j == 0);
-          if (t == 1) commit(&sm.kv_free[s]);            // every MMA that reads stage s has been issued
+          if (t == 1 && elect_one()) commit(&sm.kv_free[s]);   // every MMA that reads stage s has been issued
           if (j + 1 < n_iter) {
-            if (t == 0) ok = mbar_wait(&sm.k_full[sn], (uint32_t)((j + 1) / kStages), abort_flag);
+            if (t == 0) ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_full[sn], (uint32_t)((j + 1) / kStages), abort_flag));
             if (!ok) break;
             fence_after_sync();
             issue_qk(t, sn);
@@ -444,7 +451,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
   __syncthreads();
   if (warp == kMmaWarp) {
     if (sm.abort_flag) {
-      if (lane == 0) {
+      if (elect_one()) {                                 // the lane that issued the MMAs
         commit(&sm.drain);
         for (uint32_t k = 0; k < kSpinLimit && !mbar_try_wait(&sm.drain, 0); ++k) {}
         raise_flag(P.flags, Q4KV_FLAG_INTERNAL);

@@ -33,10 +33,26 @@ __device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ inline bool mbar_test_wait(uint64_t* bar, uint32_t parity) {      // non-blocking
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// One lane of a converged warp (the same one every time).
+__device__ inline bool elect_one() {
+  uint32_t el;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(el));
+  return el != 0;
+}
 // Wait for completion number `use` (0, 1, 2, ...) of the barrier.  Returns false when the wait ran
 // out or another thread of the CTA has given up; the caller must then leave its loop.
 __device__ inline bool mbar_wait(uint64_t* bar, uint32_t use, volatile int* abort_flag) {
   const uint32_t parity = use & 1u;
+  if (mbar_test_wait(bar, parity)) return true;      // the blocking form costs ~150 clocks even when the phase is over
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u && *abort_flag) return false;
