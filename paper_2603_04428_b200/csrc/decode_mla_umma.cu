@@ -232,36 +232,40 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
       if (lane == 0) { mbar_arrive(&sm.k_full[s]); mbar_arrive(&sm.raw_free[r]); }
     }
   } else if (warp == kMmaWarp) {
-    // =============================== MMA issue (one thread) ====================================
-    if (lane == 0) {
+    // =============================== MMA issue ==================================================
+    // The whole warp runs this code (operands are computed once for the warp); one elected lane, always
+    // the same, issues the MMAs and the commits.
+    {
       constexpr uint32_t kIdescS = idesc_f16(64, 16, 0, 0), kIdescO = idesc_f16(128, 16, 1, 1);
       const uint32_t qb = smem_u32(sm.qtile), pb = smem_u32(sm.ptile);
       auto issue_pv = [&](int i) -> bool {               // O^T += K^(first 512 dims, read along the keys) x P^T
-        if (!mbar_wait(&sm.p_full, (uint32_t)i, abort_flag)) return false;
+        if (!__all_sync(0xffffffffu, mbar_wait(&sm.p_full, (uint32_t)i, abort_flag))) return false;
         fence_after_sync();
         const uint32_t kb = smem_u32(sm.khat[i % kStages]);
 #pragma unroll
         for (int T = 0; T < 4; ++T)
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_f16_ss(tb + kColO + 16 * T, smem_desc(kb + T * 16 * 128 + ks * 2 * kGroupStride, kGroupStride, 128),
-                       smem_desc(pb + ks * 256, 128, 1024), kIdescO, (i > 0 || ks > 0) ? 1u : 0u);
-        commit(&sm.o_done);
-        commit(&sm.kv_free[i % kStages]);
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t ad = smem_desc(kb + T * 16 * 128 + ks * 2 * kGroupStride, kGroupStride, 128);
+            const uint64_t bd = smem_desc(pb + ks * 256, 128, 1024);
+            if (elect_one()) mma_f16_ss(tb + kColO + 16 * T, ad, bd, kIdescO, (i > 0 || ks > 0) ? 1u : 0u);
+          }
+        if (elect_one()) { commit(&sm.o_done); commit(&sm.kv_free[i % kStages]); }
         return true;
       };
-      bool ok = mbar_wait(&sm.q_ready, 0, abort_flag);
+      bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_ready, 0, abort_flag));
       for (int j = 0; ok && j < n_iter; ++j) {
         const int s = j % kStages;
-        ok = mbar_wait(&sm.k_full[s], (uint32_t)(j / kStages), abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_full[s], (uint32_t)(j / kStages), abort_flag));
         if (!ok) break;
         fence_after_sync();
         const uint32_t kb = smem_u32(sm.khat[s]);
-#pragma unroll 4
-        for (int ks = 0; ks < kD / 16; ++ks)             // S^T = K^ Q^T
-          mma_f16_ss(tb + kColS + 16 * (j & 1), smem_desc(kb + ks * 256, 128, kGroupStride),
-                     smem_desc(qb + ks * 256, 128, kGroupStride), kIdescS, ks > 0);
-        commit(&sm.s_full[j & 1]);
+#pragma unroll 12
+        for (int ks = 0; ks < kD / 16; ++ks) {           // S^T = K^ Q^T
+          const uint64_t ad = smem_desc(kb + ks * 256, 128, kGroupStride), bd = smem_desc(qb + ks * 256, 128, kGroupStride);
+          if (elect_one()) mma_f16_ss(tb + kColS + 16 * (j & 1), ad, bd, kIdescS, ks > 0);
+        }
+        if (elect_one()) commit(&sm.s_full[j & 1]);
         if (j > 0) ok = issue_pv(j - 1);
       }
       if (ok) issue_pv(n_iter - 1);
@@ -426,7 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   __syncthreads();
   if (warp == kMmaWarp) {
     if (sm.abort_flag) {
-      if (lane == 0) {
+      if (elect_one()) {                                 // the lane that issued the MMAs
         commit(&sm.drain);
         for (uint32_t k = 0; k < kSpinLimit && !mbar_try_wait(&sm.drain, 0); ++k) {}
         raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
@@ -438,43 +442,77 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   }
 }
 
-// grid: (16 heads, n_agents); combines the records of one (agent, head)
-__global__ void __launch_bounds__(128) merge_mla_kernel(int Hq, int n_splits, const float* __restrict__ records,
-                                                       void* __restrict__ out, int out_dtype, float* __restrict__ lse) {
-  const int h = blockIdx.x, a = blockIdx.y;
+// grid: (16 heads, n_agents), 512 threads; combines the records of one (agent, head).  The records sit in L2 a
+// microsecond away, so nothing here is a chain of dependent loads: thread s fetches (m, l) of split s, the block
+// agrees on the weights, then four groups of 128 threads each take every fourth split with their loads issued
+// together, and the groups' sums meet in shared memory.
+constexpr int kMergeThreads = 512, kMaxSplits = 512;
+__global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_splits, const float* __restrict__ records,
+                                                                  void* __restrict__ out, int out_dtype,
+                                                                  float* __restrict__ lse) {
+  __shared__ float s_w[kMaxSplits];                      // weight of each split (0: empty)
+  __shared__ float s_red[kMergeThreads / 32][2];
+  __shared__ float4 s_acc[3][128];
+  __shared__ float s_ml[2];
+  const int h = blockIdx.x, a = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the records come from the preceding kernel
   if (h >= Hq) return;
   const float* rec = records + ((size_t)a * n_splits * kHeads + h) * kRecStride;
   const size_t step = (size_t)kHeads * kRecStride;       // between the splits of one head
-  float M = -INFINITY;
-  bool poisoned = false;
-  for (int s = 0; s < n_splits; ++s) {
-    M = fmaxf(M, rec[s * step + kDv]);
-    poisoned |= rec[s * step + kDv + 1] < 0.f;
+  float ms = -INFINITY, ls = 0.f;
+  if (tid < n_splits) { ms = rec[tid * step + kDv]; ls = rec[tid * step + kDv + 1]; }
+  float M = ms, bad = ls < 0.f ? 1.f : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o)); bad = fmaxf(bad, __shfl_xor_sync(0xffffffffu, bad, o)); }
+  if (lane == 0) { s_red[warp][0] = M; s_red[warp][1] = bad; }
+  __syncthreads();
+  M = s_red[0][0]; bad = s_red[0][1];
+#pragma unroll
+  for (int w = 1; w < kMergeThreads / 32; ++w) { M = fmaxf(M, s_red[w][0]); bad = fmaxf(bad, s_red[w][1]); }
+  const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
+  if (tid < n_splits) s_w[tid] = wgt;
+  float L = wgt * ls;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+  __syncthreads();                                       // s_red is read by everyone before it is reused
+  if (lane == 0) s_red[warp][0] = L;
+  __syncthreads();
+  if (tid == 0) {
+    float t = 0.f;
+    for (int w = 0; w < kMergeThreads / 32; ++w) t += s_red[w][0];
+    s_ml[0] = M; s_ml[1] = bad > 0.f ? 0.f : t;          // a poisoned split zeroes the row
   }
-  float L = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float ms = rec[s * step + kDv];
-    if (ms != -INFINITY) L += exp2f(ms - M) * rec[s * step + kDv + 1];
-  }
-  if (poisoned) L = 0.f;
-  const float inv = L > 0.f ? 1.f / L : 0.f;
-  const size_t out_index = ((size_t)a * Hq + h) * kDv;
+  const int grp = tid >> 7, d = 4 * (tid & 127);         // 128 threads x 4 consecutive dims per group
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  const int d = 4 * threadIdx.x;                         // 128 threads x 4 consecutive dims
-  if (inv > 0.f) {
-    for (int s = 0; s < n_splits; ++s) {
-      const float ms = rec[s * step + kDv];
-      if (ms == -INFINITY) continue;
-      const float wgt = exp2f(ms - M);
-      const float2 lo2 = *reinterpret_cast<const float2*>(rec + s * step + d);      // records are 8-byte aligned
-      const float2 hi2 = *reinterpret_cast<const float2*>(rec + s * step + d + 2);
-      acc.x = fmaf(wgt, lo2.x, acc.x); acc.y = fmaf(wgt, lo2.y, acc.y);
-      acc.z = fmaf(wgt, hi2.x, acc.z); acc.w = fmaf(wgt, hi2.y, acc.w);
+  for (int s0 = grp; s0 < n_splits; s0 += 16) {
+    float2 lo2[4], hi2[4];
+    float w4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int sp = s0 + 4 * u;
+      w4[u] = sp < n_splits ? s_w[sp] : 0.f;
+      lo2[u] = make_float2(0.f, 0.f); hi2[u] = make_float2(0.f, 0.f);
+      if (w4[u] > 0.f) {                                 // an empty split's record holds no data
+        lo2[u] = *reinterpret_cast<const float2*>(rec + sp * step + d);       // records are 8-byte aligned
+        hi2[u] = *reinterpret_cast<const float2*>(rec + sp * step + d + 2);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      acc.x = fmaf(w4[u], lo2[u].x, acc.x); acc.y = fmaf(w4[u], lo2[u].y, acc.y);
+      acc.z = fmaf(w4[u], hi2[u].x, acc.z); acc.w = fmaf(w4[u], hi2[u].y, acc.w);
     }
   }
+  if (grp > 0) s_acc[grp - 1][tid & 127] = acc;
+  __syncthreads();
+  if (grp > 0) return;
+  const float Lsum = s_ml[1];
+  const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+#pragma unroll
+  for (int g = 0; g < 3; ++g) { const float4 o = s_acc[g][tid]; acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
   acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+  const size_t out_index = ((size_t)a * Hq + h) * kDv;
   if (out_dtype == Q4KV_OUT_BF16) {
     const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc.x, acc.y), b1 = __floats2bfloat162_rn(acc.z, acc.w);
     uint2 v;
@@ -484,7 +522,7 @@ __global__ void __launch_bounds__(128) merge_mla_kernel(int Hq, int n_splits, co
   } else {
     *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + out_index + d) = acc;
   }
-  if (threadIdx.x == 0 && lse) lse[(size_t)a * Hq + h] = L > 0.f ? (M + log2f(L)) / kLog2e : -INFINITY;
+  if (tid == 0 && lse) lse[(size_t)a * Hq + h] = Lsum > 0.f ? (s_ml[0] + log2f(Lsum)) / kLog2e : -INFINITY;
 }
 
 struct MlaPlan { int n_splits, blocks_per_split; };
@@ -493,6 +531,7 @@ MlaPlan plan_mla(int n_agents, int max_kv_len, int window) {
   const int blocks = (span + 63) / 64 + 1;               // a window may straddle one more 64-key block
   int n_splits = (148 + n_agents - 1) / n_agents;        // about one CTA per SM
   if (n_splits > blocks) n_splits = blocks;
+  if (n_splits > kMaxSplits) n_splits = kMaxSplits;
   if (n_splits < 1) n_splits = 1;
   MlaPlan p;
   p.blocks_per_split = (blocks + n_splits - 1) / n_splits;
@@ -549,7 +588,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t mcfg = {};
   mcfg.gridDim = dim3(kHeads, b.n_agents);
-  mcfg.blockDim = dim3(128);
+  mcfg.blockDim = dim3(kMergeThreads);
   mcfg.stream = st;
   mcfg.attrs = attr;
   mcfg.numAttrs = pdl_enabled() ? 1 : 0;
