@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
         if (!ok) break;
         fence_after_sync();
         const uint32_t kb = smem_u32(sm.khat[s]);
-#pragma unroll 12
+#pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks) {           // S^T = K^ Q^T
           const uint64_t ad = smem_desc(kb + ks * 256, 128, kGroupStride), bd = smem_desc(qb + ks * 256, 128, kGroupStride);
           if (elect_one()) mma_f16_ss(tb + kColS + 16 * (j & 1), ad, bd, kIdescS, ks > 0);
