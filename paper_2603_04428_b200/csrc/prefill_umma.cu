@@ -365,40 +365,55 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
           if (pos > pq || (W > 0 && pos <= pq - W)) sr[c] = 0xff800000u;   // -inf
         }
       }
-      float cm = __uint_as_float(sr[0]);
+      // Probabilities against the current reference, and the block maximum beside them (the two are independent
+      // instruction streams); only when some row's maximum has outgrown its reference is the reference moved,
+      // the accumulator rescaled and the probabilities taken again.  The scores stay in registers meanwhile.
+      float sum = 0.f;
+      uint32_t pr[32];
+      auto probabilities = [&](float neg_m) {
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-      for (int c = 1; c < 64; ++c) cm = fmaxf(cm, __uint_as_float(sr[c]));
+        for (int c = 0; c < 32; c += 2) {                // all on the special-function unit: a polynomial on the FMA
+          // pipe for half of them was measured 19 % slower (the issue slots are the scarcer resource here)
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), kappa, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), kappa, neg_m));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 2]), kappa, neg_m));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 3]), kappa, neg_m));
+          s0 += p0; s1 += p1; s2 += p2; s3 += p3;
+          pr[c] = f32x2_to_h2(p0, p1);
+          pr[c + 1] = f32x2_to_h2(p2, p3);
+        }
+        sum = (s0 + s1) + (s2 + s3);
+      };
+      probabilities(m_ref == -INFINITY ? 0.f : -m_ref);
+      float cm4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
+#pragma unroll
+      for (int c = 4; c < 64; ++c) cm4[c & 3] = fmaxf(cm4[c & 3], __uint_as_float(sr[c]));
+      float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
       if (cm != -INFINITY) cm *= kappa;                  // kappa > 0
       const float m_new = fmaxf(m_ref, cm);
       const bool grow = m_new > m_ref + kLazy || (m_ref == -INFINITY && m_new != -INFINITY);
-      if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        // rescale this warp's accumulator rows: the previous block's value product must have landed
-        if (!__all_sync(0xffffffffu, mbar_wait(&sm.o_done[t], (uint32_t)(j - 1), abort_flag))) { ok = false; break; }
-        fence_after_sync();
-        const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;             // m_ref = -inf: 0
+      if (__any_sync(0xffffffffu, grow)) {
+        if (j > 0) {
+          // rescale this warp's accumulator rows: the previous block's value product must have landed
+          if (!__all_sync(0xffffffffu, mbar_wait(&sm.o_done[t], (uint32_t)(j - 1), abort_flag))) { ok = false; break; }
+          fence_after_sync();
+          const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;           // m_ref = -inf: 0
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
-          uint32_t orow[32];
-          tmem_ld32(lane_addr + kColO + 128 * t + 32 * part, orow);
-          wait_ld();
+          for (int part = 0; part < 4; ++part) {
+            uint32_t orow[32];
+            tmem_ld32(lane_addr + kColO + 128 * t + 32 * part, orow);
+            wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * f);
-          tmem_st32(lane_addr + kColO + 128 * t + 32 * part, orow);
+            for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * f);
+            tmem_st32(lane_addr + kColO + 128 * t + 32 * part, orow);
+          }
+          if (grow) l *= f;
         }
-        if (grow) l *= f;
+        if (grow) m_ref = m_new;
+        probabilities(m_ref == -INFINITY ? 0.f : -m_ref);
       }
-      if (grow) m_ref = m_new;
-      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
-      float sum0 = 0.f, sum1 = 0.f;
-      uint32_t pr[32];
-#pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), kappa, neg_m));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), kappa, neg_m));
-        sum0 += p0; sum1 += p1;
-        pr[c] = f32x2_to_h2(p0, p1);
-      }
-      l += sum0 + sum1;
+      l += sum;
       tmem_st32(lane_addr + kColS + 64 * t, pr);         // P_t overlays the first 32 columns of S_t
       wait_st();
       fence_before_sync();
