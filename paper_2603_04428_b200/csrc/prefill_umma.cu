@@ -20,10 +20,10 @@
 //     f32 accumulators S_t and O_t live in tensor memory (512 columns: O 2 x 128, S 2 x 64, Q 2 x 64;
 //     P_t overlays S_t).  Only the B operands come from shared memory, which keeps the operand
 //     traffic at half of the shared-memory bandwidth and leaves the rest to the dequantize warps.
-//   * Eight softmax warps, one thread per score row (a tensor-memory lane): load the 64 scores,
-//     mask, online softmax with a lazily updated reference maximum (the accumulator is rescaled
-//     only when the maximum has grown by more than 2^8), write P_t as packed binary16.  The two
-//     tiles alternate, so one tile's softmax overlaps the other tile's MMAs.
+//   * Sixteen softmax warps, two threads per score row (a tensor-memory lane; each takes 32 of the
+//     64 scores): mask, online softmax with a lazily updated reference maximum (the accumulator is
+//     rescaled only when the maximum has grown by more than 2^8), write P_t as packed binary16.
+//     The two tiles alternate, so one tile's softmax overlaps the other tile's MMAs.
 //   * One warp streams the raw blocks through a small ring with bulk asynchronous copies.
 // All hand-offs are mbarriers; every wait is bounded and a wait that runs out raises
 // Q4KV_FLAG_INTERNAL, drains the tensor pipe and frees the tensor memory before the CTA returns.
@@ -36,9 +36,9 @@ namespace {
 
 using namespace tc;
 
-constexpr int kSoftmaxWarps = 8, kDequantWarps = 4;
+constexpr int kSoftmaxWarps = 16, kDequantWarps = 4;
 constexpr int kMmaWarp = kSoftmaxWarps + kDequantWarps, kLoadWarp = kMmaWarp + 1;
-constexpr int kThreads = (kLoadWarp + 1) * 32;           // 448
+constexpr int kThreads = (kLoadWarp + 1) * 32;           // 704
 constexpr int kStages = 3;                               // K^ / V^ tiles in flight
 constexpr int kRawSlots = 4;                             // raw 64-key blocks in flight
 constexpr int kChunkBytes = 4608;                        // d = 128: [Kc 2048 | Ksb 256 | Vc 2048 | Vsb 256]
@@ -73,6 +73,8 @@ struct UmmaSmem {
   uint64_t s_full[2], p_full[2], o_done[2], q_ready, drain;
   uint32_t tmem_base;
   int bad[kRawSlots];
+  float xchg[2][2][2][128];                              // [tile][parity][column half][row]: maxima / sums of the two threads of a row
+  int stop[2][3], spoiled[2];
   int abort_flag, poisoned;
 };
 
@@ -138,8 +140,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.k_full[s], kDequantWarps); mbar_init(&sm.v_full[s], kDequantWarps); mbar_init(&sm.kv_free[s], 1);
     }
-    for (int t = 0; t < 2; ++t) { mbar_init(&sm.s_full[t], 1); mbar_init(&sm.p_full[t], 128); mbar_init(&sm.o_done[t], 1); }
-    mbar_init(&sm.q_ready, 256);
+    for (int t = 0; t < 2; ++t) { mbar_init(&sm.s_full[t], 1); mbar_init(&sm.p_full[t], 256); mbar_init(&sm.o_done[t], 1); }
+    mbar_init(&sm.q_ready, 512);
+    for (int i = 0; i < 6; ++i) (&sm.stop[0][0])[i] = 0;
+    sm.spoiled[0] = 0; sm.spoiled[1] = 0;
     mbar_init(&sm.drain, 1);
     sm.abort_flag = 0; sm.poisoned = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -254,7 +258,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
       constexpr uint32_t kIdescS = idesc_f16(128, 64), kIdescO = idesc_f16(128, 128);
       auto issue_qk = [&](int t, int s) {                // S_t = Q_t K^T
         const uint32_t kb = smem_u32(sm.khat[s]);
-#pragma unroll
+#pragma unroll                                           // rolled, every MMA waits for its own operand arithmetic: 2x slower
         for (int k = 0; k < 8; ++k) {
           const uint64_t bd = smem_desc(kb + 256 * k, 128, 2048);
           if (elect_one()) mma_f16_ts(tb + kColS + 64 * t, tb + kColQ + 64 * t + 8 * k, bd, kIdescS, k > 0);
@@ -297,22 +301,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
       }
     }
   } else {
-    // =============================== softmax warps: one thread per score row ===================
-    const int t = warp >> 2;                             // tile
+    // =============================== softmax warps: two threads per score row ===================
+    // Warp w: tile t = w / 8, column half = (w / 4) % 2, tensor-memory lanes 32 (w % 4) ...  The two threads of a
+    // row exchange their block maxima (and at the end their sums) through shared memory; the 256 threads of a
+    // tile meet at a named barrier once per block, and they leave the loop together (one of them samples the
+    // give-up flag before the barrier).
+    const int t = warp >> 3, half = (warp >> 2) & 1;
     const int row = (warp & 3) * 32 + lane;              // tensor-memory lane
     const uint32_t lane_addr = tb + ((uint32_t)((warp & 3) * 32) << 16);
     const int h = row / tile_q, i = i_min + t * tile_q + row % tile_q;
     const bool valid = i < q_len && !bad_len;
     const int pq = prefix + i;                           // this row's position
+    const bool sampler = (warp & 7) == 0 && lane == 0;   // one thread per tile
+    auto tile_barrier = [&]() { asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory"); };
     float kappa;                                         // score in log2 units = S * kappa
     {
-      // ---- stage the query row: bf16 -> binary16 times a power of two, element order (0,4,1,5,2,6,3,7) ----
-      const uint16_t* qrow = P.q + ((size_t)(q0 + (valid ? i : 0)) * y.Hq + (size_t)hk * n_rep + h) * 128;
-      uint32_t qa[64];
+      // ---- stage this thread's half of the query row: bf16 -> binary16 times a power of two, element order
+      //      (0,4,1,5,2,6,3,7) inside every eight ----
+      const uint16_t* qrow = P.q + ((size_t)(q0 + (valid ? i : 0)) * y.Hq + (size_t)hk * n_rep + h) * 128 + 64 * half;
+      uint32_t qa[32];
       float mx = 0.f;
       if (valid) {
 #pragma unroll
-        for (int w = 0; w < 16; ++w) {
+        for (int w = 0; w < 8; ++w) {
           const uint4 v = *reinterpret_cast<const uint4*>(qrow + 8 * w);
           qa[4 * w] = v.x; qa[4 * w + 1] = v.y; qa[4 * w + 2] = v.z; qa[4 * w + 3] = v.w;
           mx = fmaxf(mx, fmaxf(fmaxf(fabsf(__uint_as_float(v.x << 16)), fabsf(__uint_as_float(v.x & 0xffff0000u))),
@@ -322,15 +333,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         }
       } else {
 #pragma unroll
-        for (int w = 0; w < 64; ++w) qa[w] = 0u;
+        for (int w = 0; w < 32; ++w) qa[w] = 0u;
       }
+      sm.xchg[t][1][half][row] = mx;                     // slot 1: block 0 of the loop below writes slot 0
+      tile_barrier();
+      mx = fmaxf(mx, sm.xchg[t][1][half ^ 1][row]);
       int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
       if (mx == 0.f) ex = 0;
       ex = min(max(ex, -100), 100);
       const float sf = __uint_as_float((uint32_t)(127 + 8 - ex) << 23);      // 256 <= max |q| * sf < 512
       kappa = P.scale_log2 * __uint_as_float((uint32_t)(127 - 8 + ex) << 23);
 #pragma unroll
-      for (int w = 0; w < 16; ++w) {
+      for (int w = 0; w < 8; ++w) {
         // elements 8w..8w+7 arrive as bf16 pairs (0,1) (2,3) (4,5) (6,7); columns hold (0,4) (1,5) (2,6) (3,7)
         const uint32_t u01 = qa[4 * w], u23 = qa[4 * w + 1], u45 = qa[4 * w + 2], u67 = qa[4 * w + 3];
         const float x0 = __uint_as_float(u01 << 16) * sf, x1 = __uint_as_float(u01 & 0xffff0000u) * sf;
@@ -340,41 +354,36 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         qa[4 * w] = f32x2_to_h2(x0, x4); qa[4 * w + 1] = f32x2_to_h2(x1, x5);
         qa[4 * w + 2] = f32x2_to_h2(x2, x6); qa[4 * w + 3] = f32x2_to_h2(x3, x7);
       }
-      tmem_st32(lane_addr + kColQ + 64 * t, qa);
-      tmem_st32(lane_addr + kColQ + 64 * t + 32, qa + 32);
+      tmem_st32(lane_addr + kColQ + 64 * t + 32 * half, qa);
       wait_st();
       fence_before_sync();
       mbar_arrive(&sm.q_ready);
     }
     float m_ref = -INFINITY, l = 0.f;                    // p = 2^(s - m_ref); m_ref trails the true maximum by at most kLazy
-    bool ok = true;
     for (int j = 0; j < n_iter; ++j) {
-      // the tensor-memory loads and stores below are warp-wide: the warp leaves the loop together
-      if (!__all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], (uint32_t)j, abort_flag))) { ok = false; break; }
+      mbar_wait(&sm.s_full[t], (uint32_t)j, abort_flag); // a wait that runs out raises the give-up flag; all leave below
       fence_after_sync();
-      uint32_t sr[64];
-      tmem_ld32(lane_addr + kColS + 64 * t, sr);
-      tmem_ld32(lane_addr + kColS + 64 * t + 32, sr + 32);
+      uint32_t sr[32];
+      tmem_ld32(lane_addr + kColS + 64 * t + 32 * half, sr);
       wait_ld();
-      const int pos0 = (it0 + j) * 64;
-      // column c of the block is key pos0 + (c & ~7) + elem_of(c & 7); causal and window masks on edge blocks only
-      if (pos0 + 63 > pq || (W > 0 && pos0 <= pq - W)) {
+      const int pos0 = (it0 + j) * 64 + 32 * half;
+      // column c of this half is key pos0 + (c & ~7) + elem_of(c & 7); causal and window masks on edge blocks only
+      if (pos0 + 31 > pq || (W > 0 && pos0 <= pq - W)) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
+        for (int c = 0; c < 32; ++c) {
           const int pos = pos0 + (c & ~7) + elem_of(c & 7);
           if (pos > pq || (W > 0 && pos <= pq - W)) sr[c] = 0xff800000u;   // -inf
         }
       }
-      // Probabilities against the current reference, and the block maximum beside them (the two are independent
-      // instruction streams); only when some row's maximum has outgrown its reference is the reference moved,
-      // the accumulator rescaled and the probabilities taken again.  The scores stay in registers meanwhile.
+      // Probabilities against the current reference, and the block maximum beside them (independent instruction
+      // streams); only when some row's maximum has outgrown its reference is the reference moved, the accumulator
+      // rescaled and the probabilities taken again.  The scores stay in registers meanwhile.
       float sum = 0.f;
-      uint32_t pr[32];
+      uint32_t pr[16];
       auto probabilities = [&](float neg_m) {
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {                // all on the special-function unit: a polynomial on the FMA
-          // pipe for half of them was measured 19 % slower (the issue slots are the scarcer resource here)
+        for (int c = 0; c < 16; c += 2) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c]), kappa, neg_m));
           const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), kappa, neg_m));
           const float p2 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 2]), kappa, neg_m));
@@ -388,25 +397,30 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
       probabilities(m_ref == -INFINITY ? 0.f : -m_ref);
       float cm4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
 #pragma unroll
-      for (int c = 4; c < 64; ++c) cm4[c & 3] = fmaxf(cm4[c & 3], __uint_as_float(sr[c]));
+      for (int c = 4; c < 32; ++c) cm4[c & 3] = fmaxf(cm4[c & 3], __uint_as_float(sr[c]));
       float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
+      sm.xchg[t][j & 1][half][row] = cm;
+      if (sampler) sm.stop[t][j % 3] = *abort_flag;
+      tile_barrier();                                    // also: every score of the tile has been read (P overlays S)
+      if (sm.stop[t][j % 3]) break;
+      cm = fmaxf(cm, sm.xchg[t][j & 1][half ^ 1][row]);
       if (cm != -INFINITY) cm *= kappa;                  // kappa > 0
       const float m_new = fmaxf(m_ref, cm);
       const bool grow = m_new > m_ref + kLazy || (m_ref == -INFINITY && m_new != -INFINITY);
       if (__any_sync(0xffffffffu, grow)) {
         if (j > 0) {
-          // rescale this warp's accumulator rows: the previous block's value product must have landed
-          if (!__all_sync(0xffffffffu, mbar_wait(&sm.o_done[t], (uint32_t)(j - 1), abort_flag))) { ok = false; break; }
+          // rescale this thread's half of the accumulator row: the previous block's value product must have landed
+          mbar_wait(&sm.o_done[t], (uint32_t)(j - 1), abort_flag);
           fence_after_sync();
           const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;           // m_ref = -inf: 0
 #pragma unroll 1
-          for (int part = 0; part < 4; ++part) {
+          for (int part = 0; part < 2; ++part) {
             uint32_t orow[32];
-            tmem_ld32(lane_addr + kColO + 128 * t + 32 * part, orow);
+            tmem_ld32(lane_addr + kColO + 128 * t + 64 * half + 32 * part, orow);
             wait_ld();
 #pragma unroll
             for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * f);
-            tmem_st32(lane_addr + kColO + 128 * t + 32 * part, orow);
+            tmem_st32(lane_addr + kColO + 128 * t + 64 * half + 32 * part, orow);
           }
           if (grow) l *= f;
         }
@@ -414,23 +428,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         probabilities(m_ref == -INFINITY ? 0.f : -m_ref);
       }
       l += sum;
-      tmem_st32(lane_addr + kColS + 64 * t, pr);         // P_t overlays the first 32 columns of S_t
+      tmem_st16(lane_addr + kColS + 64 * t + 16 * half, pr);   // P_t overlays the first 32 columns of S_t
       wait_st();
       fence_before_sync();
       mbar_arrive(&sm.p_full[t]);
     }
-    // ---- normalise and write this row ----
+    // ---- normalise and write this thread's half of the row ----
+    bool ok = !*abort_flag;
     if (ok && n_iter > 0) ok = mbar_wait(&sm.o_done[t], (uint32_t)(n_iter - 1), abort_flag);
-    ok = __all_sync(0xffffffffu, ok);                    // the loads below are warp-wide
+    const int slot = n_iter & 1;                         // not the slot the last block used
+    sm.xchg[t][slot][half][row] = l;
+    if (!ok) sm.spoiled[t] = 1;                          // anyone who gave up spoils the tile
+    tile_barrier();
+    ok = sm.spoiled[t] == 0;                             // uniform over the tile: the loads below are warp-wide
+    l += sm.xchg[t][slot][half ^ 1][row];
     if (ok) fence_after_sync();
     const bool zero = !ok || n_iter == 0 || sm.poisoned != 0 || l <= 0.f;
     const float inv = zero ? 0.f : 1.f / l;
-    const size_t orow_index = ((size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h) * 128;
+    const size_t orow_index = ((size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h) * 128 + 64 * half;
 #pragma unroll 1
-    for (int part = 0; part < 4; ++part) {
+    for (int part = 0; part < 2; ++part) {
       uint32_t orow[32];
       if (ok && n_iter > 0) {
-        tmem_ld32(lane_addr + kColO + 128 * t + 32 * part, orow);
+        tmem_ld32(lane_addr + kColO + 128 * t + 64 * half + 32 * part, orow);
         wait_ld();
       }
       if (i >= q_len) continue;
@@ -458,7 +478,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
                                  __uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
       }
     }
-    if (i < q_len && P.lse) P.lse[(size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h] = zero ? -INFINITY : (m_ref + log2f(l)) / kLog2e;
+    if (half == 0 && i < q_len && P.lse)
+      P.lse[(size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h] = zero ? -INFINITY : (m_ref + log2f(l)) / kLog2e;
   }
 
   // ---- teardown: nothing may be in flight in the tensor pipe when the columns are given back ----
