@@ -253,6 +253,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   const uint32_t kq_lane = lr * 16 + warp * kGroupStride + lm * 128;        // scores: key octet = warp; + 512 per two k-steps
   const uint32_t kv_lane = lr * 16 + (lm & 1) * kGroupStride + (8 * warp + (lm >> 1)) * 128;   // values: + 2 ks octets, + 256 per dim-core pair
 
+  // The queries never change: the A fragments of every other k-step live in registers for the whole launch (all of
+  // them would not fit), the rest is re-read from shared memory per block.
+  uint32_t qa[kD / 32][4];
+#pragma unroll
+  for (int kk = 0; kk < kD / 32; ++kk) ldmatrix_x4(qa[kk], q_lane + (2 * kk) * 256);
   float kap[2], m_ref[2], l_part[2];                     // heads g and g + 8
   kap[0] = sm.kappa[g]; kap[1] = sm.kappa[g + 8];
   m_ref[0] = -INFINITY; m_ref[1] = -INFINITY; l_part[0] = 0.f; l_part[1] = 0.f;
@@ -307,11 +312,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
       const uint32_t kb = smem_u32(sm.khat[s]) + kq_lane;
 #pragma unroll
       for (int kk = 0; kk < kD / 32; ++kk) {
-        uint32_t bq[4], a0[4], a1[4];
+        uint32_t bq[4], a1[4];
         ldmatrix_x4(bq, kb + kk * 512);
-        ldmatrix_x4(a0, q_lane + (2 * kk) * 256);
         ldmatrix_x4(a1, q_lane + (2 * kk + 1) * 256);
-        mma_f16(acc[(2 * kk) & 3], a0, bq[0], bq[1]);
+        mma_f16(acc[(2 * kk) & 3], qa[kk], bq[0], bq[1]);
         mma_f16(acc[(2 * kk + 1) & 3], a1, bq[2], bq[3]);
       }
 #pragma unroll
