@@ -9,7 +9,7 @@
 namespace q4kv {
 namespace tc {
 
-constexpr uint32_t kSpinLimit = 1u << 22;     // every wait gives up after this many polls
+constexpr uint32_t kSpinLimit = 1u << 17;     // every wait gives up after this many polls (each up to 20 us: ~2.6 s)
 
 __device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -24,12 +24,16 @@ __device__ inline void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
                "r"(bytes)
                : "memory");
 }
+// Blocking form: the thread is suspended until the phase completes or about kSuspendNs have passed, so a waiting
+// warp does not take issue slots from the working ones (without the hint it returns after a few dozen clocks, and
+// the spin loops were a third of all instructions executed).
+constexpr uint32_t kSuspendNs = 20000;
 __device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
       : "memory");
   return ok != 0;
 }
@@ -55,7 +59,7 @@ __device__ inline bool mbar_wait(uint64_t* bar, uint32_t use, volatile int* abor
   if (mbar_test_wait(bar, parity)) return true;      // the blocking form costs ~150 clocks even when the phase is over
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u && *abort_flag) return false;
+    if (*abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
