@@ -137,6 +137,26 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
                           void* workspace, size_t workspace_bytes,
                           int32_t* status_flags, void* stream);
 
+/* Update-and-fetch for one new token per agent in a single launch (Section 3.4: the cache's
+ * update_and_fetch -- quantize the step's new K/V rows into the cache, then attend over it).
+ * Equivalent to q4kv_quantize_append(pos = kv_lens - 1, one row per agent) followed by
+ * q4kv_decode_attention(kv_lens): the pool ends up with the same bytes and the output is the same
+ * attention, but the new token is quantized by the warp that attends its 32-token chunk, so no
+ * second kernel runs.
+ *   kv_lens  [A]  lengths INCLUDING the new token (it sits at position kv_len - 1); kv_len == 0:
+ *                 nothing is appended for that agent
+ *   k_new    bf16 [A][n_kv_heads][d_qk], v_new bf16 [A][n_kv_heads][d_v]: row a is agent a's token
+ * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256}, at
+ * most four query heads per KV head, V not aliasing K; anything else returns Q4KV_EUNSUPPORTED
+ * and the caller makes the two calls.  Two agents must not share the block that is written. */
+int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
+                                 const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                                 int32_t window, const void* k_new, const void* v_new,
+                                 const void* q, float softmax_scale,
+                                 void* out, int32_t out_dtype, float* lse,
+                                 void* workspace, size_t workspace_bytes,
+                                 int32_t* status_flags, void* stream);
+
 /* Decode attention without a caller-supplied workspace.  The paper has no counterpart: this entry
  * point exists for hosts that cannot allocate device memory when they call -- a runtime that
  * carved up all of its device memory at start-up, a plugin that must not touch its host's

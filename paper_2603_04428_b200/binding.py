@@ -23,7 +23,7 @@ OUT_F32, OUT_BF16 = 0, 1
 EXPORTS = [
     "q4kv_status_string", "q4kv_pool_bytes", "q4kv_packed_bytes", "q4kv_workspace_bytes",
     "q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack", "q4kv_unpack",
-    "q4kv_decode_attention_static",
+    "q4kv_decode_attention_static", "q4kv_append_decode_attention",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.q4kv_quantize_append.argtypes = [sp, vp, i32, i32, bp, vp, vp, i32, vp, vp, vp, vp]
         L.q4kv_decode_attention.restype = ctypes.c_int
         L.q4kv_decode_attention.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, f32, vp, i32, vp, vp, sz, vp, vp]
+        L.q4kv_append_decode_attention.restype = ctypes.c_int
+        L.q4kv_append_decode_attention.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, vp, vp, f32, vp, i32, vp, vp,
+                                                   sz, vp, vp]
         L.q4kv_decode_attention_static.restype = ctypes.c_int
         L.q4kv_decode_attention_static.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, f32, vp, i32, vp, vp, vp]
         L.q4kv_prefill_attention.restype = ctypes.c_int
@@ -138,6 +141,18 @@ def q4kv_decode_attention(spec, pool, n_blocks, layer, bt: Batch, kv_lens, max_k
                                        out_dtype, _ptr(lse), _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream()),
            "q4kv_decode_attention")
+
+
+def q4kv_append_decode_attention(spec, pool, n_blocks, layer, bt: Batch, kv_lens, max_kv_len, window, k_new, v_new, q,
+                                 softmax_scale, out, out_dtype, lse, workspace, status_flags=None):
+    """Update-and-fetch in one launch: quantize one new token per agent into the cache (position kv_len - 1) and
+    attend over the cache including it."""
+    _check(lib().q4kv_append_decode_attention(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt),
+                                              _ptr(kv_lens), max_kv_len, window, _ptr(k_new), _ptr(v_new), _ptr(q),
+                                              softmax_scale, _ptr(out), out_dtype, _ptr(lse), _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), _ptr(status_flags),
+                                              _stream()),
+           "q4kv_append_decode_attention")
 
 
 def q4kv_decode_attention_static(spec, pool, n_blocks, layer, bt: Batch, kv_lens, max_kv_len, window, q, softmax_scale,

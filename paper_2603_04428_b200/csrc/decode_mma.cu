@@ -37,6 +37,7 @@
 #include <cstdlib>
 
 #include "q4kv_layout.cuh"
+#include "quantize_core.cuh"
 
 namespace q4kv {
 
@@ -305,6 +306,8 @@ struct DecodeParams {
   int out_dtype;
   float* lse;
   int32_t* flags;
+  const uint16_t* k_new;      // fused append: bf16 [A][Hkv][D] rows of the token at position kv_len - 1 (null: none)
+  const uint16_t* v_new;
 };
 
 __host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
@@ -391,6 +394,61 @@ __device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], f
     if ((w & 7) == 0) qsum[h][gi] = sum * scale_log2;
     if (w == 0) kappa[h] = scale_log2 * __uint_as_float((uint32_t)(127 + 13 + ex) << 23);  // 2^24 / sf
   }
+}
+
+// Fused append (one new token per agent): the warp that owns the chunk holding an agent's newest position
+// quantizes that token's K and V rows (Section 3.2 quantizer, the same device function the append kernel uses) and
+// writes them into the chunk -- in shared memory for this launch, in the pool for the following ones.  Every chunk
+// is processed by exactly one warp of the grid, so nobody else reads or writes these words during the launch.
+// Eight consecutive lanes own one 64-element group; the 8-lane shuffles never straddle K and V (D / 8 is a multiple
+// of 16).  The value codes are token-packed: one nibble of each of the row's D words is replaced.
+template <int G>
+__device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, const Layout& y,
+                                              const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                                              int a, int hk, int tau, int lane) {
+  constexpr int D = 64 * G, W = D / 8;                   // words per row
+  const size_t row = ((size_t)a * y.Hkv + hk) * D;
+#pragma unroll
+  for (int base = 0; base < 2 * W; base += 32) {
+    const int idx = base + lane;
+    const bool is_v = idx >= W;
+    const int w = idx % W;
+    float x[8];
+    {
+      const uint4 v = *reinterpret_cast<const uint4*>((is_v ? v_new : k_new) + row + 8 * w);
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(u[i] << 16); x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
+    }
+    const QuantOut qo = quantize_eight(x);
+    const uint32_t sb = *reinterpret_cast<const uint32_t*>(&qo.sb);
+    if (!is_v) {
+      const uint32_t at = y.off_kc + 4u * k_word_offset(tau, w, G);
+      *reinterpret_cast<uint32_t*>(chunk + at) = qo.word;
+      *reinterpret_cast<uint32_t*>(gchunk + at) = qo.word;
+      if ((w & 7) == 0) {
+        const uint32_t sat = y.off_ksb + 4u * sb_offset(tau, w >> 3, G);
+        *reinterpret_cast<uint32_t*>(chunk + sat) = sb;
+        *reinterpret_cast<uint32_t*>(gchunk + sat) = sb;
+      }
+    } else {
+      const int shift = 4 * (tau & 7);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t at = y.off_vc + 4u * v_word_offset(tau >> 3, 8 * w + e);
+        const uint32_t old = *reinterpret_cast<const uint32_t*>(chunk + at);
+        const uint32_t nw = (old & ~(0xFu << shift)) | (((qo.word >> (4 * e)) & 0xFu) << shift);
+        *reinterpret_cast<uint32_t*>(chunk + at) = nw;
+        *reinterpret_cast<uint32_t*>(gchunk + at) = nw;
+      }
+      if ((w & 7) == 0) {
+        const uint32_t sat = y.off_vsb + 4u * sb_offset(tau, w >> 3, G);
+        *reinterpret_cast<uint32_t*>(chunk + sat) = sb;
+        *reinterpret_cast<uint32_t*>(gchunk + sat) = sb;
+      }
+    }
+  }
+  __syncwarp();                                          // the patched chunk is read by the same warp
 }
 
 // One 32-token chunk against this warp's query fragments.
@@ -938,6 +996,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       poisoned = true;
     } else {
       const int c = seg.c0 + (k - seg.k0);
+      if (P.k_new != nullptr && c == ((seg.n - 1) >> 5)) {
+        // the chunk of the agent's newest position: its block id has passed the producer's check
+        const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
+        uint8_t* gchunk = const_cast<uint8_t*>(head_block(P.pool, y, P.layer, blk, seg.hk)) + (size_t)(c & 7) * kChunkBytes;
+        append_new_token<G>(sm.ring + (size_t)slot * kChunkBytes, gchunk, y, P.k_new, P.v_new, seg.a, seg.hk,
+                            (seg.n - 1) & 31, lane);
+      }
       process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, c * 32, seg.lo, seg.n, g, tid, qa, qs, kap, split_mask, st);
     }
     __syncwarp();
@@ -998,7 +1063,8 @@ size_t decode_mma_workspace_bytes(const Layout& y, int n_agents) {
 
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
-                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st) {
+                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
+                              const void* k_new, const void* v_new) {
   if (b.n_agents <= 0) return cudaSuccess;
   const size_t pairs = (size_t)b.n_agents * y.Hkv;
   const size_t ticket_bytes = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
@@ -1008,6 +1074,7 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e;
   P.tickets = (int32_t*)ws; P.partials = (float*)((uint8_t*)ws + ticket_bytes);
   P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
+  P.k_new = (const uint16_t*)k_new; P.v_new = (const uint16_t*)v_new;
   const int span = (window > 0 && window + 32 < max_kv_len) ? window + 32 : max_kv_len;
   const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
   const int grid = (int)(units < kMaxCtas ? (units < 1 ? 1 : units) : kMaxCtas);

@@ -126,6 +126,32 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 
+int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
+                                 const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                                 int32_t window, const void* k_new, const void* v_new,
+                                 const void* q, float softmax_scale,
+                                 void* out, int32_t out_dtype, float* lse,
+                                 void* workspace, size_t workspace_bytes,
+                                 int32_t* status_flags, void* stream) {
+  int rc = check_spec(spec);
+  if (rc) return rc;
+  if ((rc = check_batch(batch))) return rc;
+  if (!pool || n_blocks <= 0 || layer < 0 || layer >= spec->n_layers || window < 0 || max_kv_len < 0) return Q4KV_EINVAL;
+  if (out_dtype != Q4KV_OUT_F32 && out_dtype != Q4KV_OUT_BF16) return Q4KV_EINVAL;
+  if (batch->n_agents == 0) return Q4KV_OK;
+  if (!kv_lens || !q || !out || !workspace || !k_new || !v_new) return Q4KV_EINVAL;
+  if (!aligned16(pool) || !aligned16(q) || !aligned16(out) || !aligned16(workspace) || !aligned16(k_new) || !aligned16(v_new))
+    return Q4KV_EINVAL;
+  const int cap = batch->max_blocks * kBlockTokens;
+  if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
+  const Layout y = make_layout(*spec, n_blocks);
+  if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks)) return Q4KV_EUNSUPPORTED;
+  if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
+  const cudaError_t e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,
+                                          out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream, k_new, v_new);
+  return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
+}
+
 int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                            const q4kv_batch* batch, const int32_t* kv_lens, const int32_t* q_offs,
                            int32_t total_q, int32_t max_q_len, int32_t max_kv_len,

@@ -129,7 +129,8 @@ bool pdl_enabled();
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents);
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
-                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
+                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
+                              const void* k_new = nullptr, const void* v_new = nullptr);
 
 // tensor-core prefill path (d_qk = d_v = 128, at most 4 query heads per KV head)
 bool prefill_mma_supported(const Layout& y);

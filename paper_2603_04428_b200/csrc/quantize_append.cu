@@ -8,56 +8,13 @@
 // min/max with three shuffles.  Every arithmetic step is a single rounded binary32
 // operation in the documented order so that codes/scales/biases are reproducible.
 #include "q4kv_layout.cuh"
+#include "quantize_core.cuh"
 
 namespace q4kv {
 
 namespace {
 
 constexpr int kThreads = 256;
-
-struct QuantOut { uint32_t word; __half2 sb; };
-
-// x[8]: eight consecutive elements owned by this lane; the 8 lanes of a group cooperate.
-__device__ inline QuantOut quantize_eight(const float x[8]) {
-  float mn = x[0], mx = x[0];
-#pragma unroll
-  for (int i = 1; i < 8; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
-#pragma unroll
-  for (int o = 1; o < 8; o <<= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  }
-  __half hb = __float2half_rd(mn);
-  if (__half2float(hb) == 0.0f) hb = __ushort_as_half((unsigned short)0);   // -0 -> +0
-  const float bf = __half2float(hb);
-  const float r = __fsub_rn(mx, bf);
-  const __half hs = __float2half_ru(__fdiv_rn(r, 15.0f));
-  const float sf = __half2float(hs);
-  uint32_t w = 0;
-  if (sf != 0.0f) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float t = __fdiv_rn(__fsub_rn(x[i], bf), sf);
-      int c = __float2int_rn(t);
-      c = min(max(c, 0), 15);
-      w |= (uint32_t)c << (4 * i);
-    }
-  }
-  QuantOut o;
-  o.word = w;
-  o.sb = __halves2half2(hs, hb);
-  return o;
-}
-
-__device__ inline void load_eight_bf16(const void* base, size_t elem_index, float x[8]) {
-  const uint4 v = *reinterpret_cast<const uint4*>((const uint16_t*)base + elem_index);
-  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    x[2 * i] = __uint_as_float(u[i] << 16);
-    x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
-  }
-}
 
 struct UnitInfo { int agent, first, cnt, row0, block; };
 

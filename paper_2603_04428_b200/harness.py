@@ -78,6 +78,22 @@ class DeviceCache:
                                 float(scale), out, out_dtype, lse, ws, self.flags)
         return out, lse
 
+    def append_decode(self, layer, kv_lens, window, k_bits, v_bits, q_bits, scale, out_dtype=B.OUT_F32, bt=None):
+        """One new token per agent appended at position kv_len - 1 and attended, in one launch."""
+        q = bf16_dev(q_bits) if isinstance(q_bits, np.ndarray) else q_bits
+        k = bf16_dev(k_bits) if isinstance(k_bits, np.ndarray) else k_bits
+        v = bf16_dev(v_bits) if isinstance(v_bits, np.ndarray) else v_bits
+        A = q.shape[0]
+        lens_d = dev(np.asarray(kv_lens, dtype=np.int32)) if not torch.is_tensor(kv_lens) else kv_lens
+        out = torch.empty((A, self.spec.n_q_heads, self.spec.d_v), device="cuda",
+                          dtype=torch.float32 if out_dtype == B.OUT_F32 else torch.bfloat16)
+        lse = torch.empty((A, self.spec.n_q_heads), dtype=torch.float32, device="cuda")
+        b = bt or self.bt
+        ws = self.workspace(A, b.max_blocks * 256)
+        B.q4kv_append_decode_attention(self.spec, self.pool, self.n_blocks, layer, b, lens_d, 0, window, k, v, q,
+                                       float(scale), out, out_dtype, lse, ws, self.flags)
+        return out, lse
+
     def prefill(self, layer, kv_lens, q_offs, window, q_bits, scale, out_dtype=B.OUT_F32, want_lse=True, bt=None,
                 max_kv_len=0):
         q = bf16_dev(q_bits) if isinstance(q_bits, np.ndarray) else q_bits

@@ -364,6 +364,41 @@ def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
         p.dc.flags.zero_()
 
 
+@pytest.mark.parametrize("name,lens,window", [
+    ("gqa128", [1000, 700, 0, 255, 256, 257, 31, 32, 33], 0),      # block and chunk edges, an agent without a token
+    ("gqa128", [1000, 700, 64], 300),
+    ("gqa256", [1500, 41, 2049], 1024),
+])
+def test_update_and_fetch_in_one_launch(H, name, lens, window):
+    """q4kv_append_decode_attention: same pool bytes as quantize-append, same attention as decode, step after step."""
+    from paper_2603_04428_b200 import binding as B
+    spec_args = SPECS[name]
+    steps = 3
+    p = Pair(H, spec_args, lens, seed=39, extra_tokens=steps).fill()
+    s = p.ospec
+    A = len(lens)
+    cur = list(lens)
+    scale = 1.0 / math.sqrt(s.d_qk)
+    for step in range(steps):
+        kb = synth.kv_bf16(39, 500 + step, A, s.n_kv_heads, s.d_qk)
+        vb = synth.kv_bf16(39, 600 + step, A, s.n_kv_heads, s.d_v)
+        q = p.q(70 + step, A)
+        live = [a for a in range(A) if lens[a] > 0]          # an agent that starts empty stays out of the step
+        new_lens = [n + 1 if lens[a] > 0 else 0 for a, n in enumerate(cur)]
+        for l in range(s.n_layers):
+            # oracle: append row a at position cur[a] for the live agents, then attend
+            offs = np.concatenate([[0], np.cumsum([1 if a in live else 0 for a in range(A)])]).astype(np.int32)
+            O.quantize_append(p.opool, l, p.tabs, cur, offs, f32(kb[live]), f32(vb[live]))
+            ref, lse_ref = O.decode_attention(p.opool, l, p.tabs, new_lens, window, f32(q), scale)
+            out, lse = p.dc.append_decode(l, new_lens, window, kb, vb, q, scale)
+            assert_attention_close(out.cpu().numpy(), ref, f"{name} step {step} layer {l}")
+            assert_lse_close(lse.cpu().numpy(), lse_ref, name)
+        cur = new_lens
+    p.lens = cur
+    p.check_packed_equal()                                     # the pool holds exactly what quantize-append writes
+    assert p.dc.read_flags() == 0
+
+
 # ---- prefill attention --------------------------------------------------------------------------
 @pytest.mark.parametrize("name,prefix,chunk,window", [
     ("gqa64", [300, 70], 40, 0),
