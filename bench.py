@@ -179,6 +179,7 @@ class DeviceWorkload:
         torch.cuda.synchronize()
         assert dc.read_flags() == 0
         self.launches_per_step = 0
+        self.fused = fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS")
 
     # one layer of the step ----------------------------------------------------------------------
     def append_layer(self, l):
@@ -198,10 +199,20 @@ class DeviceWorkload:
                                      w.n_agents * w.new_tokens, w.new_tokens, self.max_kv, w.layer_window(l),
                                      self.q[l], w.softmax_scale, self.out[l], B.OUT_F32, None, self.ws, dc.flags)
 
+    def fused_layer(self, l):
+        """Update-and-fetch in one launch: the new token is quantized by the warp that attends its chunk."""
+        w, dc, B = self.w, self.dc, self.B
+        B.q4kv_append_decode_attention(dc.spec, dc.pool, dc.n_blocks, l, dc.bt, self.lens1, self.max_kv,
+                                       w.layer_window(l), self.k_new[l], self.v_new[l], self.q[l], w.softmax_scale,
+                                       self.out[l], B.OUT_F32, None, self.ws, dc.flags)
+
     def step(self):
         for l in range(self.w.n_layers):
-            self.append_layer(l)
-            self.attend_layer(l)
+            if self.fused:
+                self.fused_layer(l)
+            else:
+                self.append_layer(l)
+                self.attend_layer(l)
 
 
 def time_region(torch, fn, iters):
@@ -400,12 +411,13 @@ def main():
                 fn()
             return time_region(torch, fn, reps) / reps / L * 1e3
         reps = max(5, min(args.steps, 20))
-        att_ms_avg = per_launch_ms(dw.attend_layer, reps)
+        att_ms_avg = per_launch_ms(dw.fused_layer if dw.fused else dw.attend_layer, reps)
         app_ms_avg = per_launch_ms(dw.append_layer, reps)
         gl_ms_avg = None
         if w.window:
             gl_layers = [l for l in range(L) if w.layer_window(l) == 0]
-            gl_ms_avg = per_launch_ms(lambda i: dw.attend_layer(gl_layers[i % len(gl_layers)]), reps)
+            gl_fn = dw.fused_layer if dw.fused else dw.attend_layer
+            gl_ms_avg = per_launch_ms(lambda i: gl_fn(gl_layers[i % len(gl_layers)]), reps)
         clocks = sampler.stop()
         # ---- end to end through the C ABI with host buffers ----
         hq = dw.q.cpu().pin_memory()
@@ -439,7 +451,9 @@ def main():
     if w.kind == "decode":
         step_units = float(sum(decode_layer_bytes(w, l) for l in range(L)))
         launch_units = step_units / L
-        roof = {"bound": "hbm", "kernel": "q4kv_decode_attention (one call per layer, L calls replayed back to back)",
+        call = "q4kv_append_decode_attention" if fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS") \
+            else "q4kv_decode_attention"
+        roof = {"bound": "hbm", "kernel": call + " (one call per layer, L calls replayed back to back)",
                 "achieved": launch_units / att_avg_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": peak_kind}
         if w.window:
             # window and global layers differ by ~9x in bytes: quote the global layers, which dominate the step
@@ -468,6 +482,8 @@ def main():
                    "new_tokens_per_agent": w.new_tokens, "window": w.window,
                    "l2": "inputs larger than L2: every step streams the whole multi-layer cache",
                    "launch": "cuda graph replay of the L-layer step" if graph is not None else "eager",
+                   "update_and_fetch": "one launch per layer" if (fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"))
+                   else "quantize-append launch + attention launch per layer",
                    "multi_gpu": "replicas only"},
         "agent_steps_per_s": world * w.n_agents / t_step,
         "step_bytes" if w.kind == "decode" else "step_flops": step_units,
@@ -535,13 +551,19 @@ def run_pack(args):
     print(json.dumps(line))
 
 
-def dw_launches(w):
-    """Kernels of this library launched per step: per layer one quantize-append and one attention kernel; the
-    shape-agnostic decode path (MLA latent caches, more than 4 query heads per KV head) adds a split-merge kernel."""
+def fused_update_and_fetch(w):
+    """Decode shapes that q4kv_append_decode_attention covers (one launch per layer for append + attention)."""
     n_rep = w.n_q_heads // w.n_kv_heads
-    tensor_decode = (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
-    per_layer = 2 if (w.kind == "prefill" or tensor_decode) else 3
-    return per_layer * w.n_layers
+    return w.kind == "decode" and (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
+
+
+def dw_launches(w):
+    """Kernels of this library launched per step.  GQA decode: one update-and-fetch kernel per layer.  Prefill:
+    one quantize-append and one attention kernel per layer.  MLA-latent decode: quantize-append, the key-split
+    attention kernel and its merge kernel."""
+    if fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"):
+        return w.n_layers
+    return (2 if w.kind == "prefill" else 3) * w.n_layers
 
 
 if __name__ == "__main__":

@@ -451,6 +451,17 @@ __device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, c
   __syncwarp();                                          // the patched chunk is read by the same warp
 }
 
+// Ask for the new token's rows early (when the segment's query is staged), so that the warp that later owns the
+// chunk finds them in L2.
+template <int G>
+__device__ inline void prefetch_new_token(const uint16_t* k_new, const uint16_t* v_new, int Hkv, int a, int hk, int lane) {
+  constexpr int D = 64 * G, kLines = D * 2 / 128;        // 128-byte lines per row
+  if (lane < 2 * kLines) {
+    const uint16_t* p = (lane < kLines ? k_new : v_new) + ((size_t)a * Hkv + hk) * D + (lane % kLines) * 64;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+  }
+}
+
 // One 32-token chunk against this warp's query fragments.
 template <int G>
 __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
@@ -833,7 +844,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     while (wk.next(seg)) {
       const int k_end = seg.k0 + (seg.c1 - seg.c0);
       for (int k = seg.k0 + (lane - seg.k0 % kSlots + kSlots) % kSlots; k < k_end; k += kSlots) {
-        const int c = seg.c0 + (k - seg.k0);
+        const int c = seg.c1 - 1 - (k - seg.k0);     // a segment is walked from its last chunk to its first (see the consumers)
         const int round = k / kSlots;        // k % kSlots == lane
         if (!spin_until_ge(&sm.released[lane], round, &sm.abort_flag)) {
           raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
@@ -881,6 +892,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     for (int s = 0; s < kQBufs && w2.next(s2); ++s) {
       if (s % NW != warp) continue;
       stage_query<G>(sm.qfrag[s], sm.qsum[s], sm.kappa[s], P.q, y.Hq, n_rep, P.scale_log2, s2.a, s2.hk, lane);
+      if (P.k_new != nullptr && s2.c1 == ((s2.n + 31) >> 5)) prefetch_new_token<G>(P.k_new, P.v_new, y.Hkv, s2.a, s2.hk, lane);
       __threadfence_block();
       __syncwarp();
       if (lane == 0) *(volatile int*)&sm.q_tag[s] = s + 1;
@@ -971,6 +983,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
         const int prev = cur - kQBufs;
         if (!aborted && !spin_until_ge(&sm.epilogues[prev % kMBufs], prev / kMBufs + 1, &sm.abort_flag)) aborted = true;
         stage_query<G>(sm.qfrag[qb], sm.qsum[qb], sm.kappa[qb], P.q, y.Hq, n_rep, P.scale_log2, seg.a, seg.hk, lane);
+        if (P.k_new != nullptr && seg.c1 == ((seg.n + 31) >> 5)) prefetch_new_token<G>(P.k_new, P.v_new, y.Hkv, seg.a, seg.hk, lane);
         __threadfence_block();
         __syncwarp();
         if (lane == 0) *(volatile int*)&sm.q_tag[qb] = cur + 1;
@@ -995,7 +1008,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     if (sm.bad[slot]) {
       poisoned = true;
     } else {
-      const int c = seg.c0 + (k - seg.k0);
+      // A segment is walked from its last chunk to its first: the order does not matter to the online softmax, and
+      // the chunk that may carry the fused append (the agent's newest position) then comes first, where its extra
+      // latency overlaps the other warps' chunks instead of ending the launch.
+      const int c = seg.c1 - 1 - (k - seg.k0);
       if (P.k_new != nullptr && c == ((seg.n - 1) >> 5)) {
         // the chunk of the agent's newest position: its block id has passed the producer's check
         const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
