@@ -29,10 +29,18 @@ __device__ inline QuantOut quantize_eight(const float x[8]) {
   const float sf = __half2float(hs);
   uint32_t w = 0;
   if (sf != 0.0f) {
+    // code = clamp(rne(fl((x - b) / s))).  The eight IEEE divisions dominate this function, so the quotient is
+    // taken as t * (1/s) with one fused residual correction (within an ulp of the correctly rounded quotient,
+    // 1/s being correctly rounded), which rounds to the same integer unless the quotient sits within a few ulps
+    // of k + 1/2; only there is the division itself evaluated.
+    const float inv = __frcp_rn(sf);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float t = __fdiv_rn(__fsub_rn(x[i], bf), sf);
-      int c = __float2int_rn(t);
+      const float t = __fsub_rn(x[i], bf);
+      float q = __fmul_rn(t, inv);
+      q = __fmaf_rn(__fmaf_rn(-sf, q, t), inv, q);
+      if (fabsf(q - (floorf(q) + 0.5f)) < 1e-5f) q = __fdiv_rn(t, sf);
+      int c = __float2int_rn(q);
       c = min(max(c, 0), 15);
       w |= (uint32_t)c << (4 * i);
     }

@@ -179,6 +179,39 @@ def test_unpack_from_oracle_bytes_feeds_attention(H):
         assert_lse_close(lse.cpu().numpy(), lse_ref)
 
 
+class TiePair(Pair):
+    """Keys and values whose quotients (x - bias) / scale sit exactly on, or one bf16 step beside, the rounding
+    boundaries k + 1/2: min 0 and max 15 * 2^e per group, everything else (k + 1/2) * 2^e or its neighbours."""
+
+    def kv(self, layer, agent, n):
+        s = self.ospec
+        rs = np.random.default_rng(1000 * layer + agent)
+
+        def make(d):
+            e = rs.integers(-6, 3, size=(n, s.n_kv_heads, d // 64, 1)).astype(np.float32)
+            step = np.float32(2.0) ** e
+            k = rs.integers(0, 15, size=(n, s.n_kv_heads, d // 64, 64)).astype(np.float32) + np.float32(0.5)
+            x = k * step
+            bits = synth.f32_to_bf16_bits(x.astype(np.float32))
+            nudge = rs.integers(-1, 2, size=bits.shape).astype(np.int32)            # -1, 0, +1 bf16 ulp
+            bits = (bits.astype(np.int32) + nudge).astype(np.uint16)
+            x = f32(bits)
+            x[..., 0] = 0.0
+            x[..., 1] = (np.float32(15.0) * step)[..., 0]
+            return synth.f32_to_bf16_bits(x.reshape(n, s.n_kv_heads, d).astype(np.float32))
+
+        return make(s.d_qk), (None if s.v_aliases_k else make(s.d_v))
+
+
+def test_quantizer_is_bit_exact_on_rounding_boundaries(H):
+    """Every code decided at, or a hair beside, a tie: the reciprocal-and-correct quotient must fall back to the
+    division exactly where it matters."""
+    p = TiePair(H, SPECS["gqa128"], [300, 70], seed=23).fill(chunks=[3, 64, 300])
+    p.check_packed_equal()
+    p2 = TiePair(H, SPECS["mla"], [130], seed=24).fill()
+    p2.check_packed_equal()
+
+
 # ---- decode attention ---------------------------------------------------------------------------
 def test_config1_tiny_decode_append_and_roundtrip(H):
     w = synth.workload(0)
