@@ -6,8 +6,8 @@
 // Every key serves all 16 heads and is both key and value, so the cache bytes are expanded once
 // per 64-key block into a binary16 tile that the tensor cores read twice:
 //   * Work is split along the keys: CTA (split, agent) walks its share of the agent's keys 64 at a
-//     time (two 32-token chunks = one bulk copy of 20736 bytes, issued by a loader warp into a
-//     two-slot ring), leaves an (acc, m, l) record per head, and a second kernel combines the
+//     time (two 32-token chunks = one bulk copy of 20736 bytes into a two-slot ring, issued two
+//     blocks ahead by one thread), leaves an (acc, m, l) record per head, and a second kernel combines the
 //     records of an agent.
 //   * The eight compute warps first turn the raw block into the tile K^ [64 keys][576 dims] in
 //     shared memory (x^ = c * s + b, one binary16 fma per pair of codes, rounded once), stored as
@@ -25,9 +25,10 @@
 //     scores exceed it by more than 2^8 triggers an exact per-head maximum (shuffles + shared
 //     memory) and a rescale of the register accumulators; otherwise a block costs four
 //     exponentials per thread.  Row sums stay per-thread until the end.
-// Three CTA-wide named barriers per block (tile ready, growth agreed, probabilities ready); the
-// loader hand-off is mbarriers with bounded waits (Q4KV_FLAG_INTERNAL when one runs out; the 256
-// compute threads then leave together).
+// Three CTA-wide named barriers per block (tile ready, growth agreed, probabilities ready); the raw
+// blocks arrive on mbarriers with bounded waits (Q4KV_FLAG_INTERNAL when one runs out; the 256
+// threads then leave together).  Eight warps, not nine: with a ninth the register allocation drops
+// to 168 per thread, and the queries' fragments alone take 144.
 #include "q4kv_layout.cuh"
 #include "tcgen05.cuh"
 
@@ -38,8 +39,8 @@ namespace {
 using namespace tc;   // mbarrier and bulk-copy wrappers
 
 constexpr int kD = 576, kDv = 512, kHeads = 16;
-constexpr int kComputeWarps = 8, kLoadWarp = kComputeWarps;
-constexpr int kThreads = (kLoadWarp + 1) * 32;           // 288
+constexpr int kComputeWarps = 8;
+constexpr int kThreads = kComputeWarps * 32;            // 256
 constexpr int kChunkBytes = 32 * (kD / 2 + 4 * (kD / 64));   // 10368: [Kc 9216 | Ksb 1152]
 constexpr int kRawBytes = 2 * kChunkBytes;               // one 64-key block
 constexpr int kTileBytes = 64 * kD * 2;                  // 73728
@@ -71,7 +72,7 @@ struct MlaSmem {
   float kappa[kHeads];                                   // score in log2 units = S * kappa[head]
   float wmax[kComputeWarps][kHeads];
   float wsum[kComputeWarps][kHeads];
-  alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots];
+  alignas(8) uint64_t raw_full[kRawSlots];
   int grow[3], stop[3];
   int bad[kRawSlots];
   int abort_flag, poisoned;
@@ -150,7 +151,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   }
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); mbar_init(&sm.raw_free[s], kComputeWarps); sm.bad[s] = 0; }
+    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); sm.bad[s] = 0; }
     for (int i = 0; i < 3; ++i) { sm.grow[i] = 0; sm.stop[i] = 0; }
     sm.abort_flag = 0; sm.poisoned = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -160,37 +161,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the new token was appended by the preceding kernel
   volatile int* abort_flag = &sm.abort_flag;
 
-  if (warp == kLoadWarp) {
-    // =============================== raw block loader ==========================================
-    if (lane == 0) {
-      int issued = 0;
-      for (int j = 0; j < n_iter; ++j) {
-        const int r = j % kRawSlots;
-        if (j >= kRawSlots && !mbar_wait(&sm.raw_free[r], (uint32_t)(j / kRawSlots - 1), abort_flag)) break;
-        const int c = 2 * (b0 + j);
-        const int blk = P.tables[(size_t)a * P.max_blocks + (c >> 3)];
-        if (blk < 0 || blk >= P.n_blocks) {
-          sm.bad[r] = 1;
-          sm.poisoned = 1;
-          raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
-          mbar_arrive(&sm.raw_full[r]);
-        } else {
-          sm.bad[r] = 0;
-          mbar_arrive_expect_tx(&sm.raw_full[r], kRawBytes);
-          bulk_load(sm.raw[r], head_block(P.pool, y, P.layer, blk, 0) + (size_t)(c & 7) * kChunkBytes, kRawBytes,
-                    &sm.raw_full[r]);
-        }
-        issued = j + 1;
-      }
-      if (*abort_flag) {                                 // giving up: let this thread's copies land first
-        for (int j = max(0, issued - kRawSlots); j < issued; ++j) {
-          const int r = j % kRawSlots;
-          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&sm.raw_full[r], (uint32_t)(j / kRawSlots) & 1u); ++i) {}
-        }
-        raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
-      }
+  // Raw 64-key blocks: one bulk copy each into a two-slot ring, issued by thread 0 -- blocks 0 and 1 here, block
+  // j + 2 once every warp has left block j's raw bytes (the barrier after the dequantize step).
+  auto issue_block = [&](int j) {
+    const int r = j % kRawSlots;
+    const int c = 2 * (b0 + j);
+    const int blk = P.tables[(size_t)a * P.max_blocks + (c >> 3)];
+    if (blk < 0 || blk >= P.n_blocks) {
+      sm.bad[r] = 1;
+      sm.poisoned = 1;
+      raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
+      mbar_arrive(&sm.raw_full[r]);
+    } else {
+      sm.bad[r] = 0;
+      mbar_arrive_expect_tx(&sm.raw_full[r], kRawBytes);
+      bulk_load(sm.raw[r], head_block(P.pool, y, P.layer, blk, 0) + (size_t)(c & 7) * kChunkBytes, kRawBytes, &sm.raw_full[r]);
     }
-    return;
+  };
+  int issued = 0;                                        // thread 0: blocks whose copy has been issued
+  if (threadIdx.x == 0) {
+    issue_block(0);
+    if (n_iter > 1) issue_block(1);
+    issued = min(n_iter, kRawSlots);
   }
 
   // =============================== compute warps ================================================
@@ -253,11 +245,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   const uint32_t kq_lane = lr * 16 + warp * kGroupStride + lm * 128;        // scores: key octet = warp; + 512 per two k-steps
   const uint32_t kv_lane = lr * 16 + (lm & 1) * kGroupStride + (8 * warp + (lm >> 1)) * 128;   // values: + 2 ks octets, + 256 per dim-core pair
 
-  // The queries never change: the A fragments of every other k-step live in registers for the whole launch (all of
-  // them would not fit), the rest is re-read from shared memory per block.
-  uint32_t qa[kD / 32][4];
+  // The queries never change: their A fragments (36 k-steps x 4 registers) live in registers for the whole launch.
+  uint32_t qa[kD / 16][4];
 #pragma unroll
-  for (int kk = 0; kk < kD / 32; ++kk) ldmatrix_x4(qa[kk], q_lane + (2 * kk) * 256);
+  for (int ks = 0; ks < kD / 16; ++ks) ldmatrix_x4(qa[ks], q_lane + ks * 256);
   float kap[2], m_ref[2], l_part[2];                     // heads g and g + 8
   kap[0] = sm.kappa[g]; kap[1] = sm.kappa[g + 8];
   m_ref[0] = -INFINITY; m_ref[1] = -INFINITY; l_part[0] = 0.f; l_part[1] = 0.f;
@@ -296,11 +287,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
         *reinterpret_cast<uint4*>(dst + 68 * 128) = dequant8(kw.y, s8, c8);
       }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.raw_free[r]);         // this warp is done with the raw slot
     if (tq == 0) sm.stop[j % 3] = *abort_flag;           // sampled by one thread: all 256 leave in the same block
-    compute_barrier();                                   // the tile is complete
+    compute_barrier();                                   // the tile is complete, and nobody reads the raw slot any more
     if (sm.stop[j % 3]) { stopped = true; break; }
+    if (tq == 0 && j + kRawSlots < n_iter) { issue_block(j + kRawSlots); issued = j + kRawSlots + 1; }
 
     // ---- scores of this warp's eight keys: S[16 heads][8 keys], 36 k-steps ----
     float sc[4];
@@ -312,11 +302,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
       const uint32_t kb = smem_u32(sm.khat[s]) + kq_lane;
 #pragma unroll
       for (int kk = 0; kk < kD / 32; ++kk) {
-        uint32_t bq[4], a1[4];
+        uint32_t bq[4];
         ldmatrix_x4(bq, kb + kk * 512);
-        ldmatrix_x4(a1, q_lane + (2 * kk + 1) * 256);
-        mma_f16(acc[(2 * kk) & 3], qa[kk], bq[0], bq[1]);
-        mma_f16(acc[(2 * kk + 1) & 3], a1, bq[2], bq[3]);
+        mma_f16(acc[(2 * kk) & 3], qa[2 * kk], bq[0], bq[1]);
+        mma_f16(acc[(2 * kk + 1) & 3], qa[2 * kk + 1], bq[2], bq[3]);
       }
 #pragma unroll
       for (int e = 0; e < 4; ++e) sc[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
@@ -387,7 +376,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   }
   compute_barrier();
   const bool spoiled = stopped || sm.poisoned != 0;
-  if (stopped && tq == 0) raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
+  if (stopped && tq == 0) {
+    // giving up: let the copies that may still be in flight land before shared memory is released
+    for (int jj = max(0, issued - kRawSlots); jj < issued; ++jj)
+      for (uint32_t i = 0; i < 64 && !mbar_try_wait(&sm.raw_full[jj % kRawSlots], (uint32_t)(jj / kRawSlots) & 1u); ++i) {}
+    raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
+  }
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
     // dim core 8 warp + c, slots 2 tid and 2 tid + 1 of its 16-byte row
