@@ -422,6 +422,21 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
   if (h >= Hq) return;
   const float* rec = records + ((size_t)a * n_splits * kHeads + h) * kRecStride;
   const size_t step = (size_t)kHeads * kRecStride;       // between the splits of one head
+  // The record loads of the first 4 * kPre splits do not wait for the weights: they are issued first and overlap the
+  // round trip of the (m, l) loads (an empty split's data is whatever an earlier call left there; it is dropped below).
+  constexpr int kPre = 10;
+  const int grp = tid >> 7, d = 4 * (tid & 127);         // 128 threads x 4 consecutive dims per group
+  float4 pre[kPre];
+#pragma unroll
+  for (int u = 0; u < kPre; ++u) {
+    const int sp = grp + 4 * u;
+    pre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (sp < n_splits) {
+      const float2 lo2 = *reinterpret_cast<const float2*>(rec + sp * step + d);       // records are 8-byte aligned
+      const float2 hi2 = *reinterpret_cast<const float2*>(rec + sp * step + d + 2);
+      pre[u] = make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
+    }
+  }
   float ms = -INFINITY, ls = 0.f;
   if (tid < n_splits) { ms = rec[tid * step + kDv]; ls = rec[tid * step + kDv + 1]; }
   float M = ms, bad = ls < 0.f ? 1.f : 0.f;
@@ -445,25 +460,23 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
     for (int w = 0; w < kMergeThreads / 32; ++w) t += s_red[w][0];
     s_ml[0] = M; s_ml[1] = bad > 0.f ? 0.f : t;          // a poisoned split zeroes the row
   }
-  const int grp = tid >> 7, d = 4 * (tid & 127);         // 128 threads x 4 consecutive dims per group
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = grp; s0 < n_splits; s0 += 16) {
-    float2 lo2[4], hi2[4];
-    float w4[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int sp = s0 + 4 * u;
-      w4[u] = sp < n_splits ? s_w[sp] : 0.f;
-      lo2[u] = make_float2(0.f, 0.f); hi2[u] = make_float2(0.f, 0.f);
-      if (w4[u] > 0.f) {                                 // an empty split's record holds no data
-        lo2[u] = *reinterpret_cast<const float2*>(rec + sp * step + d);       // records are 8-byte aligned
-        hi2[u] = *reinterpret_cast<const float2*>(rec + sp * step + d + 2);
-      }
+  for (int u = 0; u < kPre; ++u) {
+    const int sp = grp + 4 * u;
+    const float wu = sp < n_splits ? s_w[sp] : 0.f;
+    if (wu > 0.f) {                                      // an empty split's record holds no data
+      acc.x = fmaf(wu, pre[u].x, acc.x); acc.y = fmaf(wu, pre[u].y, acc.y);
+      acc.z = fmaf(wu, pre[u].z, acc.z); acc.w = fmaf(wu, pre[u].w, acc.w);
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      acc.x = fmaf(w4[u], lo2[u].x, acc.x); acc.y = fmaf(w4[u], lo2[u].y, acc.y);
-      acc.z = fmaf(w4[u], hi2[u].x, acc.z); acc.w = fmaf(w4[u], hi2[u].y, acc.w);
+  }
+  for (int sp = grp + 4 * kPre; sp < n_splits; sp += 4) {
+    const float wu = s_w[sp];
+    if (wu > 0.f) {
+      const float2 lo2 = *reinterpret_cast<const float2*>(rec + sp * step + d);
+      const float2 hi2 = *reinterpret_cast<const float2*>(rec + sp * step + d + 2);
+      acc.x = fmaf(wu, lo2.x, acc.x); acc.y = fmaf(wu, lo2.y, acc.y);
+      acc.z = fmaf(wu, hi2.x, acc.z); acc.w = fmaf(wu, hi2.y, acc.w);
     }
   }
   if (grp > 0) s_acc[grp - 1][tid & 127] = acc;
