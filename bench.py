@@ -285,10 +285,11 @@ def oracle_sample(w: synth.Workload, budget_s: float = 12.0):
     one()
     dt = time.perf_counter() - t0
     reps = 1
-    while (time.perf_counter() - t0) < budget_s and reps < 50:
+    while (time.perf_counter() - t0) < budget_s and reps < 1000:
         one()
         reps += 1
     dt = (time.perf_counter() - t0) / reps
+    desc += f"; {reps} repetitions, {dt * reps:.1f} s of CPU work"
     return dt, units, desc, threads
 
 
