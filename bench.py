@@ -215,6 +215,16 @@ class DeviceWorkload:
                 self.attend_layer(l)
 
 
+def slowest_rank(torch, dist, seconds, device):
+    """Replicas only: every rank times the same work on its own GPU; the job's time is the slowest rank's (element-wise
+    maximum over the ranks), and the job's throughput is world_size x units / that time."""
+    if dist is None:
+        return [float(x) for x in seconds]
+    tt = torch.tensor(seconds, device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return [float(x) for x in tt]
+
+
 def time_region(torch, fn, iters):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -442,10 +452,7 @@ def main():
         d2h = hout.numel() * 4
     assert dw.dc.read_flags() == 0, "device status flags set during the benchmark"
 
-    if dist is not None:
-        tt = torch.tensor([t_step, t_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_step, t_e2e = float(tt[0]), float(tt[1])
+    t_step, t_e2e = slowest_rank(torch, dist, [t_step, t_e2e], "cuda")
 
     hbm_peak, tf_burst, tf_sust, peak_kind = peaks()
     att_avg_s = att_ms_avg / 1e3
