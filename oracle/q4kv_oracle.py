@@ -18,7 +18,7 @@ What it follows (paper sections, not code):
   * Persisted per-block tensor schema -- Appendix A.
 
 The paper delegates the quantizer's exact arithmetic to a library, so the
-sequence below is this build's fixed reading (single binary32 operations in the
+sequence below is this library's fixed reading (single binary32 operations in the
 order written; bias rounded down, scale rounded up to binary16 so that the code
 range always covers the group's range).  Attention is the textbook definition
 in float64 over the dequantized values.
@@ -62,7 +62,7 @@ def _f16_round_up(x32: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------
-# quantizer (Section 3.2 format; arithmetic = this build's fixed reading)
+# quantizer (Section 3.2 format; arithmetic = this library's fixed reading)
 # ----------------------------------------------------------------------------
 def quantize_rows(x32: np.ndarray):
     """Quantize rows of binary32 values (already exact images of bf16 inputs).

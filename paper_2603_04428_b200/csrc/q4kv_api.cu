@@ -109,7 +109,7 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
-  // The tcgen05 kernels round each dequantized element once to binary16; the error that leaves in a score grows with
+  // The kernels that expand the cache into binary16 tiles round each dequantized element once; the error that leaves in a score grows with
   // the softmax scale and stays well inside the library's 2e-3 output bound up to 2 / sqrt(d_qk).  Sharper scales
   // take the kernels that multiply the codes exactly.
   const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
