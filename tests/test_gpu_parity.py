@@ -593,3 +593,80 @@ def test_host_side_rejections(H):
     with pytest.raises(B.Q4KVError) as e:
         B.q4kv_pack(p.dc.spec, p.dc.pool, p.n_blocks, p.dc.tables[0], 100, dst)
     assert e.value.code == B.EWORKSPACE
+
+
+# ---- the benchmark's own launches, at full size -------------------------------------------------
+class WorkloadPair(Pair):
+    """One layer of a benchmark configuration: its agents, lengths, head shapes and outlier channels."""
+
+    def __init__(self, H, w, extra_tokens):
+        super().__init__(H, (1, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k), list(w.lens), seed=w.seed,
+                         extra_tokens=extra_tokens)
+        self.w = w
+        self.ko = synth.outlier_channels(w.seed, 100, w.n_kv_heads, w.d_qk, w.outlier_frac) if w.outlier_frac else None
+        self.vo = synth.outlier_channels(w.seed, 200, w.n_kv_heads, w.d_v, w.outlier_frac) if w.outlier_frac else None
+
+    def kv(self, layer, agent, n):
+        w = self.w
+        k = synth.kv_bf16(w.seed, 10 * agent + 1, n, w.n_kv_heads, w.d_qk, outliers=self.ko)
+        v = None if w.v_aliases_k else synth.kv_bf16(w.seed, 10 * agent + 2, n, w.n_kv_heads, w.d_v, outliers=self.vo)
+        return k, v
+
+
+@pytest.mark.parametrize("index", [1, 2, 3])
+def test_full_size_decode_launches_match_the_oracle(H, index):
+    """Configurations 2, 3 and 4 exactly as bench.py launches them, one layer: every agent, every head, every
+    cached token (4096 x 5; ten ragged agents up to 32k tokens, window and global layer; 16384 x 4 MLA latents),
+    the step's new token appended by the library, then every output row against the fp64 oracle."""
+    w = synth.workload(index)
+    p = WorkloadPair(H, w, extra_tokens=1).fill(chunks=[8192] * 4)
+    s = p.ospec
+    A = w.n_agents
+    kb = synth.kv_bf16(w.seed, 501, A, w.n_kv_heads, w.d_qk)
+    vb = None if w.v_aliases_k else synth.kv_bf16(w.seed, 502, A, w.n_kv_heads, w.d_v)
+    q = synth.normal_bf16(w.seed, 7, (A, w.n_q_heads, w.d_qk))
+    lens1 = [n + 1 for n in w.lens]
+    offs = np.arange(A + 1, dtype=np.int32)
+    O.quantize_append(p.opool, 0, p.tabs, w.lens, offs, f32(kb), None if vb is None else f32(vb))
+    windows = sorted({w.layer_window(l) for l in range(w.n_layers)})          # window layers and global layers
+    fused = (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and w.n_q_heads // w.n_kv_heads <= 4
+    if not fused:
+        p.dc.append(0, w.lens, offs, kb, vb)
+    for n_call, win in enumerate(windows):
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens1, win, f32(q), w.softmax_scale)
+        if fused:
+            out, lse = p.dc.append_decode(0, lens1, win, kb, vb, q, w.softmax_scale)   # idempotent: same token, same slot
+        else:
+            out, lse = p.dc.decode(0, lens1, win, q, w.softmax_scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"{w.name} window {win}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref, w.name)
+    p.lens = lens1
+    p.check_packed_equal()
+    assert p.dc.read_flags() == 0
+
+
+def test_full_size_prefill_launch_matches_the_oracle_on_sampled_rows(H):
+    """Configuration 5 as bench.py launches it, one layer: eight agents, 8192 cached + 1024 new tokens each.  The
+    library computes all 8192 x 32 output rows; the oracle checks 24 query rows per agent (all heads), spread over the
+    phase and including its first and last token, for two of the agents, and the appended cache bytes of all."""
+    w = synth.workload(4)
+    p = WorkloadPair(H, w, extra_tokens=w.new_tokens).fill(chunks=[8192])
+    A, T = w.n_agents, w.new_tokens
+    kb = synth.kv_bf16(w.seed, 501, A * T, w.n_kv_heads, w.d_qk)
+    vb = synth.kv_bf16(w.seed, 502, A * T, w.n_kv_heads, w.d_v)
+    q = synth.normal_bf16(w.seed, 7, (A * T, w.n_q_heads, w.d_qk))
+    offs = (np.arange(A + 1) * T).astype(np.int32)
+    O.quantize_append(p.opool, 0, p.tabs, w.lens, offs, f32(kb), f32(vb))
+    p.dc.append(0, w.lens, offs, kb, vb)
+    lens1 = [n + T for n in w.lens]
+    out, lse = p.dc.prefill(0, lens1, offs, 0, q, w.softmax_scale)
+    out = out.cpu().numpy()
+    local = sorted(set([0, 1, 31, 32, 63, 64, T - 1] + list(range(17, T, 61))))[:24]
+    rows = [a * T + i for a in (0, A - 1) for i in local]
+    ref, lse_ref = O.prefill_attention(p.opool, 0, p.tabs, lens1, offs, 0, f32(q), w.softmax_scale, rows=rows)
+    assert_attention_close(out[rows], ref[rows], w.name)
+    assert_lse_close(lse.cpu().numpy()[rows], lse_ref[rows], w.name)
+    assert np.all(np.isfinite(out))
+    p.lens = lens1
+    p.check_packed_equal()
+    assert p.dc.read_flags() == 0
