@@ -190,7 +190,15 @@ int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_
  *                  (and j > position - window when window > 0)
  *   total_q, max_q_len, max_kv_len   host copies / upper bounds (size the grid)
  *   q bf16 [total_q][n_q_heads][d_qk];  out [total_q][n_q_heads][d_v];  lse optional
- *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, total_q) bytes */
+ *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, total_q) bytes
+ * Accuracy: outputs are within 2e-3 (absolute) of the attention over the exactly dequantized
+ * values.  For d_qk = d_v = 128 with 1, 2 or 4 query heads per KV head and softmax_scale at most
+ * 2/sqrt(d_qk) the dequantized keys and values are rounded once to binary16 (11 significant bits)
+ * on their way to the tensor cores; sharper scales, and every other shape, use kernels that
+ * multiply the 4-bit codes exactly.  Setting Q4KV_PREFILL_PATH=mma in the environment selects the
+ * exact kernel for d = 128 as well.  The same rule (scale at most 2/sqrt(d_qk)) selects the
+ * binary16-tile kernel of q4kv_decode_attention for the MLA-latent shape (d_qk 576, d_v 512
+ * aliasing K, one KV head, at most 16 query heads). */
 int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                            const q4kv_batch* batch, const int32_t* kv_lens, const int32_t* q_offs,
                            int32_t total_q, int32_t max_q_len, int32_t max_kv_len,
