@@ -26,6 +26,14 @@
  *   - Data pointers must be 16-byte aligned.
  *   - Calls on different streams are safe together when their outputs and
  *     workspaces do not overlap and none writes pool blocks another reads.
+ *   - The kernels are launched with programmatic stream serialization: a
+ *     kernel's prologue overlaps the tail of the preceding kernel of the
+ *     stream, and it reads the lengths (kv_lens, pos, offsets) and block tables
+ *     there.  The pool, q, new rows, outputs and workspace are touched only
+ *     after the preceding kernels have completed.  Lengths and block tables
+ *     must therefore not be written by a preceding kernel that itself signals
+ *     its dependents early; an ordinary kernel, a copy or a memset is fine.
+ *     Setting Q4KV_NO_PDL in the environment turns the overlap off.
  *
  * Q4 format (Section 3.2): groups of 64 consecutive head-dim elements; per
  * group one binary16 scale and one binary16 bias; 4-bit codes, value =

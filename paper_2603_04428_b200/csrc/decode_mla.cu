@@ -158,6 +158,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
     fence_async_smem();
   }
   __syncthreads();
+  if (threadIdx.x < 2 && threadIdx.x < n_iter)           // the first two block-table entries, fetched towards the SM meanwhile
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(P.tables + (size_t)a * P.max_blocks + ((2 * (b0 + (int)threadIdx.x)) >> 3)) : "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the new token was appended by the preceding kernel
   volatile int* abort_flag = &sm.abort_flag;
 

@@ -840,6 +840,19 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     // once the slot's previous chunk has been consumed, so the copies of all slots are issued in parallel.
     static_assert(kSlots <= 32, "one producer lane per ring slot");
     if (lane >= kSlots) return;
+    {
+      // the block-table entry of this lane's first chunk is fetched towards the SM while the preceding kernel drains
+      // (the tables, like the lengths, are inputs that no kernel writes)
+      Walker w2 = wk;
+      Segment s2;
+      while (w2.next(s2)) {
+        const int k = s2.k0 + (lane - s2.k0 % kSlots + kSlots) % kSlots;
+        if (k >= s2.k0 + (s2.c1 - s2.c0)) continue;
+        const int c = s2.c1 - 1 - (k - s2.k0);
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(P.tables + (size_t)s2.a * P.max_blocks + (c >> 3)) : "memory");
+        break;
+      }
+    }
     grid_dependency_wait();                 // the pool may still be being written by the preceding kernel
     while (wk.next(seg)) {
       const int k_end = seg.k0 + (seg.c1 - seg.c0);

@@ -77,16 +77,16 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
                        const void* __restrict__ v_new, int32_t* flags) {
   extern __shared__ uint8_t vcodes_all[];   // [M][8][Dv]
   __shared__ UnitInfo s_unit[M];
-  // let the next kernel of the stream start its prologue; wait for the preceding ones before touching the pool
+  // let the next kernel of the stream start its prologue; the unit is found from the lengths and block tables (inputs
+  // that no kernel writes) while the preceding kernels drain, and the wait comes before the new rows and the pool
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-
   if (threadIdx.x < 32) {
     for (int r = 0; r < M; ++r)
       find_unit(blockIdx.x * M + r, n_agents, max_blocks, n_blocks, tables, pos, new_offs, flags,
                 blockIdx.x == 0 && blockIdx.y == 0 && r == 0, &s_unit[r]);
   }
   __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int hk = blockIdx.y;
   const int kw = y.D / 8, vw = y.alias ? 0 : y.Dv / 8;
   const int n_items = 8 * (kw + vw);
