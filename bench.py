@@ -203,7 +203,8 @@ class DeviceWorkload:
         """Update-and-fetch in one launch: the new token is quantized by the warp that attends its chunk."""
         w, dc, B = self.w, self.dc, self.B
         B.q4kv_append_decode_attention(dc.spec, dc.pool, dc.n_blocks, l, dc.bt, self.lens1, self.max_kv,
-                                       w.layer_window(l), self.k_new[l], self.v_new[l], self.q[l], w.softmax_scale,
+                                       w.layer_window(l), self.k_new[l], None if self.v_new is None else self.v_new[l],
+                                       self.q[l], w.softmax_scale,
                                        self.out[l], B.OUT_F32, None, self.ws, dc.flags)
 
     def step(self):
@@ -342,7 +343,7 @@ def peaks():
 
 # ncu DRAM traffic (read + write) per launch of the dominant kernel, from the committed profile summary
 # (profiles/decode_mma_llama31_8b.md, profiles/decode_mma_gemma3_12b_global_layer.md)
-NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23961856, "gemma3_12b_ragged_decode": 368124672}
+NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23963136, "gemma3_12b_ragged_decode": 367183360}
 
 
 def main():
@@ -490,7 +491,7 @@ def main():
                    "new_tokens_per_agent": w.new_tokens, "window": w.window,
                    "l2": "inputs larger than L2: every step streams the whole multi-layer cache",
                    "launch": "cuda graph replay of the L-layer step" if graph is not None else "eager",
-                   "update_and_fetch": "one launch per layer" if (fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"))
+                   "update_and_fetch": "one call per layer" if (fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"))
                    else "quantize-append launch + attention launch per layer",
                    "multi_gpu": "replicas only"},
         "agent_steps_per_s": world * w.n_agents / t_step,
@@ -561,17 +562,22 @@ def run_pack(args):
 
 def fused_update_and_fetch(w):
     """Decode shapes that q4kv_append_decode_attention covers (one launch per layer for append + attention)."""
+    if w.kind != "decode":
+        return False
+    if w.v_aliases_k:      # the MLA-latent cache (at the usual softmax scales)
+        return (w.d_qk, w.d_v, w.n_kv_heads) == (576, 512, 1) and w.n_q_heads <= 16 and w.softmax_scale ** 2 * w.d_qk <= 4
     n_rep = w.n_q_heads // w.n_kv_heads
-    return w.kind == "decode" and (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
+    return w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
 
 
 def dw_launches(w):
-    """Kernels of this library launched per step.  GQA decode: one update-and-fetch kernel per layer.  Prefill:
-    one quantize-append and one attention kernel per layer.  MLA-latent decode: quantize-append, the key-split
-    attention kernel and its merge kernel."""
+    """Kernels of this library launched per step.  GQA decode: one update-and-fetch kernel per layer.  MLA-latent
+    decode: the key-split update-and-fetch kernel and its merge kernel.  Prefill: one quantize-append and one
+    attention kernel per layer.  As two calls, decode launches the quantize-append kernel as well."""
+    mla = w.kind == "decode" and w.v_aliases_k
     if fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"):
-        return w.n_layers
-    return (2 if w.kind == "prefill" else 3) * w.n_layers
+        return (2 if mla else 1) * w.n_layers
+    return (3 if mla else 2) * w.n_layers
 
 
 if __name__ == "__main__":

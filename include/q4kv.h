@@ -154,9 +154,12 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
  *   kv_lens  [A]  lengths INCLUDING the new token (it sits at position kv_len - 1); kv_len == 0:
  *                 nothing is appended for that agent
  *   k_new    bf16 [A][n_kv_heads][d_qk], v_new bf16 [A][n_kv_heads][d_v]: row a is agent a's token
- * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256}, at
- * most four query heads per KV head, V not aliasing K; anything else returns Q4KV_EUNSUPPORTED
- * and the caller makes the two calls.  Two agents must not share the block that is written. */
+ *                 (v_new is ignored, and may be NULL, when V aliases K)
+ * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256} with at
+ * most four query heads per KV head and V not aliasing K; and the MLA-latent cache (V aliasing K,
+ * d_qk 576, d_v 512, one KV head, at most 16 query heads) with softmax_scale^2 * d_qk <= 4.
+ * Anything else returns Q4KV_EUNSUPPORTED and the caller makes the two calls.  Two agents must
+ * not share the block that is written. */
 int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
                                  const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
                                  int32_t window, const void* k_new, const void* v_new,

@@ -30,6 +30,7 @@
 // threads then leave together).  Eight warps, not nine: with a ninth the register allocation drops
 // to 168 per thread, and the queries' fragments alone take 144.
 #include "q4kv_layout.cuh"
+#include "quantize_core.cuh"
 #include "tcgen05.cuh"
 
 namespace q4kv {
@@ -58,6 +59,7 @@ struct MlaParams {
   const int32_t* kv_lens;
   int window;
   const uint16_t* q;          // bf16 [n_agents][Hq][576]
+  const uint16_t* k_new;      // bf16 [n_agents][576]: the row at position kv_len - 1, quantized and stored by this launch; or null
   float scale_log2;
   int n_splits, blocks_per_split;
   float* records;             // [n_agents][n_splits][16][kRecStride]
@@ -76,6 +78,7 @@ struct MlaSmem {
   int grow[3], stop[3];
   int bad[kRawSlots];
   int abort_flag, poisoned;
+  uint32_t new_words[kD / 8], new_sb[kD / 64];           // the new token's codes and (scale, bias) pairs (update-and-fetch)
 };
 
 // Eight codes of one packed word -> eight binary16 values c * s + b in the order (0,4) (1,5) (2,6) (3,7),
@@ -187,6 +190,29 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
     issued = min(n_iter, kRawSlots);
   }
 
+  // Update-and-fetch: the CTA whose share ends with the agent's last block quantizes the row of position n - 1
+  // (one warp, while the first copies are in flight) and, once that block has landed, patches it in shared memory
+  // and stores the same words to the pool.  No other CTA reads that block.
+  const bool has_new = P.k_new != nullptr && b0 + n_iter == b_hi;
+  if (has_new && warp == 0) {
+#pragma unroll 1
+    for (int base = 0; base < kD / 8; base += 32) {
+      const int w = base + lane;
+      float x[8];
+      if (w < kD / 8) {
+        load_eight_bf16(P.k_new, (size_t)a * kD + 8 * w, x);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = 0.f;
+      }
+      const QuantOut qo = quantize_eight(x);             // eight lanes per group of 64; 72 words = 9 whole groups
+      if (w < kD / 8) {
+        sm.new_words[w] = qo.word;
+        if ((w & 7) == 0) sm.new_sb[w >> 3] = *reinterpret_cast<const uint32_t*>(&qo.sb);
+      }
+    }
+  }
+
   // =============================== compute warps ================================================
   const int tq = threadIdx.x;                            // 0..255
   const int g = lane >> 2, tid = lane & 3;               // fragment coordinates
@@ -263,6 +289,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
     const int s = j % kStages, r = j % kRawSlots;
     // ---- raw block -> binary16 tile (every thread: one token of one chunk, 18 words) ----
     mbar_wait(&sm.raw_full[r], (uint32_t)(j / kRawSlots), abort_flag);     // a wait that runs out raises the give-up flag
+    if (has_new && j == n_iter - 1) {
+      // words 0..71 and the nine (scale, bias) pairs of position n - 1, one per thread
+      if (sm.bad[r] == 0 && tq < kD / 8 + kD / 64) {
+        const int tau_n = (n - 1) & 31, c = 2 * (b0 + j);
+        const uint32_t at = (uint32_t)(((n - 1) >> 5) & 1) * kChunkBytes +
+                            (tq < kD / 8 ? y.off_kc + 4u * k_word_offset(tau_n, tq, kD / 64)
+                                         : y.off_ksb + 4u * sb_offset(tau_n, tq - kD / 8, kD / 64));
+        const uint32_t val = tq < kD / 8 ? sm.new_words[tq] : sm.new_sb[tq - kD / 8];
+        *reinterpret_cast<uint32_t*>(sm.raw[r] + at) = val;
+        const int blk = P.tables[(size_t)a * P.max_blocks + (c >> 3)];      // checked when the copy was issued
+        // the caller of the update-and-fetch entry owns the pool for writing
+        uint8_t* dst = const_cast<uint8_t*>(head_block(P.pool, y, P.layer, blk, 0)) + (size_t)(c & 7) * kChunkBytes + at;
+        *reinterpret_cast<uint32_t*>(dst) = val;
+      }
+      compute_barrier();
+    }
     {
       const uint8_t* raw = sm.raw[r];
       const bool dead = sm.bad[r] != 0 || (b0 + j) * 64 + krow >= n;       // stale bytes past the end
@@ -531,7 +573,7 @@ size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len)
 
 cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale, void* out,
-                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st) {
+                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st, const void* k_new) {
   if (b.n_agents <= 0) return cudaSuccess;
   MlaPlan plan = plan_mla(b.n_agents, max_kv_len, window);
   const MlaPlan full = plan_mla(b.n_agents, max_kv_len, 0);
@@ -539,7 +581,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   MlaParams P;
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
-  P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.n_splits = plan.n_splits;
+  P.q = (const uint16_t*)q; P.k_new = (const uint16_t*)k_new; P.scale_log2 = scale * kLog2e; P.n_splits = plan.n_splits;
   P.blocks_per_split = plan.blocks_per_split; P.records = (float*)ws; P.flags = flags;
   static bool configured[64] = {};
   const size_t smem = sizeof(MlaSmem);

@@ -139,12 +139,22 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
   if (!pool || n_blocks <= 0 || layer < 0 || layer >= spec->n_layers || window < 0 || max_kv_len < 0) return Q4KV_EINVAL;
   if (out_dtype != Q4KV_OUT_F32 && out_dtype != Q4KV_OUT_BF16) return Q4KV_EINVAL;
   if (batch->n_agents == 0) return Q4KV_OK;
-  if (!kv_lens || !q || !out || !workspace || !k_new || !v_new) return Q4KV_EINVAL;
-  if (!aligned16(pool) || !aligned16(q) || !aligned16(out) || !aligned16(workspace) || !aligned16(k_new) || !aligned16(v_new))
+  const bool need_v = !spec->v_aliases_k;                  // an aliased cache stores no V rows
+  if (!kv_lens || !q || !out || !workspace || !k_new || (need_v && !v_new)) return Q4KV_EINVAL;
+  if (!aligned16(pool) || !aligned16(q) || !aligned16(out) || !aligned16(workspace) || !aligned16(k_new) ||
+      (need_v && !aligned16(v_new)))
     return Q4KV_EINVAL;
   const int cap = batch->max_blocks * kBlockTokens;
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
+  if (decode_mla_supported(y)) {
+    // the latent-cache kernel expands the keys into binary16 tiles: usual softmax scales only (see q4kv_decode_attention)
+    if (!(softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f)) return Q4KV_EUNSUPPORTED;
+    if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
+    const cudaError_t e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,
+                                            out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream, k_new);
+    return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
+  }
   if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks)) return Q4KV_EUNSUPPORTED;
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
   const cudaError_t e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,

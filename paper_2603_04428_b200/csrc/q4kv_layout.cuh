@@ -150,6 +150,7 @@ bool decode_mla_supported(const Layout& y);
 size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len);
 cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale, void* out,
-                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st);
+                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
+                              const void* k_new = nullptr);   // k_new: update-and-fetch (the pool is written)
 
 }  // namespace q4kv

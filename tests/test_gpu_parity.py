@@ -401,6 +401,8 @@ def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
     ("gqa128", [1000, 700, 0, 255, 256, 257, 31, 32, 33], 0),      # block and chunk edges, an agent without a token
     ("gqa128", [1000, 700, 64], 300),
     ("gqa256", [1500, 41, 2049], 1024),
+    ("mla", [1000, 700, 0, 63, 64, 65, 129, 31, 32, 33], 0),       # the latent cache: 64-key block and chunk edges
+    ("mla", [2500, 300, 4000], 200),
 ])
 def test_update_and_fetch_in_one_launch(H, name, lens, window):
     """q4kv_append_decode_attention: same pool bytes as quantize-append, same attention as decode, step after step."""
@@ -629,7 +631,8 @@ def test_full_size_decode_launches_match_the_oracle(H, index):
     offs = np.arange(A + 1, dtype=np.int32)
     O.quantize_append(p.opool, 0, p.tabs, w.lens, offs, f32(kb), None if vb is None else f32(vb))
     windows = sorted({w.layer_window(l) for l in range(w.n_layers)})          # window layers and global layers
-    fused = (not w.v_aliases_k) and w.d_qk == w.d_v and w.d_qk in (128, 256) and w.n_q_heads // w.n_kv_heads <= 4
+    import bench
+    fused = bench.fused_update_and_fetch(w)               # all three take the update-and-fetch call, as the benchmark does
     if not fused:
         p.dc.append(0, w.lens, offs, kb, vb)
     for n_call, win in enumerate(windows):
