@@ -42,18 +42,29 @@ def test_binding_lists_the_same_symbols_and_size_queries_match_the_paper():
 
 
 def test_update_and_fetch_refuses_shapes_it_does_not_cover_before_touching_the_device():
-    """q4kv_append_decode_attention is host-checked first: an MLA-latent spec (V aliases K) and a head dim outside
-    {128, 256} come back as Q4KV_EUNSUPPORTED without a launch (the pointers below are never dereferenced)."""
+    """q4kv_append_decode_attention is host-checked first: a head dim outside {128, 256}, and an MLA-latent spec with a
+    softmax scale too sharp for its binary16-tile kernel (0.1^2 x 576 > 4), come back as Q4KV_EUNSUPPORTED without a
+    launch (the pointers below are never dereferenced; every call here is one the host checks refuse)."""
     from paper_2603_04428_b200 import binding as B
     lib = B.lib()
     fake = ctypes.c_void_p(0x1000)                      # aligned, never read
     tabs = (ctypes.c_int32 * 4)(0, 1, 2, 3)
     bt = B.Batch(1, 4, ctypes.cast(tabs, ctypes.c_void_p))
+    sharp = 0.1
+    assert sharp * sharp * 576 > 4
     for spec in (B.Spec.make(1, 16, 1, 576, 512, True), B.Spec.make(1, 4, 4, 192, 128)):
         rc = lib.q4kv_append_decode_attention(ctypes.byref(spec), fake, 4, 0, ctypes.byref(bt), fake, 0, 0, fake, fake,
-                                              fake, 0.1, fake, B.OUT_F32, None, fake, 1 << 20, None, None)
+                                              fake, sharp, fake, B.OUT_F32, None, fake, 1 << 20, None, None)
         assert rc == B.EUNSUPPORTED
+    # an aliased cache stores no V rows: a missing v_new is not an error there (the sharp scale still refuses the call)
+    mla = B.Spec.make(1, 16, 1, 576, 512, True)
+    rc = lib.q4kv_append_decode_attention(ctypes.byref(mla), fake, 4, 0, ctypes.byref(bt), fake, 0, 0, fake, None,
+                                          fake, sharp, fake, B.OUT_F32, None, fake, 1 << 20, None, None)
+    assert rc == B.EUNSUPPORTED
     llama = B.Spec.make(1, 8, 2, 128, 128)
     rc = lib.q4kv_append_decode_attention(ctypes.byref(llama), fake, 4, 0, ctypes.byref(bt), fake, 0, 0, None, fake,
                                           fake, 0.1, fake, B.OUT_F32, None, fake, 1 << 20, None, None)
     assert rc == B.EINVAL                                # a missing k_new row pointer
+    rc = lib.q4kv_append_decode_attention(ctypes.byref(llama), fake, 4, 0, ctypes.byref(bt), fake, 0, 0, fake, None,
+                                          fake, 0.1, fake, B.OUT_F32, None, fake, 1 << 20, None, None)
+    assert rc == B.EINVAL                                # V is stored here: a missing v_new row pointer
