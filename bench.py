@@ -357,12 +357,23 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--op", default="step", choices=["step", "pack"],
                     help="step: the append + attention step of --workload; pack: q4kv_pack / q4kv_unpack / bulk append")
+    ap.add_argument("--agents", type=int, default=0,
+                    help="scaled variant of a uniform-length configuration: this many agents (named so in config.workload)")
+    ap.add_argument("--layers", type=int, default=0, help="scaled variant: this many layers")
     args = ap.parse_args()
     if args.op == "pack":
         run_pack(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
     w = synth.workload(args.workload)
+    if args.agents > 0 or args.layers > 0:
+        # not one of the five configurations any more: the name says so, and no stored counter applies to it
+        import dataclasses
+        if args.agents > 0 and len(set(w.lens)) != 1:
+            raise SystemExit("--agents scales configurations whose agents have one common length")
+        lens = [w.lens[0]] * args.agents if args.agents > 0 else w.lens
+        layers = args.layers if args.layers > 0 else w.n_layers
+        w = dataclasses.replace(w, lens=lens, n_layers=layers, name=f"{w.name}_scaled_{len(lens)}agents_{layers}layers")
     if args.impl == "reference":
         run_reference(args, w)
         return
