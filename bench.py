@@ -125,7 +125,7 @@ class DeviceWorkload:
     """All state of one workload resident on the GPU: the Q4 pool (filled by the library's own quantizer
     from seeded on-device N(0,1) bf16 values), block tables, per-layer q / new K,V, outputs."""
 
-    def __init__(self, w: synth.Workload, device_index: int):
+    def __init__(self, w: synth.Workload, device_index: int, two_calls: bool = False):
         import torch
         from paper_2603_04428_b200 import binding as B, harness as H
         self.torch, self.B, self.w = torch, B, w
@@ -178,8 +178,7 @@ class DeviceWorkload:
                                   B.q4kv_workspace_bytes(dc.spec, A, self.max_kv, nq)), dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
         assert dc.read_flags() == 0
-        self.launches_per_step = 0
-        self.fused = fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS")
+        self.fused = fused_update_and_fetch(w) and not two_calls
 
     # one layer of the step ----------------------------------------------------------------------
     def append_layer(self, l):
@@ -235,6 +234,23 @@ def time_region(torch, fn, iters):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / 1e3
+
+
+def timed_batches(torch, fn, k, min_total_s=0.5, max_batches=400):
+    """Batches of exactly k calls of fn, back to back on the current stream, an event between consecutive batches and
+    one synchronize at the end; enough batches that the timed region lasts at least min_total_s.  Returns the batch
+    times in seconds (their median is what the line reports)."""
+    t1 = time_region(torch, fn, k)                         # sizes the region (not reported)
+    n = int(min(max_batches, max(3, math.ceil(min_total_s / max(t1, 1e-9)))))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(n):
+        for _ in range(k):
+            fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return [ev[i].elapsed_time(ev[i + 1]) / 1e3 for i in range(n)]
 
 
 # ------------------------------------------------------------------------------------------------
@@ -300,7 +316,8 @@ def oracle_sample(w: synth.Workload, budget_s: float = 12.0):
         one()
         reps += 1
     dt = (time.perf_counter() - t0) / reps
-    desc += f"; {reps} repetitions, {dt * reps:.1f} s of CPU work"
+    desc += (f"; {reps} repetitions, {dt * reps:.1f} s of CPU work; the oracle's loops over agents and heads are "
+             "single-threaded Python, 'cores' is the size of the BLAS thread pool its matrix products may use")
     return dt, units, desc, threads
 
 
@@ -341,9 +358,144 @@ def peaks():
     return 6650.0, 1590.0, 1400.0, "fallback"
 
 
-# ncu DRAM traffic (read + write) per launch of the dominant kernel, from the committed profile summary
-# (profiles/decode_mma_llama31_8b.md, profiles/decode_mma_gemma3_12b_global_layer.md)
-NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23963136, "gemma3_12b_ragged_decode": 367183360}
+NOMINAL_BF16_TFLOPS = 2250.0
+
+# DRAM bytes (read + write) of one launch of each workload's dominant kernel, from one profiler capture of that
+# kernel; None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"llama31_8b_decode": None, "gemma3_12b_ragged_decode": None, "dsv2lite_mla_decode": None,
+                     "llama31_8b_chunked_prefill": None, "pack": None, "unpack": None, "append_8x1024": None}
+
+
+def measure(w, args, local, dist=None, full=True):
+    """One workload on this rank's GPU: the L-layer step as a CUDA graph, timed in batches of args.steps replays over a
+    region of at least half a second (median batch), the per-launch time of the attention kernel from a graph of the L
+    attention calls, clocks sampled meanwhile; with full=True also the end-to-end step through host buffers."""
+    import torch
+    dw = DeviceWorkload(w, local, two_calls=args.two_calls)
+    L = w.n_layers
+    use_graph = not args.no_graph
+    stream = torch.cuda.Stream()
+    res = {}
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            dw.step()
+        stream.synchronize()
+        graph = None
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                dw.step()
+        run = graph.replay if graph is not None else dw.step
+        for _ in range(args.warmup):
+            run()
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        torch.cuda.synchronize()
+        k = args.steps if full or time_region(torch, run, 1) * args.steps < args.min_seconds / 2 else 1
+        batches = timed_batches(torch, run, k, min_total_s=args.min_seconds)
+        t_step = float(np.median(batches)) / k
+
+        # per-launch durations: the L attention calls of a step (one per layer, each over its own layer's cache, so
+        # every launch streams from HBM) replayed back to back from a graph of their own; likewise the L append calls
+        def per_launch_s(layer_fn):
+            for l in range(L):
+                layer_fn(l)
+            stream.synchronize()
+            if use_graph:
+                g2 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g2, stream=stream):
+                    for l in range(L):
+                        layer_fn(l)
+                fn = g2.replay
+            else:
+                def fn():
+                    for l in range(L):
+                        layer_fn(l)
+            for _ in range(3):
+                fn()
+            return float(np.median(timed_batches(torch, fn, 1, min_total_s=args.min_seconds / 2))) / L
+        att_s = per_launch_s(dw.fused_layer if dw.fused else dw.attend_layer)
+        app_s = per_launch_s(dw.append_layer)
+        gl_s = None
+        if w.window:
+            gl_layers = [l for l in range(L) if w.layer_window(l) == 0]
+            gl_fn = dw.fused_layer if dw.fused else dw.attend_layer
+            gl_s = per_launch_s(lambda i: gl_fn(gl_layers[i % len(gl_layers)]))
+        clocks = sampler.stop()
+        res.update(t_step=t_step, k=k, n_batches=len(batches), region_s=float(np.sum(batches)), att_s=att_s, app_s=app_s,
+                   gl_s=gl_s, clocks=clocks, graph=graph is not None, fused=dw.fused)
+        if full:
+            # ---- end to end through the C ABI with host buffers ----
+            hq = dw.q.cpu().pin_memory()
+            hk = dw.k_new.cpu().pin_memory()
+            hv = None if dw.v_new is None else dw.v_new.cpu().pin_memory()
+            hout = torch.empty(dw.out.shape, dtype=dw.out.dtype).pin_memory()
+
+            def e2e_step():
+                dw.q.copy_(hq, non_blocking=True)
+                dw.k_new.copy_(hk, non_blocking=True)
+                if hv is not None:
+                    dw.v_new.copy_(hv, non_blocking=True)
+                run()
+                hout.copy_(dw.out, non_blocking=True)
+                stream.synchronize()
+            for _ in range(2):
+                e2e_step()
+            e2e_iters = max(3, min(args.steps, 10))
+            res["t_e2e"] = time_region(torch, e2e_step, e2e_iters) / e2e_iters
+            res["h2d"] = hq.numel() * 2 + hk.numel() * 2 + (0 if hv is None else hv.numel() * 2)
+            res["d2h"] = hout.numel() * 4
+    assert dw.dc.read_flags() == 0, "device status flags set during the benchmark"
+    del dw
+    torch.cuda.empty_cache()
+    return res
+
+
+def roofline_of(w, res):
+    hbm_peak, tf_burst, tf_sust, peak_kind = peaks()
+    L = w.n_layers
+    att_s = res["att_s"]
+    if w.kind == "decode":
+        step_units = float(sum(decode_layer_bytes(w, l) for l in range(L)))
+        launch_units = step_units / L
+        call = "q4kv_append_decode_attention" if res["fused"] else "q4kv_decode_attention"
+        roof = {"bound": "hbm", "kernel": call + " (one call per layer, L calls replayed back to back)",
+                "achieved": launch_units / att_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": peak_kind}
+        if w.window:
+            # window and global layers differ by ~9x in bytes: quote the global layers, which dominate the step
+            gl = [l for l in range(L) if w.layer_window(l) == 0]
+            att_s = res["gl_s"]
+            roof["achieved"] = float(np.mean([decode_layer_bytes(w, l) for l in gl])) / att_s / 1e9
+            roof["kernel"] += ", global layers only"
+        roof["frac"] = roof["achieved"] / roof["peak"]
+    else:
+        step_units = prefill_layer_flops(w) * L
+        launch_units = step_units / L
+        ach = launch_units / att_s / 1e12
+        roof = {"bound": "tensor", "kernel": "q4kv_prefill_attention (one call per layer)",
+                "achieved": ach, "peak": tf_sust, "unit": "TFLOP/s", "peak_kind": peak_kind + " sustained bf16",
+                "frac": ach / tf_sust, "frac_of_burst": ach / tf_burst, "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
+    roof["avg_launch_us"] = att_s * 1e6
+    return step_units, roof
+
+
+def config_of(w, res):
+    L = w.n_layers
+    return {"workload": workload_name(w), "layers": L, "agents": w.n_agents,
+            "kv_lens": w.lens if len(set(w.lens)) > 1 else w.lens[0],
+            "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "d_qk": w.d_qk, "d_v": w.d_v,
+            "new_tokens_per_agent": w.new_tokens, "window": w.window,
+            "l2": "inputs larger than L2: every step streams the whole multi-layer cache",
+            "launch": "cuda graph replay of the L-layer step" if res["graph"] else "eager",
+            "timing": f"median of {res['n_batches']} back-to-back batches of {res['k']} steps "
+                      f"({res['region_s']:.2f} s timed)",
+            "update_and_fetch": "one call per layer" if res["fused"]
+            else "quantize-append launch + attention launch per layer",
+            "multi_gpu": "replicas only"}
 
 
 def main():
@@ -351,10 +503,17 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", type=int, default=1, help="index into the five configurations (0-based); default 1")
+    ap.add_argument("--workload", type=int, default=None,
+                    help="index into the five configurations (0-based).  Default: configuration 1 as the headline, "
+                         "with the other configurations and the copy-like kernels under all_configs")
     ap.add_argument("--impl", default="q4kv", choices=["q4kv", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-all-configs", action="store_true", help="headline workload only")
+    ap.add_argument("--two-calls", action="store_true",
+                    help="decode step as a quantize-append launch plus an attention launch per layer instead of the "
+                         "one-launch update-and-fetch")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="least duration of each timed region")
     ap.add_argument("--op", default="step", choices=["step", "pack"],
                     help="step: the append + attention step of --workload; pack: q4kv_pack / q4kv_unpack / bulk append")
     ap.add_argument("--agents", type=int, default=0,
@@ -362,10 +521,11 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="scaled variant: this many layers")
     args = ap.parse_args()
     if args.op == "pack":
-        run_pack(args)
+        print(json.dumps(run_pack(args)))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
-    w = synth.workload(args.workload)
+    default_run = args.workload is None and args.agents == 0 and args.layers == 0
+    w = synth.workload(1 if args.workload is None else args.workload)
     if args.agents > 0 or args.layers > 0:
         # not one of the five configurations any more: the name says so, and no stored counter applies to it
         import dataclasses
@@ -386,134 +546,44 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dw = DeviceWorkload(w, local)
+    torch.cuda.set_device(local)
     metric, unit, div = metric_of(w)
-    L = w.n_layers
-
-    # ---- the step: eager or one CUDA graph replay ----
-    use_graph = not args.no_graph
-    stream = torch.cuda.Stream()
-    graph = None
-    with torch.cuda.stream(stream):
-        for _ in range(2):
-            dw.step()
-        stream.synchronize()
-        if use_graph:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                dw.step()
-        run = graph.replay if graph is not None else dw.step
-        for _ in range(args.warmup):
-            run()
-        stream.synchronize()
-        if dist is not None:
-            dist.barrier()
-        sampler = ClockSampler(local)
-        sampler.start()
-        torch.cuda.synchronize()
-        dt = time_region(torch, run, args.steps)
-        t_step = dt / args.steps
-        # ---- per-kernel launch durations: the L attention calls of a step (one per layer, each over its own
-        # layer's cache, so every launch streams from HBM) replayed back to back from a graph of their own, and
-        # likewise the L append calls.  Events bracket the replays on the launching stream.
-        def per_launch_ms(layer_fn, reps):
-            for l in range(L):
-                layer_fn(l)
-            stream.synchronize()
-            if use_graph:
-                g2 = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g2, stream=stream):
-                    for l in range(L):
-                        layer_fn(l)
-                fn = g2.replay
-            else:
-                def fn():
-                    for l in range(L):
-                        layer_fn(l)
-            for _ in range(3):
-                fn()
-            return time_region(torch, fn, reps) / reps / L * 1e3
-        reps = max(5, min(args.steps, 20))
-        att_ms_avg = per_launch_ms(dw.fused_layer if dw.fused else dw.attend_layer, reps)
-        app_ms_avg = per_launch_ms(dw.append_layer, reps)
-        gl_ms_avg = None
-        if w.window:
-            gl_layers = [l for l in range(L) if w.layer_window(l) == 0]
-            gl_fn = dw.fused_layer if dw.fused else dw.attend_layer
-            gl_ms_avg = per_launch_ms(lambda i: gl_fn(gl_layers[i % len(gl_layers)]), reps)
-        clocks = sampler.stop()
-        # ---- end to end through the C ABI with host buffers ----
-        hq = dw.q.cpu().pin_memory()
-        hk = dw.k_new.cpu().pin_memory()
-        hv = None if dw.v_new is None else dw.v_new.cpu().pin_memory()
-        hout = torch.empty(dw.out.shape, dtype=dw.out.dtype).pin_memory()
-
-        def e2e_step():
-            dw.q.copy_(hq, non_blocking=True)
-            dw.k_new.copy_(hk, non_blocking=True)
-            if hv is not None:
-                dw.v_new.copy_(hv, non_blocking=True)
-            run()
-            hout.copy_(dw.out, non_blocking=True)
-            stream.synchronize()
-        for _ in range(2):
-            e2e_step()
-        e2e_iters = max(3, min(args.steps, 10))
-        t_e2e = time_region(torch, e2e_step, e2e_iters) / e2e_iters
-        h2d = hq.numel() * 2 + hk.numel() * 2 + (0 if hv is None else hv.numel() * 2)
-        d2h = hout.numel() * 4
-    assert dw.dc.read_flags() == 0, "device status flags set during the benchmark"
-
-    t_step, t_e2e = slowest_rank(torch, dist, [t_step, t_e2e], "cuda")
-
-    hbm_peak, tf_burst, tf_sust, peak_kind = peaks()
-    att_avg_s = att_ms_avg / 1e3
-    if w.kind == "decode":
-        step_units = float(sum(decode_layer_bytes(w, l) for l in range(L)))
-        launch_units = step_units / L
-        call = "q4kv_append_decode_attention" if fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS") \
-            else "q4kv_decode_attention"
-        roof = {"bound": "hbm", "kernel": call + " (one call per layer, L calls replayed back to back)",
-                "achieved": launch_units / att_avg_s / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": peak_kind}
-        if w.window:
-            # window and global layers differ by ~9x in bytes: quote the global layers, which dominate the step
-            gl = [l for l in range(L) if w.layer_window(l) == 0]
-            att_avg_s = gl_ms_avg / 1e3
-            roof["achieved"] = float(np.mean([decode_layer_bytes(w, l) for l in gl])) / att_avg_s / 1e9
-            roof["kernel"] += ", global layers only"
-    else:
-        step_units = prefill_layer_flops(w) * L
-        launch_units = step_units / L
-        roof = {"bound": "tensor", "kernel": "q4kv_prefill_attention (one call per layer)",
-                "achieved": launch_units / att_avg_s / 1e12, "peak": tf_sust, "unit": "TFLOP/s",
-                "peak_kind": peak_kind + " sustained bf16"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
-    roof["avg_launch_us"] = att_avg_s * 1e6
+    res = measure(w, args, local, dist, full=True)
+    t_step, t_e2e = slowest_rank(torch, dist, [res["t_step"], res["t_e2e"]], "cuda")
+    step_units, roof = roofline_of(w, res)
     value = world * step_units / t_step / div
     e2e_val = world * step_units / t_e2e / div
-
+    clocks = res["clocks"]
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16 tensor-core products on u4 codes, f32 accumulate", "data": "synthetic",
-        "config": {"workload": workload_name(w), "layers": L, "agents": w.n_agents, "kv_lens": w.lens if len(set(w.lens)) > 1 else w.lens[0],
-                   "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "d_qk": w.d_qk, "d_v": w.d_v,
-                   "new_tokens_per_agent": w.new_tokens, "window": w.window,
-                   "l2": "inputs larger than L2: every step streams the whole multi-layer cache",
-                   "launch": "cuda graph replay of the L-layer step" if graph is not None else "eager",
-                   "update_and_fetch": "one call per layer" if (fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"))
-                   else "quantize-append launch + attention launch per layer",
-                   "multi_gpu": "replicas only"},
+        "config": config_of(w, res),
         "agent_steps_per_s": world * w.n_agents / t_step,
         "step_bytes" if w.kind == "decode" else "step_flops": step_units,
-        "append_avg_us": app_ms_avg * 1e3,
+        "append_avg_us": res["app_s"] * 1e6,
         "roofline": roof,
-        "e2e": {"value": e2e_val, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        "e2e": {"value": e2e_val, "unit": unit, "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"],
                 "ms_per_step": t_e2e * 1e3},
-        "gpu_launches": dw_launches(w) * args.steps,
+        "gpu_launches": dw_launches(w, args.two_calls) * args.steps,
         "clocks": clocks,
+        "ms_per_step_x_sm_mhz": None if not clocks.get("sm_mhz") else t_step * 1e3 * clocks["sm_mhz"],
     }
+    if rank == 0 and world == 1 and default_run and not args.no_all_configs:
+        allc = {}
+        for idx in (2, 3, 4):
+            wi = synth.workload(idx)
+            ri = measure(wi, args, local, None, full=False)
+            units_i, roof_i = roofline_of(wi, ri)
+            mi, ui, di = metric_of(wi)
+            allc[wi.name] = {"metric": mi, "value": units_i / ri["t_step"] / di, "unit": ui,
+                             "ms_per_step": ri["t_step"] * 1e3, "agent_steps_per_s": wi.n_agents / ri["t_step"],
+                             "append_avg_us": ri["app_s"] * 1e6, "roofline": roof_i, "config": config_of(wi, ri),
+                             "gpu_launches_per_step": dw_launches(wi, args.two_calls), "clocks": ri["clocks"]}
+        pk = run_pack(args)
+        for name in ("pack", "unpack", "append_8x1024"):
+            allc[name] = pk["kernels"][name]
+        line["all_configs"] = allc
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt_o, units_o, desc, threads = oracle_sample(w)
         line["cpu_baseline"] = {"value": units_o / dt_o / div, "unit": unit, "cores": threads, "kind": "oracle",
@@ -537,38 +607,53 @@ def run_pack(args):
     dc = H.DeviceCache(L, Hq, Hkv, D, D, False, nb, synth.block_tables(synth.BASE_SEED, 99, [n], nb), fill_byte=7)
     nbytes = B.q4kv_packed_bytes(dc.spec, n)
     dst = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    min_s = getattr(args, "min_seconds", 0.5) / 2
 
     def timed(fn):
         for _ in range(max(3, args.warmup)):
             fn()
-        return time_region(torch, fn, args.steps) / args.steps
+        return float(np.median(timed_batches(torch, fn, 1, min_total_s=min_s, max_batches=2000)))
     t_pack = timed(lambda: B.q4kv_pack(dc.spec, dc.pool, dc.n_blocks, dc.tables[0], n, dst, dc.flags))
     t_unpack = timed(lambda: B.q4kv_unpack(dc.spec, dst, n, dc.pool, dc.n_blocks, dc.tables[0], dc.flags))
     A, new = 8, 1024
     lens = [8192] * A
     nb2 = sum(-(-(x + new) // 256) for x in lens) + 2
-    dc2 = H.DeviceCache(1, Hq, Hkv, D, D, False, nb2, synth.block_tables(synth.BASE_SEED, 98, lens, nb2, extra_tokens=new),
+    # 32 layers' worth of new rows (1.07 GB), so that consecutive launches do not find their inputs in L2
+    LA = 32
+    dc2 = H.DeviceCache(LA, Hq, Hkv, D, D, False, nb2, synth.block_tables(synth.BASE_SEED, 98, lens, nb2, extra_tokens=new),
                         fill_byte=None)
-    k = torch.randn((A * new, Hkv, D), device="cuda").to(torch.bfloat16)
-    v = torch.randn((A * new, Hkv, D), device="cuda").to(torch.bfloat16)
+    k = torch.randn((LA, A * new, Hkv, D), device="cuda").to(torch.bfloat16)
+    v = torch.randn((LA, A * new, Hkv, D), device="cuda").to(torch.bfloat16)
     pos = H.dev(np.asarray(lens, dtype=np.int32))
     offs = H.dev(np.arange(A + 1, dtype=np.int32) * new)
-    t_app = timed(lambda: B.q4kv_quantize_append(dc2.spec, dc2.pool, dc2.n_blocks, 0, dc2.bt, pos, offs, A * new, k, v,
-                                                 dc2.flags))
-    app_bytes = k.numel() * 2 * 2 + A * new * Hkv * 144
+
+    def append_all():
+        for l in range(LA):
+            B.q4kv_quantize_append(dc2.spec, dc2.pool, dc2.n_blocks, l, dc2.bt, pos, offs, A * new, k[l], v[l], dc2.flags)
+    t_app = timed(append_all) / LA
+    app_bytes = A * new * Hkv * D * 2 * 2 + A * new * Hkv * 144
     assert dc.read_flags() == 0 and dc2.read_flags() == 0
-    line = {"metric": "q4_pack_hbm_gbps", "value": 2 * nbytes / t_pack / 1e9, "unit": "GB/s", "n_gpus": 1,
+
+    def entry(kernel, nbytes_moved, t, note):
+        ach = nbytes_moved / t / 1e9
+        return {"metric": "hbm_gbps", "value": ach, "unit": "GB/s", "ms_per_step": t * 1e3,
+                "roofline": {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
+                             "frac": ach / hbm_peak, "peak_kind": peak_kind, "avg_launch_us": t * 1e6,
+                             "traffic": NCU_TRAFFIC_BYTES.get(note)},
+                "bytes": nbytes_moved}
+    kernels = {"pack": entry("q4kv_pack", 2 * nbytes, t_pack, "pack"),
+               "unpack": entry("q4kv_unpack", 2 * nbytes, t_unpack, "unpack"),
+               "append_8x1024": entry("q4kv_quantize_append (8 agents x 1024 new tokens, one layer per launch)", app_bytes,
+                                      t_app, "append_8x1024")}
+    line = {"metric": "q4_pack_hbm_gbps", "value": kernels["pack"]["value"], "unit": "GB/s", "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_pack * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
             "config": {"workload": "pack_unpack_append_llama31_8b_agent", "packed_bytes": nbytes,
-                       "l2": "packed buffer + pool (302 MB) larger than L2"},
-            "roofline": {"bound": "hbm", "kernel": "q4kv_pack", "achieved": 2 * nbytes / t_pack / 1e9, "peak": hbm_peak,
-                         "unit": "GB/s", "frac": 2 * nbytes / t_pack / 1e9 / hbm_peak, "peak_kind": peak_kind, "traffic": None},
-            "unpack": {"achieved": 2 * nbytes / t_unpack / 1e9, "frac": 2 * nbytes / t_unpack / 1e9 / hbm_peak, "us": t_unpack * 1e6},
-            "append_8x1024": {"achieved": app_bytes / t_app / 1e9, "frac": app_bytes / t_app / 1e9 / hbm_peak, "us": t_app * 1e6,
-                              "bytes": app_bytes},
-            "gpu_launches": args.steps}
-    print(json.dumps(line))
+                       "l2": "packed buffer + pool (302 MB) larger than L2; append: 32 layers of new rows (1.07 GB)"},
+            "roofline": kernels["pack"]["roofline"], "kernels": kernels, "gpu_launches": args.steps}
+    del dc, dc2, k, v, dst
+    torch.cuda.empty_cache()
+    return line
 
 
 def fused_update_and_fetch(w):
@@ -581,12 +666,12 @@ def fused_update_and_fetch(w):
     return w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
 
 
-def dw_launches(w):
+def dw_launches(w, two_calls=False):
     """Kernels of this library launched per step.  GQA decode: one update-and-fetch kernel per layer.  MLA-latent
     decode: the key-split update-and-fetch kernel and its merge kernel.  Prefill: one quantize-append and one
     attention kernel per layer.  As two calls, decode launches the quantize-append kernel as well."""
     mla = w.kind == "decode" and w.v_aliases_k
-    if fused_update_and_fetch(w) and not os.environ.get("Q4KV_BENCH_TWO_CALLS"):
+    if fused_update_and_fetch(w) and not two_calls:
         return (2 if mla else 1) * w.n_layers
     return (3 if mla else 2) * w.n_layers
 

@@ -33,7 +33,7 @@
  *     after the preceding kernels have completed.  Lengths and block tables
  *     must therefore not be written by a preceding kernel that itself signals
  *     its dependents early; an ordinary kernel, a copy or a memset is fine.
- *     Setting Q4KV_NO_PDL in the environment turns the overlap off.
+ *   - The library reads no environment variable; every choice is an argument.
  *
  * Q4 format (Section 3.2): groups of 64 consecutive head-dim elements; per
  * group one binary16 scale and one binary16 bias; 4-bit codes, value =
@@ -74,6 +74,9 @@ typedef struct {
   int32_t group;         /* quantization group, must be 64                                          */
   int32_t block_tokens;  /* tokens per pool block, must be 256                                      */
   int32_t sb_dtype;      /* scale/bias type: 0 = binary16 (only value supported)                    */
+  int32_t exact_products;/* 0: attention kernels may expand the cache into binary16 tiles (one rounding
+                            of every dequantized value, see "Accuracy" below); 1: always multiply the
+                            4-bit codes exactly.  Ignored by append, pack and unpack.               */
 } q4kv_spec;
 
 /* One batch of agents. */
@@ -97,6 +100,24 @@ enum {
   Q4KV_FLAG_INTERNAL = 4     /* a bounded wait inside a kernel ran out (the output is not valid)    */
 };
 enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
+
+/* Accuracy of the attention entry points (float32 output, against the attention over the exactly
+ * dequantized values evaluated in float64).  Let M be the largest |code*scale + bias| among the
+ * attended keys and values.
+ *   - Kernels that multiply the 4-bit codes (GQA decode with d_qk = d_v in {128, 256} and at most
+ *     four query heads per KV head; prefill with d = 128 and exact_products = 1; the shape-agnostic
+ *     kernels every other case falls back to): the products are exact, sums are float32, the
+ *     probabilities enter the value product as a two-term binary16 pair or as float32.  Error
+ *     at most 2e-5 * M + 1e-5, i.e. within 2e-3 for any cache with M <= 64.
+ *   - Kernels that expand the cache into binary16 tiles (prefill with d_qk = d_v = 128 and 1, 2 or 4
+ *     query heads per KV head; decode on the MLA-latent cache: V aliasing K, d_qk 576, d_v 512, one
+ *     KV head, at most 16 query heads) round every dequantized value once to binary16, a relative
+ *     error of 2^-11 at most, and the probabilities likewise.  They are chosen only when
+ *     exact_products == 0 and softmax_scale <= 2/sqrt(d_qk).  Their error is at most
+ *     2^-10 * M * (1 + softmax_scale * ||q||_1 * M): the value and probability roundings, plus what
+ *     the rounded keys do to the softmax weights.  On caches of unit-variance values (M about 5) the
+ *     roundings average out over the attended keys and the measured error is below 3e-4; a cache
+ *     with outlier channels or a gain (M >= 8) needs exact_products = 1 to stay within 2e-3. */
 
 const char* q4kv_status_string(int code);
 
@@ -129,15 +150,21 @@ int q4kv_quantize_append(const q4kv_spec* spec, void* pool, int32_t n_blocks, in
  * the dequantized values, keys [lo, kv_len) with lo = max(0, kv_len - window) when window > 0
  * (sliding-window layers), lo = 0 when window == 0.
  *   kv_lens    [A]  cached tokens to attend (the query sits at position kv_len-1)
- *   max_kv_len      host upper bound on every kv_len (sizes the split grid); 0 = max_blocks*256
+ *   max_kv_len      host upper bound on every kv_len (sizes the split grid); 0 = max_blocks*256.
+ *                   An agent whose kv_len exceeds it is treated like any other bad length:
+ *                   Q4KV_FLAG_BAD_LENGTH, zeros for that agent.
  *   q          bf16 [A][n_q_heads][d_qk]
  *   out        [A][n_q_heads][d_v], float32 or bf16 per out_dtype
  *   lse        optional float32 [A][n_q_heads], natural-log sum of exponentials; may be NULL
- *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, 0) bytes.  Fill it with zero bytes once
- *              after allocating it: its head holds the arrival counters of the split merge, which
- *              every call finds at zero and leaves at zero.  (If a call ever reports
- *              Q4KV_FLAG_INTERNAL, zero it again.)  Nothing else in it carries over between calls.
+ *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, 0) bytes.  Its first
+ *              Q4KV_WORKSPACE_HEADER_BYTES hold the arrival counters of the split merge: fill them
+ *              with zero bytes once after allocating the workspace; every call finds them at zero
+ *              and leaves them at zero, whatever the spec, the batch size or the kernel chosen, so
+ *              one workspace sized for the largest batch serves all calls.  (If a call ever reports
+ *              Q4KV_FLAG_INTERNAL, zero the header again.)  Nothing behind the header carries over
+ *              between calls.
  * kv_len == 0 gives zeros and lse = -inf without a flag. */
+#define Q4KV_WORKSPACE_HEADER_BYTES 65536u
 int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                           const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
                           int32_t window, const void* q, float softmax_scale,
@@ -157,7 +184,8 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
  *                 (v_new is ignored, and may be NULL, when V aliases K)
  * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256} with at
  * most four query heads per KV head and V not aliasing K; and the MLA-latent cache (V aliasing K,
- * d_qk 576, d_v 512, one KV head, at most 16 query heads) with softmax_scale^2 * d_qk <= 4.
+ * d_qk 576, d_v 512, one KV head, at most 16 query heads) with exact_products == 0 and
+ * softmax_scale^2 * d_qk <= 4.
  * Anything else returns Q4KV_EUNSUPPORTED and the caller makes the two calls.  Two agents must
  * not share the block that is written. */
 int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
@@ -182,9 +210,13 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
  *     The first call on each device looks up the array's device address (a host-side query, no
  *     launch); make that first call before any stream capture begins on that device.
  *   - All calls on one device share the one array, and it keeps whatever the last call left in
- *     it (no call depends on those contents).  Two calls that overlap on the GPU -- different
- *     streams, or one stream per thread -- race on it and give wrong results: order them on one
- *     stream, or give the concurrent ones their own workspace through q4kv_decode_attention. */
+ *     it.  Each call first clears the arrival counters at the head of the array with a memset
+ *     enqueued on its own stream (no allocation), so a call never depends on what an earlier one
+ *     left there -- not even one that ended with Q4KV_FLAG_INTERNAL; the partial records behind
+ *     the counters are written before they are read within a call.  Two calls that overlap on the
+ *     GPU -- different streams, or one stream per thread -- race on the array and give wrong
+ *     results: order them on one stream, or give the concurrent ones their own workspace through
+ *     q4kv_decode_attention. */
 #define Q4KV_STATIC_SCRATCH_BYTES (8u << 20)
 int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                                  const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
@@ -202,14 +234,8 @@ int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_
  *   total_q, max_q_len, max_kv_len   host copies / upper bounds (size the grid)
  *   q bf16 [total_q][n_q_heads][d_qk];  out [total_q][n_q_heads][d_v];  lse optional
  *   workspace  at least q4kv_workspace_bytes(spec, A, max_kv_len, total_q) bytes
- * Accuracy: outputs are within 2e-3 (absolute) of the attention over the exactly dequantized
- * values.  For d_qk = d_v = 128 with 1, 2 or 4 query heads per KV head and softmax_scale at most
- * 2/sqrt(d_qk) the dequantized keys and values are rounded once to binary16 (11 significant bits)
- * on their way to the tensor cores; sharper scales, and every other shape, use kernels that
- * multiply the 4-bit codes exactly.  Setting Q4KV_PREFILL_PATH=mma in the environment selects the
- * exact kernel for d = 128 as well.  The same rule (scale at most 2/sqrt(d_qk)) selects the
- * binary16-tile kernel of q4kv_decode_attention for the MLA-latent shape (d_qk 576, d_v 512
- * aliasing K, one KV head, at most 16 query heads). */
+ * Accuracy: see "Accuracy of the attention entry points" above (spec->exact_products selects
+ * between the binary16-tile kernel and the kernel that multiplies the codes). */
 int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer,
                            const q4kv_batch* batch, const int32_t* kv_lens, const int32_t* q_offs,
                            int32_t total_q, int32_t max_q_len, int32_t max_kv_len,

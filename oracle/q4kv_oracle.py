@@ -39,12 +39,6 @@ BLOCK_TOKENS = 256  # tokens per pool block (Section 3.1)
 # ----------------------------------------------------------------------------
 # number formats
 # ----------------------------------------------------------------------------
-def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
-    """bfloat16 bit patterns (uint16) -> binary32, exact."""
-    bits = np.asarray(bits, dtype=np.uint16)
-    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
-
-
 def _f16_round_down(x32: np.ndarray) -> np.ndarray:
     """binary32 -> binary16, rounding toward -infinity."""
     h = x32.astype(np.float16)                       # round to nearest first

@@ -26,6 +26,7 @@ EXPORTS = [
     "q4kv_decode_attention_static", "q4kv_append_decode_attention",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
+WORKSPACE_HEADER_BYTES = 65536
 
 
 class Q4KVError(RuntimeError):
@@ -36,11 +37,13 @@ class Q4KVError(RuntimeError):
 
 class Spec(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
-        "n_layers", "n_q_heads", "n_kv_heads", "d_qk", "d_v", "v_aliases_k", "group", "block_tokens", "sb_dtype")]
+        "n_layers", "n_q_heads", "n_kv_heads", "d_qk", "d_v", "v_aliases_k", "group", "block_tokens", "sb_dtype",
+        "exact_products")]
 
     @classmethod
-    def make(cls, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False):
-        return cls(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), 64, 256, 0)
+    def make(cls, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False, exact_products=False):
+        return cls(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), 64, 256, 0,
+                   int(bool(exact_products)))
 
 
 class Batch(ctypes.Structure):

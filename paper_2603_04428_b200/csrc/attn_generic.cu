@@ -22,8 +22,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct ItemInfo { int agent, q_row, pos_end, lo; };   // keys [lo, pos_end)
 
 // Decode: item = agent.  Prefill: item = global query row; agent found by scanning q_offs.
+// len_cap: the host's bound on every length (at most max_blocks * 256); the key splits cover exactly that many keys
 __device__ inline bool locate_item(int item, int n_agents, const int32_t* kv_lens, const int32_t* q_offs,
-                                   int window, int max_blocks, int32_t* flags, ItemInfo& it) {
+                                   int window, int len_cap, int32_t* flags, ItemInfo& it) {
   int a, pos_end;
   if (q_offs == nullptr) {
     a = item;
@@ -42,7 +43,7 @@ __device__ inline bool locate_item(int item, int n_agents, const int32_t* kv_len
   }
   it.agent = a; it.q_row = item;
   const int n_all = kv_lens[a];
-  if (n_all < 0 || n_all > max_blocks * kBlockTokens) {
+  if (n_all < 0 || n_all > len_cap) {
     raise_flag(flags, Q4KV_FLAG_BAD_LENGTH);
     it.pos_end = -1; it.lo = 0;
     return false;
@@ -56,7 +57,7 @@ __device__ inline bool locate_item(int item, int n_agents, const int32_t* kv_len
 //       + kWarps * (Dv + 2) floats (cross-warp merge)
 __global__ void __launch_bounds__(kThreads)
 attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, int layer, int n_agents,
-                    int max_blocks, const int32_t* __restrict__ tables, const int32_t* __restrict__ kv_lens,
+                    int max_blocks, int len_cap, const int32_t* __restrict__ tables, const int32_t* __restrict__ kv_lens,
                     const int32_t* __restrict__ q_offs, int window, const uint16_t* __restrict__ q,
                     float scale_log2, int n_splits, int split_tokens,
                     float* __restrict__ partials, void* __restrict__ out, int out_dtype,
@@ -72,7 +73,7 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
   const int nd = Dv / 32;
 
   ItemInfo it;
-  const bool ok = locate_item(item, n_agents, kv_lens, q_offs, window, max_blocks, flags, it);
+  const bool ok = locate_item(item, n_agents, kv_lens, q_offs, window, len_cap, flags, it);
   const size_t out_index = ((size_t)it.q_row * y.Hq + h) * Dv;
   float* part = partials + (((size_t)item * y.Hq + h) * n_splits + split) * (Dv + 2);
 
@@ -258,7 +259,7 @@ DecodePlan plan_decode(const Layout& y, int n_agents, int max_kv_len, int window
   // keys one query can touch (the window start is rounded down to a multiple of 8)
   const int span = (window > 0 && window + 8 < max_kv_len) ? window + 8 : max_kv_len;
   const int ctas = n_agents * y.Hq;
-  int n_splits = (4 * 148 + ctas - 1) / ctas;
+  int n_splits = (4 * sm_count() + ctas - 1) / ctas;
   const int max_splits = (span + 255) / 256;
   if (n_splits > max_splits) n_splits = max_splits;
   if (n_splits < 1) n_splits = 1;
@@ -290,7 +291,7 @@ cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_bl
   {
     dim3 grid(items, y.Hq, plan.n_splits);
     attn_generic_kernel<<<grid, kThreads, smem, st>>>(
-        y, (const uint8_t*)pool, n_blocks, layer, b.n_agents, b.max_blocks, b.block_tables, kv_lens, q_offs,
+        y, (const uint8_t*)pool, n_blocks, layer, b.n_agents, b.max_blocks, max_kv_len, b.block_tables, kv_lens, q_offs,
         window, (const uint16_t*)q, scale * kLog2e, plan.n_splits, plan.split_tokens, (float*)ws, out, out_dtype,
         lse, flags);
     e = cudaGetLastError();

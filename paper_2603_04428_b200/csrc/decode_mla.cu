@@ -57,6 +57,7 @@ struct MlaParams {
   int n_blocks, layer, n_agents, max_blocks;
   const int32_t* tables;
   const int32_t* kv_lens;
+  int len_cap;
   int window;
   const uint16_t* q;          // bf16 [n_agents][Hq][576]
   const uint16_t* k_new;      // bf16 [n_agents][576]: the row at position kv_len - 1, quantized and stored by this launch; or null
@@ -138,7 +139,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- this CTA's share of the agent's keys (inputs no kernel writes) ----
   int n = P.kv_lens[a];
-  const bool bad_len = n < 0 || n > P.max_blocks * kBlockTokens;
+  const bool bad_len = n < 0 || n > P.len_cap;       // the host's bound on every length: the key shares cover that many keys
   if (bad_len) n = 0;
   const int lo = P.window > 0 ? max(0, n - P.window) : 0;
   const int b_lo = lo >> 6, b_hi = (n + 63) >> 6;        // 64-key blocks of the attended range
@@ -548,7 +549,7 @@ struct MlaPlan { int n_splits, blocks_per_split; };
 MlaPlan plan_mla(int n_agents, int max_kv_len, int window) {
   const int span = (window > 0 && window + 64 < max_kv_len) ? window + 64 : max_kv_len;
   const int blocks = (span + 63) / 64 + 1;               // a window may straddle one more 64-key block
-  int n_splits = (148 + n_agents - 1) / n_agents;        // about one CTA per SM
+  int n_splits = (sm_count() + n_agents - 1) / n_agents;   // about one CTA per SM
   if (n_splits > blocks) n_splits = blocks;
   if (n_splits > kMaxSplits) n_splits = kMaxSplits;
   if (n_splits < 1) n_splits = 1;
@@ -580,7 +581,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   if (plan.n_splits > full.n_splits) plan = full;        // never more records than the workspace was sized for
   MlaParams P;
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
-  P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
+  P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.len_cap = max_kv_len; P.window = window;
   P.q = (const uint16_t*)q; P.k_new = (const uint16_t*)k_new; P.scale_log2 = scale * kLog2e; P.n_splits = plan.n_splits;
   P.blocks_per_split = plan.blocks_per_split; P.records = (float*)ws; P.flags = flags;
   static bool configured[64] = {};
@@ -602,7 +603,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, decode_mla_kernel, P);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t mcfg = {};
@@ -610,7 +611,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   mcfg.blockDim = dim3(kMergeThreads);
   mcfg.stream = st;
   mcfg.attrs = attr;
-  mcfg.numAttrs = pdl_enabled() ? 1 : 0;
+  mcfg.numAttrs = 1;
   return cudaLaunchKernelEx(&mcfg, merge_mla_kernel, (int)y.Hq, plan.n_splits, (const float*)ws, out, out_dtype, lse);
 }
 

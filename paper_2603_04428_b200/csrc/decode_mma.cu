@@ -34,8 +34,6 @@
 //     the query heads and rows 4..7 repeat them; rows 4..7 go on to carry the low half of a
 //     two-term binary16 split of p*s, which makes the value product accurate to ~2^-22 at no
 //     extra MMA.
-#include <cstdlib>
-
 #include "q4kv_layout.cuh"
 #include "quantize_core.cuh"
 
@@ -43,7 +41,7 @@ namespace q4kv {
 
 namespace {
 
-constexpr int kMaxCtas = 148;                          // one persistent CTA per SM
+constexpr int kMaxGrid = 512;                          // upper bound on the persistent grid (one CTA per SM)
 constexpr uint32_t kSpinLimit = 1u << 22;              // bounded mbarrier waits (each try blocks a while in hardware)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kMaskLo = 0x000F000Fu, kMaskHi = 0x00F000F0u;
@@ -139,11 +137,12 @@ __device__ inline uint32_t f32x2_to_h2_rn(float lo, float hi) {
 // ---------------------------------------------------------------------------------------------
 struct AgentRange { int n, lo, cf, nc; };   // keys [lo, n); chunks cf .. cf+nc-1
 
-__device__ inline AgentRange agent_range(const int32_t* __restrict__ kv_lens, int a, int window, int max_blocks,
+// len_cap: the host's bound on every length (at most max_blocks * 256); longer or negative lengths are rejected
+__device__ inline AgentRange agent_range(const int32_t* __restrict__ kv_lens, int a, int window, int len_cap,
                                          bool& bad) {
   AgentRange r;
   r.n = kv_lens[a];
-  bad = r.n < 0 || r.n > max_blocks * kBlockTokens;
+  bad = r.n < 0 || r.n > len_cap;
   if (bad) r.n = 0;
   r.lo = window > 0 ? max(0, r.n - window) : 0;
   r.cf = r.lo >> 5;
@@ -168,7 +167,7 @@ struct Partition {
 struct RangeStart { uint32_t U, u_begin, u_end, agent_start; int n_ctas, agent; bool any_bad; Partition part; };
 
 __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int n_agents, int Hkv, int window,
-                                        int max_blocks, int cta, int grid) {
+                                        int len_cap, int cta, int grid) {
   const int lane = threadIdx.x & 31;
   RangeStart rs;
   rs.any_bad = false;
@@ -179,7 +178,7 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
     const int a = base + lane;
     uint32_t cnt = 0;
     bool bad = false;
-    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, max_blocks, bad).nc * Hkv);
+    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, len_cap, bad).nc * Hkv);
     rs.any_bad |= __any_sync(0xffffffffu, bad);
     uint32_t inc = cnt;
 #pragma unroll
@@ -211,7 +210,7 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
     const int a = base + lane;
     uint32_t cnt = 0;
     bool bad = false;
-    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, max_blocks, bad).nc * Hkv);
+    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, len_cap, bad).nc * Hkv);
     uint32_t inc = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -242,20 +241,20 @@ struct Segment {
 
 struct Walker {
   const int32_t* kv_lens;
-  int n_agents, Hkv, window, max_blocks;
+  int n_agents, Hkv, window, len_cap;
   uint32_t u, u_end;
   int k, a, hk, c;
   AgentRange r;
 
-  __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int max_blocks_,
+  __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int len_cap_,
                        const RangeStart& rs) {
-    kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; max_blocks = max_blocks_;
+    kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; len_cap = len_cap_;
     u = rs.u_begin; u_end = rs.u_end; k = 0;
     a = rs.agent; hk = 0; c = 0;
     r.n = 0; r.lo = 0; r.cf = 0; r.nc = 0;
     if (u < u_end && a >= 0) {
       bool bad;
-      r = agent_range(kv_lens, a, window, max_blocks, bad);
+      r = agent_range(kv_lens, a, window, len_cap, bad);
       const uint32_t rem = u - rs.agent_start;
       hk = (int)(rem / (uint32_t)r.nc);
       c = r.cf + (int)(rem - (uint32_t)hk * (uint32_t)r.nc);
@@ -277,7 +276,7 @@ struct Walker {
         do {
           ++a;
           if (a >= n_agents) { a = -1; break; }
-          r = agent_range(kv_lens, a, window, max_blocks, bad);
+          r = agent_range(kv_lens, a, window, len_cap, bad);
         } while (r.nc == 0);
       }
       if (a >= 0) c = r.cf;
@@ -294,14 +293,14 @@ struct Walker {
 struct DecodeParams {
   Layout y;
   const uint8_t* pool;
-  int n_blocks, layer, n_agents, max_blocks;
+  int n_blocks, layer, n_agents, max_blocks, len_cap;
   const int32_t* tables;
   const int32_t* kv_lens;
   int window;
   const uint16_t* q;          // bf16 [A][Hq][D]
   float scale_log2;           // softmax_scale * log2(e)
   int32_t* tickets;           // [A*Hkv], zero between calls
-  float* partials;            // [A*Hkv + kMaxCtas][n_rep][Dv + 4]
+  float* partials;            // [A*Hkv + grid][n_rep][Dv + 4]
   void* out;
   int out_dtype;
   float* lse;
@@ -827,11 +826,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   __syncthreads();
 
   // ---- this CTA's unit range (every warp computes it for itself; these inputs are not written by any kernel) ----
-  const RangeStart rs = find_range(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, cta, gridDim.x);
+  const RangeStart rs = find_range(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, cta, gridDim.x);
   if (rs.any_bad && cta == 0 && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
   const int n_chunks = (int)(rs.u_end - rs.u_begin);
   Walker wk;
-  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.max_blocks, rs);
+  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, rs);
   Segment seg;
 
   // =============================== producer warp ===============================================
@@ -892,7 +891,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   // agents without any key (kv_len == 0 or a rejected length): zeros, lse = -inf
   for (int a = cta * NW + warp; a < P.n_agents; a += gridDim.x * NW) {
     bool bad_len;
-    if (agent_range(P.kv_lens, a, P.window, P.max_blocks, bad_len).nc > 0) continue;
+    if (agent_range(P.kv_lens, a, P.window, P.len_cap, bad_len).nc > 0) continue;
     for (int i = lane; i < y.Hq * Dv; i += 32) store_out(P, (size_t)a * y.Hq * Dv + i, 0.f);
     if (P.lse) for (int i = lane; i < y.Hq; i += 32) P.lse[(size_t)a * y.Hq + i] = -INFINITY;
   }
@@ -1067,27 +1066,33 @@ cudaError_t launch_g(const DecodeParams& P, int grid, bool pdl, cudaStream_t st)
 
 }  // namespace
 
-// Programmatic dependent launch lets a kernel's prologue overlap the tail of its predecessor in the
-// stream; every kernel of this library waits on its predecessors before it reads or writes shared
-// state.  Setting Q4KV_NO_PDL in the environment falls back to plain stream order.
-bool pdl_enabled() {
-  static const bool on = std::getenv("Q4KV_NO_PDL") == nullptr;
-  return on;
+// Number of SMs of the current device (one persistent CTA each), looked up once per device.
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 148; }
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = 148; }
+    cached[dev] = n < kMaxGrid ? n : kMaxGrid;
+  }
+  return cached[dev];
 }
 
 bool decode_mma_supported(const Layout& y) {
   return !y.alias && y.D == y.Dv && (y.D == 128 || y.D == 256) && y.n_rep <= 4;
 }
 
-// the kernel counts work units in 32 bits
+// the kernel counts work units in 32 bits and keeps one arrival counter per (agent, KV head) pair in the
+// workspace header
 bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks) {
-  return (long long)n_agents * y.Hkv * (max_blocks * 8ll) < (1ll << 30);
+  return (long long)n_agents * y.Hkv * (max_blocks * 8ll) < (1ll << 30) && (long long)n_agents * y.Hkv <= kMaxTicketPairs;
 }
 
+// bytes behind the workspace header: one record per pair and per CTA of the largest grid
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents) {
   const size_t pairs = (size_t)n_agents * y.Hkv;
-  const size_t tickets = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
-  return tickets + (pairs + kMaxCtas) * y.n_rep * kRecStride(y.Dv) * sizeof(float);
+  return (pairs + kMaxGrid) * y.n_rep * kRecStride(y.Dv) * sizeof(float);
 }
 
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
@@ -1095,22 +1100,18 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
                               void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
                               const void* k_new, const void* v_new) {
   if (b.n_agents <= 0) return cudaSuccess;
-  const size_t pairs = (size_t)b.n_agents * y.Hkv;
-  const size_t ticket_bytes = (pairs * sizeof(int32_t) + 255) & ~(size_t)255;
   DecodeParams P;
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
-  P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
+  P.max_blocks = b.max_blocks; P.len_cap = max_kv_len; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e;
-  P.tickets = (int32_t*)ws; P.partials = (float*)((uint8_t*)ws + ticket_bytes);
+  P.tickets = (int32_t*)ws; P.partials = (float*)((uint8_t*)ws + kWorkspaceHeaderBytes);
   P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
   P.k_new = (const uint16_t*)k_new; P.v_new = (const uint16_t*)v_new;
   const int span = (window > 0 && window + 32 < max_kv_len) ? window + 32 : max_kv_len;
   const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
-  const int grid = (int)(units < kMaxCtas ? (units < 1 ? 1 : units) : kMaxCtas);
-  const bool pdl = pdl_enabled();
-  static const int nw = std::getenv("Q4KV_DECODE_NW") ? std::atoi(std::getenv("Q4KV_DECODE_NW")) : 7;
-  if (nw == 11) return y.G == 2 ? launch_g<2, 11>(P, grid, pdl, st) : launch_g<4, 11>(P, grid, pdl, st);
-  return y.G == 2 ? launch_g<2, 7>(P, grid, pdl, st) : launch_g<4, 7>(P, grid, pdl, st);
+  const int n_sm = sm_count();
+  const int grid = (int)(units < n_sm ? (units < 1 ? 1 : units) : n_sm);
+  return y.G == 2 ? launch_g<2, 7>(P, grid, true, st) : launch_g<4, 7>(P, grid, true, st);
 }
 
 }  // namespace q4kv

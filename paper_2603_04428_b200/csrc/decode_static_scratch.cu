@@ -58,10 +58,11 @@ int q4kv_decode_attention_static(const q4kv_spec* spec, const void* pool, int32_
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);
   if (rc != Q4KV_OK) return rc;
-  // The arrival counters at the head of the scratch must be zero when a call starts: the array is
-  // zero at module load and the kernel puts each counter back to zero when its last arrival is
-  // drawn.  Every partial record read from the rest was written earlier in the same call, so the
-  // previous call's records are simply overwritten.
+  // The arrival counters at the head of the scratch must be zero when the kernel starts.  A call that ran to its end
+  // leaves them at zero, but one that gave up (Q4KV_FLAG_INTERNAL) may not have, and this caller has no buffer of its
+  // own to clear: so every call clears the header first, with a memset enqueued on its stream (no allocation).  The
+  // partial records behind the header are written before they are read within a call.
+  if (cudaMemsetAsync(scratch, 0, q4kv::kWorkspaceHeaderBytes, (cudaStream_t)stream) != cudaSuccess) return Q4KV_ECUDA;
   return q4kv_decode_attention(spec, pool, n_blocks, layer, batch, kv_lens, max_kv_len, window, q, softmax_scale,
                                out, out_dtype, lse, scratch, kStaticScratchBytes, status_flags, stream);
 }

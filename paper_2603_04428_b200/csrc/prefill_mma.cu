@@ -16,7 +16,8 @@
 //     scale, and the token's bias meets the row's per-group query sum.
 //   * Values: mma.sync m16n8k16 f16 with the value codes as binary16 subnormals c * 2^-24 (masked in
 //     place from the token-packed words) and probabilities pre-multiplied by the token's group scale,
-//     rounded once to binary16; the bias part is a per-row scalar sum.
+//     carried as a two-term binary16 sum (two products per value tile), so the value product is good
+//     to ~2^-22 of the cached magnitudes; the bias part is a per-row float32 scalar sum.
 //   * The score fragment of two adjacent key tiles is the A fragment of the value product, as in any
 //     register-resident flash attention, so probabilities never leave their lane.
 #include "q4kv_layout.cuh"
@@ -242,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
       const int pos0 = (c_begin + k) * 32;
       const bool tail = pos0 + 32 > kv_len;              // slots past the cache end may hold stale bytes
 
-      uint32_t apv[R][G][2][4];                          // value-product A operands: [tile][group][MMA][register]
+      uint32_t apv[R][G][2][4], apl[R][G][2][4];         // value-product A operands, high and low term: [tile][group][MMA][register]
       bool active[R];
 #pragma unroll
       for (int rt = 0; rt < R; ++rt) {
@@ -330,7 +331,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
             o[rt][nt][0] *= corr[0]; o[rt][nt][1] *= corr[0]; o[rt][nt][2] *= corr[1]; o[rt][nt][3] *= corr[1];
           }
         }
-        // ---- p * s_v per group, rounded once to binary16: the A operand of the value product ----
+        // ---- p * s_v per group as a two-term binary16 sum (high part + rounded remainder): the A operands of the
+        // value product, which is then good to ~2^-22 whatever the magnitude of the cached values ----
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 sb = vsb4[i * 4 + tid];
@@ -344,7 +346,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
           for (int gi = 0; gi < G; ++gi)
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-              apv[rt][gi][i >> 1][(i & 1) * 2 + r] = f32x2_to_h2(s[i][0][r] * v[0][gi].x, s[i][1][r] * v[1][gi].x);
+              const float x0 = s[i][0][r] * v[0][gi].x, x1 = s[i][1][r] * v[1][gi].x;
+              const uint32_t hi = f32x2_to_h2(x0, x1);
+              const float2 hf = h2_to_f2(hi);
+              apv[rt][gi][i >> 1][(i & 1) * 2 + r] = hi;
+              apl[rt][gi][i >> 1][(i & 1) * 2 + r] = f32x2_to_h2(x0 - hf.x, x1 - hf.y);
               const float b = fmaf(s[i][0][r], v[0][gi].y, s[i][1][r] * v[1][gi].y);
               if (i & 1) bias_o[rt][r][gi] += b; else bias_e[rt][r][gi] += b;
             }
@@ -369,6 +375,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
               if (!active[rt]) continue;
               mma_f16(o[rt][4 * q4 + j], apv[rt][gi][0], be0, be1);
               mma_f16(o[rt][4 * q4 + j], apv[rt][gi][1], bo0, bo1);
+              mma_f16(o[rt][4 * q4 + j], apl[rt][gi][0], be0, be1);
+              mma_f16(o[rt][4 * q4 + j], apl[rt][gi][1], bo0, bo1);
             }
           }
         }
@@ -442,7 +450,7 @@ cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, prefill_mma_kernel<R>, P);
 }
 

@@ -533,7 +533,7 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, prefill_umma_kernel, P);
 }
 

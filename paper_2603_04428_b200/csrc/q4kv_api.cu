@@ -1,7 +1,5 @@
 // C ABI of libq4kv.so: host-side validation, sizing and dispatch.  See include/q4kv.h for
 // the contract of every entry point.
-#include <cstdlib>
-
 #include "q4kv_layout.cuh"
 
 using namespace q4kv;
@@ -14,6 +12,7 @@ int check_spec(const q4kv_spec* s) {
   if (!s) return Q4KV_EINVAL;
   if (s->n_layers <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->d_qk <= 0 || s->d_v <= 0) return Q4KV_EINVAL;
   if (s->group != 64 || s->block_tokens != 256 || s->sb_dtype != 0) return Q4KV_EUNSUPPORTED;
+  if (s->exact_products != 0 && s->exact_products != 1) return Q4KV_EINVAL;
   if (s->d_qk % 64 || s->d_v % 64 || s->n_q_heads % s->n_kv_heads) return Q4KV_EUNSUPPORTED;
   if (s->d_qk > 1024 || s->d_v > 512) return Q4KV_EUNSUPPORTED;
   if (s->v_aliases_k && s->d_v > s->d_qk) return Q4KV_EUNSUPPORTED;
@@ -26,17 +25,28 @@ int check_batch(const q4kv_batch* b) {
   return Q4KV_OK;
 }
 
+// Every decode kernel keeps its partial records behind a header of fixed size (the arrival counters
+// of the kernels that merge in the same launch), so that one workspace serves any sequence of calls.
 size_t workspace_need(const Layout& y, int n_agents, int max_kv_len, int total_q) {
   if (total_q > 0) return 16;   // the prefill path keeps no partials
   const DecodePlan p = plan_decode(y, n_agents, max_kv_len, 0);
-  size_t generic = (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
+  size_t need = (size_t)n_agents * y.Hq * p.n_splits * (y.Dv + 2) * sizeof(float) + 16;
   if (decode_mla_supported(y)) {
     const size_t mla = decode_mla_workspace_bytes(y, n_agents, max_kv_len);
-    if (mla > generic) generic = mla;
+    if (mla > need) need = mla;
   }
-  if (!decode_mma_supported(y)) return generic;
-  const size_t mma = decode_mma_workspace_bytes(y, n_agents);
-  return mma > generic ? mma : generic;
+  if (decode_mma_supported(y)) {
+    const size_t mma = decode_mma_workspace_bytes(y, n_agents);
+    if (mma > need) need = mma;
+  }
+  return kWorkspaceHeaderBytes + need;
+}
+
+// The kernels that expand the cache into binary16 tiles round each dequantized element once; they are taken only when
+// the spec allows it and the softmax scale is at most 2 / sqrt(d_qk) (the error a rounded key leaves in a score grows
+// with the scale).  Everything else multiplies the codes exactly.
+bool tiles_allowed(const q4kv_spec* s, float softmax_scale) {
+  return s->exact_products == 0 && softmax_scale > 0.f && softmax_scale * softmax_scale * (float)s->d_qk <= 4.f;
 }
 
 }  // namespace
@@ -109,20 +119,17 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
-  // The kernels that expand the cache into binary16 tiles round each dequantized element once; the error that leaves in a score grows with
-  // the softmax scale and stays well inside the library's 2e-3 output bound up to 2 / sqrt(d_qk).  Sharper scales
-  // take the kernels that multiply the codes exactly.
-  const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
+  void* records = (uint8_t*)workspace + kWorkspaceHeaderBytes;
   cudaError_t e;
-  if (decode_mla_supported(y) && usual_scale)
+  if (decode_mla_supported(y) && tiles_allowed(spec, softmax_scale))
     e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out, out_dtype,
-                          lse, workspace, status_flags, (cudaStream_t)stream);
+                          lse, records, status_flags, (cudaStream_t)stream);
   else if (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
     e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out,
                           out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
   else
     e = launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, nullptr, 0, 1, max_kv_len, window, q,
-                                 softmax_scale, out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
+                                 softmax_scale, out, out_dtype, lse, records, status_flags, (cudaStream_t)stream);
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 
@@ -148,11 +155,12 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
   if (decode_mla_supported(y)) {
-    // the latent-cache kernel expands the keys into binary16 tiles: usual softmax scales only (see q4kv_decode_attention)
-    if (!(softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f)) return Q4KV_EUNSUPPORTED;
+    // the latent-cache kernel expands the keys into binary16 tiles (see q4kv_decode_attention)
+    if (!tiles_allowed(spec, softmax_scale)) return Q4KV_EUNSUPPORTED;
     if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
     const cudaError_t e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,
-                                            out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream, k_new);
+                                            out, out_dtype, lse, (uint8_t*)workspace + kWorkspaceHeaderBytes, status_flags,
+                                            (cudaStream_t)stream, k_new);
     return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
   }
   if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks)) return Q4KV_EUNSUPPORTED;
@@ -184,12 +192,8 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (max_q_len == 0 || max_q_len > total_q) max_q_len = total_q;
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
-  // Q4KV_PREFILL_PATH=mma in the environment keeps the register-level mma.sync kernel for shapes both cover.
-  static const bool force_mma = [] { const char* v = std::getenv("Q4KV_PREFILL_PATH"); return v && v[0] == 'm'; }();
-  // same rule as in q4kv_decode_attention: sharp softmax scales take the kernel that multiplies the codes exactly
-  const bool usual_scale = softmax_scale > 0.f && softmax_scale * softmax_scale * (float)spec->d_qk <= 4.f;
   cudaError_t e;
-  if (prefill_umma_supported(y) && usual_scale && !force_mma)
+  if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale))
     e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                             out_dtype, lse, status_flags, (cudaStream_t)stream);
   else if (prefill_mma_supported(y))

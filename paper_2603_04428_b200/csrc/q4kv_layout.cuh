@@ -42,6 +42,10 @@ constexpr int kBlockTokens = 256;
 constexpr int kGroup = 64;
 constexpr int kChunkTokens = 32;
 constexpr int kChunksPerBlock = kBlockTokens / kChunkTokens;
+// Head of every decode workspace: arrival counters of the split merge, one per (agent, KV head) pair, at zero
+// between calls.  Its size does not depend on the call, so calls of any shape can share one workspace.
+constexpr size_t kWorkspaceHeaderBytes = Q4KV_WORKSPACE_HEADER_BYTES;
+constexpr int kMaxTicketPairs = (int)(kWorkspaceHeaderBytes / sizeof(int32_t));
 
 struct Layout {
   int L, Hq, Hkv, D, Dv, G, Gv, alias, n_rep;
@@ -125,7 +129,7 @@ cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_bl
 // tensor-core decode path (GQA shapes with d_qk = d_v in {128, 256}, at most 4 query heads per KV head)
 bool decode_mma_supported(const Layout& y);
 bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks);
-bool pdl_enabled();
+int sm_count();   // SMs of the current device (148 when no device can be asked)
 size_t decode_mma_workspace_bytes(const Layout& y, int n_agents);
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,

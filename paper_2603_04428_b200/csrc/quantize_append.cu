@@ -167,7 +167,7 @@ cudaError_t launch_m(const Layout& y, uint8_t* pool, int n_blocks, int layer, co
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, quantize_append_kernel<M>, y, pool, n_blocks, layer, b.n_agents, b.max_blocks,
                             b.block_tables, pos, new_offs, k_new, v_new, flags);
 }

@@ -23,8 +23,8 @@ def bf16_dev(bits: np.ndarray) -> torch.Tensor:
 
 class DeviceCache:
     def __init__(self, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k, n_blocks, block_tables: np.ndarray,
-                 fill_byte: int | None = 0xFF):
-        self.spec = B.Spec.make(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k)
+                 fill_byte: int | None = 0xFF, exact_products: bool = False):
+        self.spec = B.Spec.make(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k, exact_products)
         self.n_blocks = int(n_blocks)
         nbytes = B.q4kv_pool_bytes(self.spec, self.n_blocks)
         assert nbytes > 0, "unsupported spec"

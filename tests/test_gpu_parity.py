@@ -51,20 +51,25 @@ def assert_lse_close(gpu, ref, what=""):
 class Pair:
     """The same cache on both sides: an oracle pool and a device pool behind one block table."""
 
-    def __init__(self, H, spec_args, lens, seed, spare_blocks=3, extra_tokens=0, gain=1.0):
+    def __init__(self, H, spec_args, lens, seed, spare_blocks=3, extra_tokens=0, gain=1.0, outlier_frac=0.0,
+                 exact_products=False):
         L, Hq, Hkv, D, Dv, alias = spec_args
-        self.H, self.lens, self.seed, self.gain = H, list(lens), seed, gain
+        self.H, self.lens, self.seed, self.gain, self.outlier_frac = H, list(lens), seed, gain, outlier_frac
         self.ospec = O.Spec(L, Hq, Hkv, D, Dv, alias)
         need = sum(-(-(n + extra_tokens) // 256) for n in lens)
         self.n_blocks = need + spare_blocks
         self.tabs = synth.block_tables(seed, 99, lens, self.n_blocks, extra_tokens=extra_tokens)
         self.opool = O.Pool(self.ospec, self.n_blocks, fill=0xFFFFFFFF)
-        self.dc = H.DeviceCache(L, Hq, Hkv, D, Dv, alias, self.n_blocks, self.tabs)
+        self.dc = H.DeviceCache(L, Hq, Hkv, D, Dv, alias, self.n_blocks, self.tabs, exact_products=exact_products)
 
     def kv(self, layer, agent, n):
         s = self.ospec
-        k = synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 1, n, s.n_kv_heads, s.d_qk)
-        v = None if s.v_aliases_k else synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 2, n, s.n_kv_heads, s.d_v)
+        ko = vo = None
+        if self.outlier_frac > 0:      # the recipe of the Llama-shaped configuration: a few channels carry 8x the values
+            ko = synth.outlier_channels(self.seed, 100 + layer, s.n_kv_heads, s.d_qk, self.outlier_frac)
+            vo = synth.outlier_channels(self.seed, 200 + layer, s.n_kv_heads, s.d_v, self.outlier_frac)
+        k = synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 1, n, s.n_kv_heads, s.d_qk, ko)
+        v = None if s.v_aliases_k else synth.kv_bf16(self.seed, 1000 * layer + 10 * agent + 2, n, s.n_kv_heads, s.d_v, vo)
         if self.gain != 1.0:
             k = synth.f32_to_bf16_bits(f32(k) * np.float32(self.gain))
             v = None if v is None else synth.f32_to_bf16_bits(f32(v) * np.float32(self.gain))
@@ -434,6 +439,130 @@ def test_update_and_fetch_in_one_launch(H, name, lens, window):
     assert p.dc.read_flags() == 0
 
 
+
+# ---- decode: head-group sizes, routes and workspace reuse that the cases above do not reach ------
+@pytest.mark.parametrize("spec_args,lens,window", [
+    ((1, 2, 2, 128, 128, False), [700, 33, 1000], 0),        # one query head per KV head
+    ((1, 6, 2, 128, 128, False), [700, 33, 1000], 0),        # three: the fourth score row is absent
+    ((1, 6, 2, 128, 128, False), [700, 33, 1000], 200),
+    ((1, 3, 1, 256, 256, False), [1500, 41], 0),
+    ((1, 2, 2, 256, 256, False), [1500, 41], 1024),
+    ((1, 16, 2, 128, 128, False), [700, 300], 0),            # eight: beyond the tensor-core kernel, shape-agnostic path
+    ((1, 16, 2, 128, 128, False), [700, 300], 100),
+])
+def test_decode_query_heads_per_kv_head(H, spec_args, lens, window):
+    p = Pair(H, spec_args, lens, seed=41).fill()
+    q = p.q(7, len(lens))
+    scale = 1.0 / math.sqrt(spec_args[3])
+    ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, window, f32(q), scale)
+    out = torch.full((len(lens), spec_args[1], spec_args[4]), float("nan"), device="cuda")
+    out, lse = p.dc.decode(0, lens, window, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    assert p.dc.read_flags() == 0
+
+
+@pytest.mark.parametrize("window", [0, 150])
+def test_decode_latent_cache_at_a_sharp_scale_takes_the_exact_kernel(H, window):
+    """scale^2 * d_qk > 4 on the V-aliasing cache: routed to the kernel that keeps the values exact."""
+    lens = [600, 70, 257]
+    p = Pair(H, SPECS["mla"], lens, seed=42).fill()
+    q = p.q(7, len(lens))
+    scale = 0.1
+    assert scale * scale * 576 > 4
+    ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, window, f32(q), scale)
+    out, lse = p.dc.decode(0, lens, window, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    assert p.dc.read_flags() == 0
+
+
+def max_dequantized_magnitude(p, layer):
+    m = 0.0
+    for a, n in enumerate(p.lens):
+        K, V = O.gather_dequant(p.opool, layer, p.tabs[a], 0, n, 0)
+        m = max(m, float(np.abs(K).max()), float(np.abs(V).max()))
+    return m
+
+
+def tile_kernel_bound(p, layer, q_bits, scale):
+    """The bound include/q4kv.h states for the kernels that round every dequantized value once to binary16:
+    2^-10 * M * (1 + softmax_scale * max_rows ||q||_1 * M), M the largest dequantized magnitude (value and probability
+    roundings, plus what the rounded keys do to the softmax weights)."""
+    M = max_dequantized_magnitude(p, layer)
+    q1 = float(np.abs(f32(q_bits)).sum(axis=-1).max())
+    return M, 2.0 ** -10 * M * (1.0 + scale * q1 * M)
+
+
+@pytest.mark.parametrize("gain,outlier_frac", [(8.0, 0.0), (1.0, 0.01)])
+def test_latent_decode_on_large_magnitude_caches(H, gain, outlier_frac):
+    """A cache with a gain of 8, or with 1 % of the channels carrying 8x the values: with exact_products the usual
+    bound holds; without it the binary16-tile kernel stays inside the bound the header states for it."""
+    lens = [900, 40, 1]
+    q_bits = None
+    for exact in (True, False):
+        p = Pair(H, SPECS["mla"], lens, seed=43, gain=gain, outlier_frac=outlier_frac, exact_products=exact).fill()
+        q_bits = p.q(7, len(lens))
+        scale = 1.0 / math.sqrt(192)
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, 0, f32(q_bits), scale)
+        out, lse = p.dc.decode(0, lens, 0, q_bits, scale)
+        got = out.cpu().numpy().astype(np.float64)
+        if exact:
+            assert_attention_close(got, ref, "exact products")
+            assert_lse_close(lse.cpu().numpy(), lse_ref)
+        else:
+            M, bound = tile_kernel_bound(p, 0, q_bits, scale)
+            assert M >= 8.0
+            assert np.abs(got - ref).max() <= bound
+        assert p.dc.read_flags() == 0
+
+
+def test_one_workspace_serves_growing_batches_and_every_kernel(H):
+    """One workspace, allocated once for the largest call and zero-filled once: a latent-cache call, a d = 192 call
+    (shape-agnostic kernel) and GQA calls of 2 agents and then of 10 agents x 8 KV heads (more pairs than arrival
+    counters fit in 256 bytes) all run on it, each compared with the oracle, outputs pre-filled with NaN."""
+    from paper_2603_04428_b200 import binding as B
+    cases = [
+        (SPECS["mla"], [600, 70], 1.0 / math.sqrt(192)),
+        (SPECS["asym"], [400, 300], 1.0 / math.sqrt(192)),
+        ((1, 32, 8, 128, 128, False), [700, 300], 1.0 / math.sqrt(128)),
+        ((1, 32, 8, 128, 128, False), [700, 300, 260, 5000, 90, 1200, 64, 33, 2000, 513], 1.0 / math.sqrt(128)),
+        ((1, 32, 8, 128, 128, False), [700, 300], 1.0 / math.sqrt(128)),
+    ]
+    pairs = [Pair(H, sa, lens, seed=44 + i).fill() for i, (sa, lens, _) in enumerate(cases)]
+    need = max(B.q4kv_workspace_bytes(p.dc.spec, len(p.lens), p.dc.bt.max_blocks * 256, 0) for p in pairs)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for rounds in range(2):
+        for p, (sa, lens, scale) in zip(pairs, cases):
+            q = p.q(7 + rounds, len(lens))
+            ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, 0, f32(q), scale)
+            out = torch.full((len(lens), sa[1], sa[4]), float("nan"), device="cuda")
+            lse = torch.full((len(lens), sa[1]), float("nan"), device="cuda")
+            B.q4kv_decode_attention(p.dc.spec, p.dc.pool, p.dc.n_blocks, 0, p.dc.bt, H.dev(np.asarray(lens, dtype=np.int32)),
+                                    0, 0, H.bf16_dev(q), scale, out, B.OUT_F32, lse, ws, p.dc.flags)
+            assert_attention_close(out.cpu().numpy(), ref, f"{sa} {len(lens)} agents")
+            assert_lse_close(lse.cpu().numpy(), lse_ref)
+            assert p.dc.read_flags() == 0
+    assert int(ws[:B.WORKSPACE_HEADER_BYTES].max()) == 0          # every call left the arrival counters at zero
+
+
+@pytest.mark.parametrize("name", ["gqa128", "mla", "asym"])
+def test_length_beyond_the_stated_maximum_is_flagged_on_every_kernel(H, name):
+    """max_kv_len is the caller's bound on every length: an agent above it gets zeros and Q4KV_FLAG_BAD_LENGTH,
+    whichever kernel serves the spec; the other agents are unaffected."""
+    from paper_2603_04428_b200 import binding as B
+    lens = [900, 300]
+    p = Pair(H, SPECS[name], lens, seed=45).fill()
+    q = p.q(7, 2)
+    scale = 1.0 / math.sqrt(192 if name == "mla" else p.ospec.d_qk)
+    ref, _ = O.decode_attention(p.opool, 0, p.tabs, lens, 0, f32(q), scale)
+    out, lse = p.dc.decode(0, lens, 0, q, scale, max_kv_len=512)
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    assert torch.all(out[0] == 0) and torch.isneginf(lse[0]).all()
+    assert_attention_close(out[1].cpu().numpy(), ref[1])
+    p.dc.flags.zero_()
+
+
 # ---- prefill attention --------------------------------------------------------------------------
 @pytest.mark.parametrize("name,prefix,chunk,window", [
     ("gqa64", [300, 70], 40, 0),
@@ -507,6 +636,7 @@ class QuietStartPair(Pair):
     ((1, 8, 2, 128, 128, False), [3000], [200], 700, 1.0),               # the window starts many 64-key blocks in
     ((1, 8, 2, 128, 128, False), [1500, 64], [129, 64], 0, 2.0),         # the row maximum jumps by more than 2^8, late
     ((1, 8, 2, 128, 128, False), [1500, 64], [129, 64], 0, 8.0),         # a sharp scale is routed to the exact-code kernel
+    ((1, 6, 2, 128, 128, False), [700, 30], [100, 64], 0, 1.0),          # three query heads per KV head: exact-code kernel
     ((1, 4, 4, 128, 128, False), [0], [257], 0, 1.0),                    # no prefix at all: purely causal
 ])
 def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
@@ -527,6 +657,33 @@ def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
     out16, _ = p.dc.prefill(0, lens, q_offs, window, q, scale, out_dtype=B.OUT_BF16)
     assert torch.allclose(out16.float(), out.to(torch.bfloat16).float(), atol=1e-5, rtol=2.0 ** -7)
     assert p.dc.read_flags() == 0
+
+
+@pytest.mark.parametrize("gain,outlier_frac", [(8.0, 0.0), (1.0, 0.01)])
+@pytest.mark.parametrize("prefix,chunks", [([0, 40], [70, 30]), ([300], [64])])
+def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks):
+    """Rows that attend 1 to 64 keys of a cache with a gain of 8, or with 1 % of the channels carrying 8x the
+    values, return value rows almost verbatim, so a single binary16 rounding of a dequantized value (half an ulp of
+    2^-8 for magnitudes in [8, 16)) is visible.  With exact_products the usual bound holds; without it the
+    binary16-tile kernel stays inside the bound the header states for it."""
+    spec_args = (1, 8, 2, 128, 128, False)
+    lens = [p0 + c for p0, c in zip(prefix, chunks)]
+    q_offs = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
+    scale = 1.0 / math.sqrt(128)
+    for exact in (True, False):
+        p = Pair(H, spec_args, lens, seed=48, gain=gain, outlier_frac=outlier_frac, exact_products=exact).fill()
+        q = p.q(9, int(q_offs[-1]))
+        ref, lse_ref = O.prefill_attention(p.opool, 0, p.tabs, lens, q_offs, 0, f32(q), scale)
+        out, lse = p.dc.prefill(0, lens, q_offs, 0, q, scale)
+        got = out.cpu().numpy().astype(np.float64)
+        if exact:
+            assert_attention_close(got, ref, "exact products")
+            assert_lse_close(lse.cpu().numpy(), lse_ref)
+        else:
+            M, bound = tile_kernel_bound(p, 0, q, scale)
+            assert M >= 8.0
+            assert np.abs(got - ref).max() <= bound
+        assert p.dc.read_flags() == 0
 
 
 def test_prefill_bad_block_and_bad_length(H):

@@ -44,7 +44,12 @@ def test_binding_lists_the_same_symbols_and_size_queries_match_the_paper():
 def test_update_and_fetch_refuses_shapes_it_does_not_cover_before_touching_the_device():
     """q4kv_append_decode_attention is host-checked first: a head dim outside {128, 256}, and an MLA-latent spec with a
     softmax scale too sharp for its binary16-tile kernel (0.1^2 x 576 > 4), come back as Q4KV_EUNSUPPORTED without a
-    launch (the pointers below are never dereferenced; every call here is one the host checks refuse)."""
+    launch.  The pointers are placeholders that the host checks must never pass on, so the test only runs where no
+    CUDA device exists: there a regression in the order of the checks cannot launch a kernel on them."""
+    import pytest
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("placeholder pointers are only handed to the library on a host without a CUDA device")
     from paper_2603_04428_b200 import binding as B
     lib = B.lib()
     fake = ctypes.c_void_p(0x1000)                      # aligned, never read

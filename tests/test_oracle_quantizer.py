@@ -64,6 +64,52 @@ def test_pack_buffer_has_paper_size_and_zero_tail():
     assert np.all(kc[:, 44:] == 0) and np.all(kc[:, :44] == 0xFFFFFFFF)
 
 
+def test_pack_tensor_order_and_byte_offsets_are_literal():
+    """Appendix A order inside one persisted block: K codes, K scales, K biases, V codes, V scales, V biases, each
+    [Hkv][256][...] row-major.  Every tensor carries its own sentinel, and the offsets below are typed out for
+    Hkv 2, d_qk 128, d_v 64: K codes 2*256*64 = 32768 B, K scales / biases 2*256*2*2 = 2048 B each, V codes
+    2*256*32 = 16384 B, V scales / biases 2*256*1*2 = 1024 B each; block = 55296 B; two layers, two blocks each."""
+    spec = O.Spec(2, 2, 2, 128, 64)
+    pool = O.Pool(spec, 3)
+    pool.Kc[:] = 0x11111111
+    pool.Ks[:] = np.float16(2.0)       # 0x4000
+    pool.Kb[:] = np.float16(-3.0)      # 0xC200
+    pool.Vc[:] = 0x44444444
+    pool.Vs[:] = np.float16(5.0)       # 0x4500
+    pool.Vb[:] = np.float16(-6.0)      # 0xC600
+    # single elements that name their own coordinates: (layer 1, physical block 0 = logical block 1, head 1, slot 7)
+    pool.Kc[1, 0, 1, 7, 3] = 0xA1B2C3D4
+    pool.Ks[1, 0, 1, 7, 1] = np.float16(0.5)    # 0x3800
+    pool.Kb[1, 0, 1, 7, 0] = np.float16(0.25)   # 0x3400
+    pool.Vc[1, 0, 1, 7, 2] = 0x0BADF00D
+    pool.Vs[1, 0, 1, 7, 0] = np.float16(0.125)  # 0x3000
+    pool.Vb[1, 0, 1, 7, 0] = np.float16(64.0)   # 0x5400
+    buf = O.pack(pool, [2, 0], 512)
+    assert spec.block_bytes() == 55296 and buf.size == 4 * 55296
+    u16 = lambda off: int(buf[off]) | int(buf[off + 1]) << 8
+    u32 = lambda off: u16(off) | u16(off + 2) << 16
+    for blk in range(4):                                        # tensor starts inside every block
+        base = blk * 55296
+        assert u32(base) == 0x11111111 and u32(base + 32764) == 0x11111111
+        assert u16(base + 32768) == 0x4000 and u16(base + 34814) == 0x4000
+        assert u16(base + 34816) == 0xC200 and u16(base + 36862) == 0xC200
+        assert u32(base + 36864) == 0x44444444 and u32(base + 53244) == 0x44444444
+        assert u16(base + 53248) == 0x4500 and u16(base + 54270) == 0x4500
+        assert u16(base + 54272) == 0xC600 and u16(base + 55294) == 0xC600
+    base = 3 * 55296                                            # layer 1, logical block 1
+    assert u32(base + ((1 * 256 + 7) * 16 + 3) * 4) == 0xA1B2C3D4
+    assert u16(base + 32768 + ((1 * 256 + 7) * 2 + 1) * 2) == 0x3800
+    assert u16(base + 34816 + ((1 * 256 + 7) * 2 + 0) * 2) == 0x3400
+    assert u32(base + 36864 + ((1 * 256 + 7) * 8 + 2) * 4) == 0x0BADF00D
+    assert u16(base + 53248 + (1 * 256 + 7) * 2) == 0x3000
+    assert u16(base + 54272 + (1 * 256 + 7) * 2) == 0x5400
+    # and unpack puts every byte back where it came from
+    pool2 = O.Pool(spec, 3)
+    O.unpack(pool2, [1, 2], 512, buf)
+    assert pool2.Kc[1, 2, 1, 7, 3] == 0xA1B2C3D4 and pool2.Vb[1, 2, 1, 7, 0] == np.float16(64.0)
+    assert pool2.Ks[1, 2, 1, 7, 1] == np.float16(0.5) and pool2.Kb[0, 1, 0, 0, 0] == np.float16(-3.0)
+
+
 # ---- hand-worked literals -------------------------------------------------------------------
 def test_literal_unit_scale_and_ties_to_even():
     g = np.zeros(64, dtype=np.float32)
