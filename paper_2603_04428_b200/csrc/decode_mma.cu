@@ -11,13 +11,17 @@
 //     otherwise every CTA that holds a piece writes a partial (m, l, acc) record and takes a
 //     ticket, and the CTA that draws the last ticket combines the records -- one launch, no
 //     waiting on other CTAs.
-//   * A producer warp streams the CTA's chunks through a shared-memory ring with one bulk
-//     asynchronous copy per chunk (a chunk is one contiguous byte range of the pool) completing
-//     on an mbarrier.  The consumer warps run independently of one another: each claims the next
-//     chunk from a shared counter, keeps its own online-softmax state, and on leaving a segment
-//     deposits that state in shared memory; the warp that makes the deposit count complete
-//     combines the deposits and does the segment's epilogue (output, or record + ticket) while
-//     the others are already working on the next segment.  No CTA-wide barrier after start-up.
+//   * The CTA's chunks stream through a shared-memory ring with one bulk asynchronous copy per
+//     chunk (a chunk is one contiguous byte range of the pool) completing on an mbarrier.  A
+//     planner warp walks the CTA's range ahead of the copies, 32 chunks per step in lockstep, and
+//     leaves each chunk's pool offset in a small shared-memory table; between steps it polls the
+//     ring, one lane per slot but all lanes on one path, and issues the copy of the next chunk of
+//     every slot whose previous chunk has been consumed.  The
+//     consumer warps run independently of one another: each claims the next chunk from a shared
+//     counter, keeps its own online-softmax state, and on leaving a segment deposits that state in
+//     shared memory; the warp that makes the deposit count complete combines the deposits and does
+//     the segment's epilogue (output, or record + ticket) while the others are already working on
+//     the next segment.  No CTA-wide barrier after start-up.
 //   * Arithmetic runs on the 4-bit codes, not on dequantized values.  With x^ = c*s + b and one
 //     (s, b) per token and 64-element group,
 //         q.k_t   = sum_g [ s_tg * (sum_{d in g} q_d c_td) + b_tg * (sum_{d in g} q_d) ]
@@ -34,6 +38,8 @@
 //     the query heads and rows 4..7 repeat them; rows 4..7 go on to carry the low half of a
 //     two-term binary16 split of p*s, which makes the value product accurate to ~2^-22 at no
 //     extra MMA.
+#include <climits>
+
 #include "q4kv_layout.cuh"
 #include "quantize_core.cuh"
 
@@ -72,7 +78,17 @@ __device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: gives up after kSpinLimit tries or as soon as another warp has given up.
+__device__ inline bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_test_wait(bar, parity)) return true;        // the usual case: the chunk landed long ago (a blocking try costs more)
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u && *abort_flag) return false;
@@ -84,6 +100,9 @@ __device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* a
 __device__ inline bool spin_until_ge(volatile int* word, int want, volatile int* abort_flag) {
   for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
     if (*word >= want) return true;
+#ifdef Q4KV_SPIN_SLEEP
+    __nanosleep(Q4KV_SPIN_SLEEP);
+#endif
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -311,20 +330,35 @@ struct DecodeParams {
 
 __host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
 constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
-constexpr int kMBufs = 2;      // deposit buffers
+constexpr int kOffCap = 256;   // entries of the planner's offset table (a ring over the CTA's chunk indices)
+constexpr uint32_t kOffBad = 0xFFFFFFFFu;   // table entry of a chunk whose block id is outside the pool
+constexpr int kSmemBudget = 232448 - 2048;   // 227 KB per CTA, less the small arrays of the structure below
+
+// consumer warps per CTA.  Two warps per scheduler: the hot loop wants ~180 registers per thread at d = 128 and ~245 at
+// d = 256, and with three warps per scheduler (168 registers) what the compiler moves to local memory costs more than
+// the third warp brings, since almost no L1 is left beside the ring (measured: 78 against 71 us on 40 agents x 4096)
+#ifndef Q4KV_DECODE_WARPS_D128
+#define Q4KV_DECODE_WARPS_D128 7
+#endif
+#ifndef Q4KV_DECODE_WARPS_D256
+#define Q4KV_DECODE_WARPS_D256 7
+#endif
 
 template <int G, int NW>
 struct Smem {
   static constexpr int D = 64 * G;
   static constexpr int kChunkBytes = 32 * (D / 2 + 4 * G) * 2;
-  static constexpr int kSlots = (G == 2 ? 147456 : 110592) / kChunkBytes;   // 32 chunks at d = 128, 12 at d = 256
   static constexpr int kMergeStride = D + 8;            // acc[Dv], m, l, bias[Gv], pad
+  static constexpr int kMBufs = (G == 4 && NW > 7) ? 1 : 2;                  // deposit buffers (consecutive segments alternate)
+  static constexpr int kRingBudget = kSmemBudget - kMBufs * NW * 4 * kMergeStride * 4 - kQBufs * 2 * G * 32 * 16;
+  static constexpr int kSlots = kRingBudget / kChunkBytes < 32 ? kRingBudget / kChunkBytes : 32;   // one producer lane per slot
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
   alignas(16) float merge[kMBufs][NW][4][kMergeStride];
   alignas(16) uint4 qfrag[kQBufs][2 * G][32];           // [buffer][key word of a lane][lane = row * 4 + tid] = A registers
   float qsum[kQBufs][4][G];                             // scale_log2 * sum of the true q over each group
   float kappa[kQBufs][4];                               // scale_log2 * 2^(ex + 13)
   alignas(8) uint64_t full[kSlots];
+  uint32_t src_off[kOffCap];    // pool offset (16-byte units inside the layer) of chunk k at k % kOffCap; kOffBad: bad block id
   int released[kSlots];         // number of times each slot has been consumed (monotonic: no parity aliasing)
   int bad[kSlots];
   int q_tag[kQBufs];            // s + 1 once the query of segment s is staged in buffer s % kQBufs
@@ -334,15 +368,20 @@ struct Smem {
   int abort_flag;
 };
 
-// Online-softmax state of one warp for one segment (fragment layout, see the header comment).
+// Online-softmax state of one warp for one segment.  A lane owns two score columns (2 * tid, 2 * tid + 1 of eight:
+// columns 0..3 are the query heads, 4..7 repeat them) and, of every 32-token chunk, the four tokens 4 * g .. 4 * g + 3;
+// m, l and the bias sums are per column, partial over the lane's tokens.
 template <int G>
 struct WarpState {
-  float m, l_e, l_o, bias_e[G], bias_o[G];
+  float m[2], l_e[2], l_o[2], bias_e[2][G], bias_o[2][G];
   float o[4 * G][4];
   __device__ void reset() {
-    m = -INFINITY; l_e = 0.f; l_o = 0.f;
 #pragma unroll
-    for (int i = 0; i < G; ++i) { bias_e[i] = 0.f; bias_o[i] = 0.f; }
+    for (int c = 0; c < 2; ++c) {
+      m[c] = -INFINITY; l_e[c] = 0.f; l_o[c] = 0.f;
+#pragma unroll
+      for (int i = 0; i < G; ++i) { bias_e[c][i] = 0.f; bias_o[c][i] = 0.f; }
+    }
 #pragma unroll
     for (int i = 0; i < 4 * G; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
   }
@@ -461,143 +500,155 @@ __device__ inline void prefetch_new_token(const uint16_t* k_new, const uint16_t*
   }
 }
 
+// Transpose of an 8 x 8 matrix of 16-bit elements held one row per lane group (lane l: row l / 4, columns 2 * (l % 4)
+// and + 1): afterwards lane l holds row l / 4 of the transposed matrix.
+__device__ inline uint32_t transpose_8x8_b16(uint32_t a) {
+  uint32_t d;
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
 // One 32-token chunk against this warp's query fragments.
+//   Scores: the key codes are the A operand (16 tokens x 16 head-dim elements per product: lane (g, tid) holds the words
+//   of the tokens 4g + i, i = 0..3, so products pair the token rows (0, 1) and (2, 3)), the query the B operand (eight
+//   columns: heads 0..3 and their repeats).  A lane ends up with the scores of its four tokens for columns 2 tid and
+//   2 tid + 1.  The probabilities, multiplied by the token's value scale, are packed two columns to a register and
+//   transposed across the warp (movmatrix) into the B operand of the value product, whose A operand is the token-packed
+//   value words; columns 4..7 carry the low half of the two-term split of p * s.
 template <int G>
 __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
-                                              const uint4* qa, const float (&qs)[G], float kap,
+                                              const uint4* qb, const float (&qs)[2][G], const float (&kap)[2],
                                               uint32_t split_mask, WarpState<G>& st) {
   constexpr int D = 64 * G, Dv = D, Gv = G;
   const uint4* kc4 = reinterpret_cast<const uint4*>(chunk);
-  const uint4* ksb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2));
+  const uint8_t* ksb = chunk + 32 * (D / 2);
   const uint4* vc4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G);
-  const uint4* vsb4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G + 32 * (Dv / 2));
+  const uint8_t* vsb = chunk + 32 * (D / 2) + 128 * G + 32 * (Dv / 2);
   const bool edge = pos0 < key_lo || pos0 + 32 > key_n;
 
-  // ---- scores of the 4 key tiles: s2[i][e] for token 8*tid + 4*e + i, in log2 units ----
-  float s2[4][2];
+  // ---- scores sc[i][c] of token 4g + i for column 2 tid + c, in log2 units ----
+  float sc[4][2];
   {
-    float t[4][2];
+    float acc[2][G][4];                                  // [token-row pair][group]
 #pragma unroll
-    for (int half = 0; half < G / 2; ++half) {        // groups 2*half, 2*half+1
+    for (int pr = 0; pr < 2; ++pr)
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) { acc[pr][gi][0] = 0.f; acc[pr][gi][1] = 0.f; acc[pr][gi][2] = 0.f; acc[pr][gi][3] = 0.f; }
+#pragma unroll
+    for (int half = 0; half < G / 2; ++half) {           // groups 2*half, 2*half+1
       uint4 kw[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) kw[i] = kc4[((i * (G / 2) + half) * 8 + g) * 4 + tid];
-      float acc[4][2][4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {                     // word p = 4*half + j: group 2*half + j/2, i2 = j%2
-        const uint4 a = qa[(4 * half + j) * 32];
+      for (int j = 0; j < 4; ++j) {                      // word p = 4*half + j: group 2*half + j/2
+        const uint4 b = qb[(4 * half + j) * 32];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t w = j == 0 ? kw[i].x : j == 1 ? kw[i].y : j == 2 ? kw[i].z : kw[i].w;
-          const uint32_t wh = w >> 8;
-          if ((j & 1) == 0) mma_f16_rows8_first(acc[i][j >> 1], a.x, a.y, w & kMaskLo, w & kMaskHi);
-          else mma_f16_rows8(acc[i][j >> 1], a.x, a.y, w & kMaskLo, w & kMaskHi);
-          mma_f16_rows8(acc[i][j >> 1], a.z, a.w, wh & kMaskLo, wh & kMaskHi);
-        }
-      }
-      // scale of the two tokens this lane owns in each tile
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if (G == 2) {
-          const uint4 sb = ksb4[i * 4 + tid];
-          const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
-          t[i][0] = fmaf(acc[i][1][0], a1.x, acc[i][0][0] * a0.x);
-          t[i][1] = fmaf(acc[i][1][1], b1.x, acc[i][0][1] * b0.x);
-          s2[i][0] = fmaf(qs[1], a1.y, qs[0] * a0.y);
-          s2[i][1] = fmaf(qs[1], b1.y, qs[0] * b0.y);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const uint4 sb = ksb4[(i * 4 + tid) * 2 + e];
-            const float2 f0 = h2_to_f2(half == 0 ? sb.x : sb.z), f1 = h2_to_f2(half == 0 ? sb.y : sb.w);
-            const float tt = fmaf(acc[i][1][e], f1.x, acc[i][0][e] * f0.x);
-            const float uu = fmaf(qs[2 * half + 1], f1.y, qs[2 * half] * f0.y);
-            t[i][e] = half == 0 ? tt : t[i][e] + tt;
-            s2[i][e] = half == 0 ? uu : s2[i][e] + uu;
-          }
+        for (int pr = 0; pr < 2; ++pr) {
+          const uint4 &k0 = kw[2 * pr], &k1 = kw[2 * pr + 1];
+          const uint32_t w0 = j == 0 ? k0.x : j == 1 ? k0.y : j == 2 ? k0.z : k0.w;
+          const uint32_t w1 = j == 0 ? k1.x : j == 1 ? k1.y : j == 2 ? k1.z : k1.w;
+          const uint32_t h0 = w0 >> 8, h1 = w1 >> 8;
+          float (&a)[4] = acc[pr][2 * half + (j >> 1)];
+          mma_f16(a, w0 & kMaskLo, w1 & kMaskLo, w0 & kMaskHi, w1 & kMaskHi, b.x, b.y);
+          mma_f16(a, h0 & kMaskLo, h1 & kMaskLo, h0 & kMaskHi, h1 & kMaskHi, b.z, b.w);
         }
       }
     }
-    // rows g and g + 4 carry the same head, so both lanes hold its score
+    // the token's scale meets the integer dot products, its bias the per-group query sums
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i) {
+      float ks[G], kb[G];
+      if (G == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(ksb + (i * 8 + g) * 8);
+        const float2 f0 = h2_to_f2(v.x), f1 = h2_to_f2(v.y);
+        ks[0] = f0.x; kb[0] = f0.y; ks[1] = f1.x; kb[1] = f1.y;
+      } else {
+        const uint4 v = *reinterpret_cast<const uint4*>(ksb + (i * 8 + g) * 16);
+        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int e = 0; e < 2; ++e) s2[i][e] = fmaf(kap, t[i][e], s2[i][e]);
+        for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(u[gi]); ks[gi] = f.x; kb[gi] = f.y; }
+      }
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float t = acc[i >> 1][0][2 * (i & 1) + c] * ks[0], u = qs[c][0] * kb[0];
+#pragma unroll
+        for (int gi = 1; gi < G; ++gi) { t = fmaf(acc[i >> 1][gi][2 * (i & 1) + c], ks[gi], t); u = fmaf(qs[c][gi], kb[gi], u); }
+        sc[i][c] = fmaf(kap[c], t, u);
+      }
+    }
   }
   if (edge) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int pos = pos0 + 8 * tid + 4 * e + i;
-        if (pos < key_lo || pos >= key_n) s2[i][e] = -INFINITY;
-      }
+    for (int i = 0; i < 4; ++i) {
+      const int pos = pos0 + 4 * g + i;
+      if (pos < key_lo || pos >= key_n) { sc[i][0] = -INFINITY; sc[i][1] = -INFINITY; }
+    }
   }
   // ---- online softmax over the chunk ----
-  float cm = fmaxf(fmaxf(fmaxf(s2[0][0], s2[0][1]), fmaxf(s2[1][0], s2[1][1])),
-                   fmaxf(fmaxf(s2[2][0], s2[2][1]), fmaxf(s2[3][0], s2[3][1])));
-  cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-  cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-  float m_new = fmaxf(st.m, cm);
-  if (m_new == -INFINITY) m_new = 0.f;
-  const float corr = fast_exp2(st.m - m_new);
-  st.m = m_new;
-  float p[4][2];
+  float p[4][2], corr[2];
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    float cm = fmaxf(fmaxf(sc[0][c], sc[1][c]), fmaxf(sc[2][c], sc[3][c]));
+    cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 4));
+    cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 8));
+    cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));
+    float m_new = fmaxf(st.m[c], cm);
+    if (m_new == -INFINITY) m_new = 0.f;
+    corr[c] = fast_exp2(st.m[c] - m_new);
+    st.m[c] = m_new;
+    p[0][c] = fast_exp2(sc[0][c] - m_new);
+    p[1][c] = fast_exp2(sc[1][c] - (m_new + 4.f));       // odd token rows: p / 16 (their value codes carry a factor 16)
+    p[2][c] = fast_exp2(sc[2][c] - m_new);
+    p[3][c] = fast_exp2(sc[3][c] - (m_new + 4.f));
+    st.l_e[c] = fmaf(st.l_e[c], corr[c], p[0][c] + p[2][c]);
+    st.l_o[c] = fmaf(st.l_o[c], corr[c], p[1][c] + p[3][c]);
+  }
+  // rescale the accumulators when any head's running maximum moved (the lane owns the same two columns there)
+  if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int gi = 0; gi < Gv; ++gi) { st.bias_e[c][gi] *= corr[c]; st.bias_o[c][gi] *= corr[c]; }
+#pragma unroll
+    for (int mt = 0; mt < Dv / 16; ++mt) { st.o[mt][0] *= corr[0]; st.o[mt][1] *= corr[1]; st.o[mt][2] *= corr[0]; st.o[mt][3] *= corr[1]; }
+  }
+  // ---- p * s_v per group as two-term binary16 (columns 0..3: high part, columns 4..7: low part), transposed into
+  // the B operand of the value product: bfr[group][token row] = half2(tokens 8 tid + i, 8 tid + 4 + i) of column g ----
+  uint32_t bfr[Gv][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float off = (i & 1) ? m_new + 4.f : m_new;     // odd tiles: p / 16 (their value codes carry a factor 16)
-    p[i][0] = fast_exp2(s2[i][0] - off);
-    p[i][1] = fast_exp2(s2[i][1] - off);
-  }
-  st.l_e = fmaf(st.l_e, corr, (p[0][0] + p[0][1]) + (p[2][0] + p[2][1]));
-  st.l_o = fmaf(st.l_o, corr, (p[1][0] + p[1][1]) + (p[3][0] + p[3][1]));
-  // rescale the accumulators when any head's running maximum moved
-  if (__any_sync(0xffffffffu, corr != 1.f)) {
-#pragma unroll
-    for (int gi = 0; gi < Gv; ++gi) { st.bias_e[gi] *= corr; st.bias_o[gi] *= corr; }
-    const float c0 = __shfl_sync(0xffffffffu, corr, ((2 * tid) & 3) * 4);
-    const float c1 = __shfl_sync(0xffffffffu, corr, ((2 * tid + 1) & 3) * 4);
-#pragma unroll
-    for (int mt = 0; mt < Dv / 16; ++mt) { st.o[mt][0] *= c0; st.o[mt][1] *= c1; st.o[mt][2] *= c0; st.o[mt][3] *= c1; }
-  }
-  // ---- p * s_v per group as two-term binary16 (rows 0..3: high part, rows 4..7: low part) ----
-  uint32_t bfr[Gv][4];                                  // [group][tile] = half2(token e=0, token e=1)
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float vs[2][Gv], vb[2][Gv];
+    float vs[Gv], vb[Gv];
     if (G == 2) {
-      const uint4 sb = vsb4[i * 4 + tid];
-      const float2 a0 = h2_to_f2(sb.x), a1 = h2_to_f2(sb.y), b0 = h2_to_f2(sb.z), b1 = h2_to_f2(sb.w);
-      vs[0][0] = a0.x; vb[0][0] = a0.y; vs[0][1] = a1.x; vb[0][1] = a1.y;
-      vs[1][0] = b0.x; vb[1][0] = b0.y; vs[1][1] = b1.x; vb[1][1] = b1.y;
+      const uint2 v = *reinterpret_cast<const uint2*>(vsb + (i * 8 + g) * 8);
+      const float2 f0 = h2_to_f2(v.x), f1 = h2_to_f2(v.y);
+      vs[0] = f0.x; vb[0] = f0.y; vs[1] = f1.x; vb[1] = f1.y;
     } else {
+      const uint4 v = *reinterpret_cast<const uint4*>(vsb + (i * 8 + g) * 16);
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const uint4 sb = vsb4[(i * 4 + tid) * 2 + e];
-        const uint32_t v[4] = {sb.x, sb.y, sb.z, sb.w};
-#pragma unroll
-        for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(v[gi]); vs[e][gi] = f.x; vb[e][gi] = f.y; }
-      }
+      for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(u[gi]); vs[gi] = f.x; vb[gi] = f.y; }
     }
     if (edge) {
+      const int pos = pos0 + 4 * g + i;
+      if (pos < key_lo || pos >= key_n) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int pos = pos0 + 8 * tid + 4 * e + i;
-        if (pos < key_lo || pos >= key_n) {
-#pragma unroll
-          for (int gi = 0; gi < Gv; ++gi) { vs[e][gi] = 0.f; vb[e][gi] = 0.f; }
-        }
+        for (int gi = 0; gi < Gv; ++gi) { vs[gi] = 0.f; vb[gi] = 0.f; }
       }
     }
 #pragma unroll
     for (int gi = 0; gi < Gv; ++gi) {
-      const float x0 = p[i][0] * vs[0][gi], x1 = p[i][1] * vs[1][gi];
-      // rows 0..3: trunc16(x); rows 4..7: trunc16(x - trunc11bits(x)) -- the binary16 conversion truncates
+      const float x0 = p[i][0] * vs[gi], x1 = p[i][1] * vs[gi];
+      // columns 0..3: trunc16(x); columns 4..7: trunc16(x - trunc11bits(x)) -- the binary16 conversion truncates
       const float r0 = x0 - __uint_as_float(__float_as_uint(x0) & split_mask);
       const float r1 = x1 - __uint_as_float(__float_as_uint(x1) & split_mask);
-      bfr[gi][i] = f32x2_to_h2_rz(r0, r1);
-      if (i & 1) st.bias_o[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], st.bias_o[gi]));
-      else st.bias_e[gi] = fmaf(p[i][0], vb[0][gi], fmaf(p[i][1], vb[1][gi], st.bias_e[gi]));
+      bfr[gi][i] = transpose_8x8_b16(f32x2_to_h2_rz(r0, r1));
+      if (i & 1) {
+        st.bias_o[0][gi] = fmaf(p[i][0], vb[gi], st.bias_o[0][gi]);
+        st.bias_o[1][gi] = fmaf(p[i][1], vb[gi], st.bias_o[1][gi]);
+      } else {
+        st.bias_e[0][gi] = fmaf(p[i][0], vb[gi], st.bias_e[0][gi]);
+        st.bias_e[1][gi] = fmaf(p[i][1], vb[gi], st.bias_e[1][gi]);
+      }
     }
   }
   // ---- P.V on the codes: 16 value rows x 8 columns (heads hi|lo) x 32 tokens per tile pair ----
@@ -627,16 +678,17 @@ __device__ inline void store_out(const DecodeParams& P, size_t index, float v) {
 // the NW deposits; a pair that lies wholly inside this CTA is normalised and written out, otherwise
 // the combination becomes this CTA's partial record and the warp takes a ticket -- the CTA whose
 // ticket is the pair's last combines all records of the pair.  Each lane owns 4 consecutive output
-// elements (per 128), so every access is a 16-byte one, and the loads of a step are all issued
-// before the first is used (the records sit in L2, a microsecond away).
+// elements (per 128), so every access is a 16-byte one.  Deposits and records are walked in loops with a
+// few loads in flight and running sums in registers: the register need does not grow with the number of
+// warps or records.
 template <int G, int NW>
-__device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilogues_word, int use, const DecodeParams& P,
+__device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* epilogues_word, int use, const DecodeParams& P,
                                               const Segment& seg, int cta, const Partition& part, int lane) {
   constexpr int Dv = 64 * G, V = Dv / 128;
   constexpr int kStride = Dv + 8;
+  static_assert(NW <= 32, "one lane per deposit in the weight pass");
   const Layout& y = P.y;
   const int n_rep = y.n_rep;
-  auto mrg = [&](int w, int h) { return merge_buf + ((size_t)w * 4 + h) * kStride; };
   const int pair = seg.a * y.Hkv + seg.hk;
   const bool whole = seg.c0 == seg.cf && seg.c1 == seg.cf + seg.nc;
   const size_t row0 = (size_t)seg.a * y.Hq + (size_t)seg.hk * n_rep;
@@ -652,46 +704,42 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
     }
   };
   for (int h = 0; h < n_rep; ++h) {
-    float mw[NW], lw[NW];
+    // weights: lane w looks at deposit w
+    const float* mine = merge_buf + ((size_t)(lane < NW ? lane : 0) * 4 + h) * kStride;
+    const float2 ml = *reinterpret_cast<const float2*>(mine + Dv);
+    const float mw = lane < NW ? ml.x : -INFINITY, lw = lane < NW ? ml.y : 0.f;
+    float M = mw;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) { const float2 t = *reinterpret_cast<const float2*>(mrg(w, h) + Dv); mw[w] = t.x; lw[w] = t.y; }
-    float4 x[V][NW];
-    float bs[V][NW];
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    const float wgt = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
+    float Lsum = wgt * lw;
 #pragma unroll
-    for (int v = 0; v < V; ++v)
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        x[v][w] = *reinterpret_cast<const float4*>(mrg(w, h) + 128 * v + 4 * lane);
-        bs[v][w] = mrg(w, h)[Dv + 2 + ((128 * v + 4 * lane) >> 6)];
-      }
-    float M = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
-    float wgt[NW], Lsum = 0.f;
-    bool bad = false;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      if (lw[w] < 0.f) bad = true;
-      wgt[w] = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);
-      Lsum = fmaf(wgt[w], lw[w], Lsum);
-    }
+    for (int o = 16; o > 0; o >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, o);
+    const bool bad = __any_sync(0xffffffffu, lw < 0.f);
     if (bad) Lsum = 0.f;
     const float inv = whole ? (Lsum > 0.f ? 1.f / Lsum : 0.f) : 1.f;
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int w = 0; w < NW; ++w) {
+      const float ww = __shfl_sync(0xffffffffu, wgt, w);
+      const bool on = ww != 0.f;                         // an empty deposit holds stale bytes
+      const float* dep = merge_buf + ((size_t)w * 4 + h) * kStride;
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        const float4 x = *reinterpret_cast<const float4*>(dep + 128 * v + 4 * lane);
+        const float bs = dep[Dv + 2 + ((128 * v + 4 * lane) >> 6)];
+        acc[v].x = fmaf(ww, on ? x.x + bs : 0.f, acc[v].x); acc[v].y = fmaf(ww, on ? x.y + bs : 0.f, acc[v].y);
+        acc[v].z = fmaf(ww, on ? x.z + bs : 0.f, acc[v].z); acc[v].w = fmaf(ww, on ? x.w + bs : 0.f, acc[v].w);
+      }
+    }
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        const bool on = wgt[w] != 0.f;                 // an empty deposit holds stale bytes
-        acc.x = fmaf(wgt[w], on ? x[v][w].x + bs[v][w] : 0.f, acc.x);
-        acc.y = fmaf(wgt[w], on ? x[v][w].y + bs[v][w] : 0.f, acc.y);
-        acc.z = fmaf(wgt[w], on ? x[v][w].z + bs[v][w] : 0.f, acc.z);
-        acc.w = fmaf(wgt[w], on ? x[v][w].w + bs[v][w] : 0.f, acc.w);
-      }
-      acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      acc[v].x *= inv; acc[v].y *= inv; acc[v].z *= inv; acc[v].w *= inv;
       const int d = 128 * v + 4 * lane;
-      if (whole) store4(h, d, acc);
-      else *reinterpret_cast<float4*>(rec + (size_t)h * kRecStride(Dv) + d) = acc;
+      if (whole) store4(h, d, acc[v]);
+      else *reinterpret_cast<float4*>(rec + (size_t)h * kRecStride(Dv) + d) = acc[v];
     }
     if (lane == 0) {
       if (whole) { if (P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY; }
@@ -719,8 +767,9 @@ __device__ __noinline__ void segment_epilogue(const float* merge_buf, int* epilo
   __threadfence();
   const int R = c_last - c_first + 1;
   const float* base = P.partials + (size_t)(pair + c_first) * rstride;
-  // The first batch of record loads is issued before the (m, l) pass, so that both travel together.
-  constexpr int RB = G == 2 ? 6 : 3;
+  // The records sit in L2, a microsecond away: all heads travel together, and the first batch of record loads is issued
+  // before the (m, l) pass, so that a pair with few records costs two round trips in all.
+  constexpr int RB = G == 2 ? 5 : 2;
   float mr[RB][4];
   float4 xv[RB][4][V];
   auto load_batch = [&](int rb) {
@@ -802,7 +851,8 @@ template <int G, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __grid_constant__ DecodeParams P) {
   constexpr int D = 64 * G, Dv = D, Gv = G;
   using S = Smem<G, NW>;
-  constexpr int kSlots = S::kSlots, kChunkBytes = S::kChunkBytes;
+  constexpr int kSlots = S::kSlots, kChunkBytes = S::kChunkBytes, kMBufs = S::kMBufs;
+  static_assert(kSlots >= NW + 4, "the ring must hold the chunks in work and a few in flight");
   extern __shared__ __align__(128) uint8_t smem_raw[];
   S& sm = *reinterpret_cast<S*>(smem_raw);
 
@@ -833,49 +883,81 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, rs);
   Segment seg;
 
-  // =============================== producer warp ===============================================
+  const uint8_t* layer_base = P.pool + (uint64_t)P.layer * y.layer_bytes;
+  // hand ring slot `slot` to the chunk whose table entry is `off`
+  auto issue_copy = [&](int slot, uint32_t off) {
+    if (off == kOffBad) {
+      sm.bad[slot] = 1;
+      mbar_arrive(&sm.full[slot]);
+    } else {
+      sm.bad[slot] = 0;
+      mbar_arrive_expect_tx(&sm.full[slot], kChunkBytes);
+      bulk_load(sm.ring + (size_t)slot * kChunkBytes, layer_base + (uint64_t)off * 16u, kChunkBytes, &sm.full[slot]);
+    }
+  };
+
+  // =============================== planner warp ================================================
   if (warp == NW) {
-    // Lane s owns ring slot s (kSlots <= 32): it issues the chunks k = s, s + kSlots, ... in order, each
-    // once the slot's previous chunk has been consumed, so the copies of all slots are issued in parallel.
-    static_assert(kSlots <= 32, "one producer lane per ring slot");
-    if (lane >= kSlots) return;
-    {
-      // the block-table entry of this lane's first chunk is fetched towards the SM while the preceding kernel drains
-      // (the tables, like the lengths, are inputs that no kernel writes)
-      Walker w2 = wk;
-      Segment s2;
-      while (w2.next(s2)) {
-        const int k = s2.k0 + (lane - s2.k0 % kSlots + kSlots) % kSlots;
-        if (k >= s2.k0 + (s2.c1 - s2.c0)) continue;
-        const int c = s2.c1 - 1 - (k - s2.k0);
-        asm volatile("prefetch.global.L1 [%0];" ::"l"(P.tables + (size_t)s2.a * P.max_blocks + (c >> 3)) : "memory");
+    // Planning step: 32 chunks, one per lane: block-table entry -> pool offset -> table entry k % kOffCap.  Issue
+    // step: lane s owns ring slot s and the chunks s, s + kSlots, ...; it copies its next chunk once the slot's
+    // previous chunk has been consumed and the chunk has its table entry.  All lanes follow one path.  Lengths and
+    // block tables are inputs that no kernel writes, so the first planning steps run while the preceding kernel drains;
+    // the pool is read only after it.
+    static_assert(kSlots <= 32 && kOffCap >= 2 * 32 + kSlots, "table ring: a step of entries ahead of every reader");
+    bool waited = false, bad_block = false, more = wk.next(seg);
+    int kb = 0;                              // chunks of `seg` already planned
+    int planned = 0;                         // chunks of the CTA that have their table entry
+    int next_k = lane < kSlots ? lane : INT_MAX, round = 0;   // this lane's next chunk and its round in the slot
+    const volatile int* my_released = &sm.released[lane < kSlots ? lane : 0];
+    uint32_t idle = 0;
+    for (;;) {
+      // ---- plan as far as the table allows: entries below every lane's next chunk are dead ----
+      if (more) {
+        int lo = next_k;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        while (more && planned + 32 <= lo + kOffCap) {
+          const int cnt = seg.c1 - seg.c0;
+          if (kb + lane < cnt) {
+            const int c = seg.c1 - 1 - (kb + lane);   // a segment is walked from its last chunk to its first (see the consumers)
+            const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
+            uint32_t off = kOffBad;
+            if (blk >= 0 && blk < P.n_blocks)
+              off = (uint32_t)(((uint64_t)blk * y.block_bytes + (uint64_t)seg.hk * y.head_block_bytes +
+                                (uint64_t)(c & 7) * kChunkBytes) >> 4);
+            else
+              bad_block = true;
+            sm.src_off[(seg.k0 + kb + lane) % kOffCap] = off;
+          }
+          kb += 32;
+          if (kb >= cnt) { planned = seg.k0 + cnt; kb = 0; more = wk.next(seg); } else { planned = seg.k0 + kb; }
+        }
+        __syncwarp();
+      }
+      if (!waited) { grid_dependency_wait(); waited = true; }
+      // ---- issue: a short polling loop, left from time to time to plan further ----
+      bool any_left = true;
+      for (int it = 0; it < 64 && any_left; ++it) {
+        const bool can = next_k < planned && *my_released >= round;
+        if (can) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the consumer's reads and patches of the slot come first
+          issue_copy(lane, sm.src_off[next_k % kOffCap]);
+          next_k += kSlots;
+          ++round;
+        }
+        any_left = __any_sync(0xffffffffu, next_k < n_chunks);
+        if (__any_sync(0xffffffffu, can)) { idle = 0; continue; }
+        if (more && __all_sync(0xffffffffu, next_k >= planned)) break;   // nothing to issue before more is planned
+        ++idle;
+        __nanosleep(200);
+      }
+      if (!any_left) break;                  // every chunk has been issued
+      if (idle > (kSpinLimit >> 2) || *(volatile int*)&sm.abort_flag) {
+        if (lane == 0) { sm.abort_flag = 1; raise_flag(P.flags, Q4KV_FLAG_INTERNAL); }
         break;
       }
     }
-    grid_dependency_wait();                 // the pool may still be being written by the preceding kernel
-    while (wk.next(seg)) {
-      const int k_end = seg.k0 + (seg.c1 - seg.c0);
-      for (int k = seg.k0 + (lane - seg.k0 % kSlots + kSlots) % kSlots; k < k_end; k += kSlots) {
-        const int c = seg.c1 - 1 - (k - seg.k0);     // a segment is walked from its last chunk to its first (see the consumers)
-        const int round = k / kSlots;        // k % kSlots == lane
-        if (!spin_until_ge(&sm.released[lane], round, &sm.abort_flag)) {
-          raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
-          return;
-        }
-        const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
-        if (blk < 0 || blk >= P.n_blocks) {
-          sm.bad[lane] = 1;
-          raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
-          mbar_arrive(&sm.full[lane]);
-        } else {
-          sm.bad[lane] = 0;
-          mbar_arrive_expect_tx(&sm.full[lane], kChunkBytes);
-          bulk_load(sm.ring + (size_t)lane * kChunkBytes,
-                    head_block(P.pool, y, P.layer, blk, seg.hk) + (size_t)(c & 7) * kChunkBytes, kChunkBytes,
-                    &sm.full[lane]);
-        }
-      }
-    }
+    if (bad_block) raise_flag(P.flags, Q4KV_FLAG_BAD_BLOCK);
     return;
   }
 
@@ -884,9 +966,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   // the preceding kernels of the stream until they have completed.
   grid_dependency_wait();
   const int g = lane >> 2, tid = lane & 3;
-  const int hrow = g & 3;                              // query head (within the KV head) of this lane's score row
-  const bool live = hrow < n_rep;
-  const uint32_t split_mask = g >= 4 ? 0xFFFFE000u : 0u;   // rows 4..7 carry p*s minus its binary16 truncation
+  // this lane's two score columns 2 tid, 2 tid + 1 of eight: columns 0..3 are the query heads of the KV head, 4..7
+  // repeat them and carry p*s minus its binary16 truncation
+  const int hcol[2] = {(2 * tid) & 3, (2 * tid + 1) & 3};
+  const bool live[2] = {hcol[0] < n_rep, hcol[1] < n_rep};
+  const uint32_t split_mask = tid >= 2 ? 0xFFFFE000u : 0u;
 
   // agents without any key (kv_len == 0 or a rejected length): zeros, lse = -inf
   for (int a = cta * NW + warp; a < P.n_agents; a += gridDim.x * NW) {
@@ -915,7 +999,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   int cur = -1;                 // index of the segment `seg` describes (-1: none yet)
   bool have_seg = false;        // this warp holds state for segment `cur`
   const uint4* qa = nullptr;    // this lane's A registers of the segment's query, in shared memory
-  float qs[G], kap = 0.f;
+  float qs[2][G], kap[2] = {0.f, 0.f};
   WarpState<G> st;
   st.reset();
 
@@ -927,22 +1011,29 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     if (!aborted && !spin_until_ge(&sm.epilogues[b], use, &sm.abort_flag)) aborted = true;
     float (*mg)[S::kMergeStride] = sm.merge[b][warp];
     if (real) {
-      float l = st.l_e + 16.f * st.l_o;
-      l += __shfl_xor_sync(0xffffffffu, l, 1);
-      l += __shfl_xor_sync(0xffffffffu, l, 2);
-      float bias[Gv];
+      // sums over the lane's tokens -> sums over the chunk's tokens (the eight lanes of equal tid)
 #pragma unroll
-      for (int gi = 0; gi < Gv; ++gi) {
-        float bb = st.bias_e[gi] + 16.f * st.bias_o[gi];
-        bb += __shfl_xor_sync(0xffffffffu, bb, 1);
-        bb += __shfl_xor_sync(0xffffffffu, bb, 2);
-        bias[gi] = bb;
-      }
-      if (g < 4 && tid == 0) {
-        mg[g][Dv] = st.m;
-        mg[g][Dv + 1] = (poisoned || aborted) ? -1.f : l;
+      for (int c = 0; c < 2; ++c) {
+        float l = st.l_e[c] + 16.f * st.l_o[c];
+        l += __shfl_xor_sync(0xffffffffu, l, 4);
+        l += __shfl_xor_sync(0xffffffffu, l, 8);
+        l += __shfl_xor_sync(0xffffffffu, l, 16);
+        float bias[Gv];
 #pragma unroll
-        for (int gi = 0; gi < Gv; ++gi) mg[g][Dv + 2 + gi] = bias[gi];
+        for (int gi = 0; gi < Gv; ++gi) {
+          float bb = st.bias_e[c][gi] + 16.f * st.bias_o[c][gi];
+          bb += __shfl_xor_sync(0xffffffffu, bb, 4);
+          bb += __shfl_xor_sync(0xffffffffu, bb, 8);
+          bb += __shfl_xor_sync(0xffffffffu, bb, 16);
+          bias[gi] = bb;
+        }
+        if (g == 0 && tid < 2) {
+          float* row = mg[2 * tid + c];
+          row[Dv] = st.m[c];
+          row[Dv + 1] = (poisoned || aborted) ? -1.f : l;
+#pragma unroll
+          for (int gi = 0; gi < Gv; ++gi) row[Dv + 2 + gi] = bias[gi];
+        }
       }
       // columns 4..7 (lanes tid 2,3) hold the low-part products of heads 0..3
 #pragma unroll
@@ -967,13 +1058,17 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     segment_epilogue<G, NW>(&sm.merge[b][0][0][0], &sm.epilogues[b], use, P, seg, cta, rs.part, lane);
   };
 
+  // Chunks are claimed one ahead: the claim of the following chunk is taken before this one is worked on, so that the
+  // shared-memory atomic's latency is off the path.
   bool out_of_chunks = false;
+  int k_ahead = 0;
+  if (lane == 0) k_ahead = atomicAdd(&sm.next_chunk, 1);
   for (;;) {
     int k = 0;
     if (!out_of_chunks) {
-      if (lane == 0) k = atomicAdd(&sm.next_chunk, 1);
-      k = __shfl_sync(0xffffffffu, k, 0);
+      k = __shfl_sync(0xffffffffu, k_ahead, 0);
       out_of_chunks = k >= n_chunks;
+      if (!out_of_chunks && lane == 0) k_ahead = atomicAdd(&sm.next_chunk, 1);
     }
     // move to the segment that holds chunk k (to the end of the list when out of chunks), leaving a
     // deposit in every segment passed
@@ -1004,8 +1099,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       __threadfence_block();
       qa = &sm.qfrag[qb][0][lane];
 #pragma unroll
-      for (int gi = 0; gi < G; ++gi) qs[gi] = live ? sm.qsum[qb][hrow][gi] : 0.f;
-      kap = live ? sm.kappa[qb][hrow] : 0.f;
+      for (int c = 0; c < 2; ++c) {
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) qs[c][gi] = live[c] ? sm.qsum[qb][hcol[c]][gi] : 0.f;
+        kap[c] = live[c] ? sm.kappa[qb][hcol[c]] : 0.f;
+      }
       st.reset();
       have_seg = true;
     }
@@ -1111,7 +1209,8 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
   const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
   const int n_sm = sm_count();
   const int grid = (int)(units < n_sm ? (units < 1 ? 1 : units) : n_sm);
-  return y.G == 2 ? launch_g<2, 7>(P, grid, true, st) : launch_g<4, 7>(P, grid, true, st);
+  return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128>(P, grid, true, st)
+                  : launch_g<4, Q4KV_DECODE_WARPS_D256>(P, grid, true, st);
 }
 
 }  // namespace q4kv
