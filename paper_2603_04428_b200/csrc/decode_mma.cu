@@ -249,13 +249,26 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
   return rs;
 }
 
-// One segment: the part of pair (agent a, KV head hk) inside this CTA's unit range.
+// One segment: the part of pair (agent a, KV head hk) inside this CTA's unit range.  A segment is walked from its last
+// chunk to its first (the order does not matter to the online softmax).  With the fused append, the chunk of the agent's
+// newest position -- the pair's last chunk -- is patched by the planner warp after it has landed; it is moved a few
+// places back in the walk (to place tail_pos), so that the consumers have other chunks to work on meanwhile.
+constexpr int kTailPos = 14;
 struct Segment {
   int a, hk, c0, c1;      // logical chunk indices [c0, c1) of the agent
   int n, lo;              // key range of the agent
   int cf, nc;             // the pair's whole chunk range
   int k0;                 // running chunk counter of the CTA at c0
   uint32_t u0;            // global unit index at c0
+  int tail_pos;           // place in the walk of the chunk that receives the new token; -1: none in this segment
+  __device__ void set_tail(bool fused) {
+    const int cnt = c1 - c0;
+    tail_pos = (fused && c1 == cf + nc) ? (cnt - 1 < kTailPos ? cnt - 1 : kTailPos) : -1;
+  }
+  __device__ int chunk_at(int j) const {    // logical chunk at place j of the walk, 0 <= j < c1 - c0
+    if (tail_pos < 0 || j > tail_pos) return c1 - 1 - j;
+    return j == tail_pos ? c1 - 1 : c1 - 2 - j;
+  }
 };
 
 struct Walker {
@@ -263,11 +276,12 @@ struct Walker {
   int n_agents, Hkv, window, len_cap;
   uint32_t u, u_end;
   int k, a, hk, c;
+  bool fused;               // the launch appends one token per agent
   AgentRange r;
 
   __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int len_cap_,
-                       const RangeStart& rs) {
-    kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; len_cap = len_cap_;
+                       const RangeStart& rs, bool fused_) {
+    kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; len_cap = len_cap_; fused = fused_;
     u = rs.u_begin; u_end = rs.u_end; k = 0;
     a = rs.agent; hk = 0; c = 0;
     r.n = 0; r.lo = 0; r.cf = 0; r.nc = 0;
@@ -285,6 +299,7 @@ struct Walker {
     const uint32_t left = u_end - u;
     const int c1 = (uint32_t)(pair_end - c) <= left ? pair_end : c + (int)left;
     s.a = a; s.hk = hk; s.c0 = c; s.c1 = c1; s.n = r.n; s.lo = r.lo; s.cf = r.cf; s.nc = r.nc; s.k0 = k; s.u0 = u;
+    s.set_tail(fused);
     const int cnt = c1 - c;
     u += (uint32_t)cnt; k += cnt;
     if (c1 == pair_end) {
@@ -331,6 +346,7 @@ struct DecodeParams {
 __host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
 constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
 constexpr int kOffCap = 256;   // entries of the planner's offset table (a ring over the CTA's chunk indices)
+constexpr int kTailQ = 8;      // chunks waiting for the planner's patch (planning stops while the queue is full)
 constexpr uint32_t kOffBad = 0xFFFFFFFFu;   // table entry of a chunk whose block id is outside the pool
 constexpr int kSmemBudget = 232448 - 2048;   // 227 KB per CTA, less the small arrays of the structure below
 
@@ -360,6 +376,8 @@ struct Smem {
   alignas(8) uint64_t full[kSlots];
   uint32_t src_off[kOffCap];    // pool offset (16-byte units inside the layer) of chunk k at k % kOffCap; kOffBad: bad block id
   int released[kSlots];         // number of times each slot has been consumed (monotonic: no parity aliasing)
+  int patched[kSlots];          // round + 1 of the last chunk the planner has patched in each slot (fused append)
+  int4 tail_q[kTailQ];          // planner's queue of chunks to patch: (chunk index in the CTA, agent, KV head, token in chunk)
   int bad[kSlots];
   int q_tag[kQBufs];            // s + 1 once the query of segment s is staged in buffer s % kQBufs
   int deposits[kMBufs];         // running count of deposits into each buffer
@@ -434,10 +452,11 @@ __device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], f
   }
 }
 
-// Fused append (one new token per agent): the warp that owns the chunk holding an agent's newest position
+// Fused append (one new token per agent): the planner warp of the CTA that holds the chunk of an agent's newest position
 // quantizes that token's K and V rows (Section 3.2 quantizer, the same device function the append kernel uses) and
-// writes them into the chunk -- in shared memory for this launch, in the pool for the following ones.  Every chunk
-// is processed by exactly one warp of the grid, so nobody else reads or writes these words during the launch.
+// writes them into the chunk once it has landed -- in shared memory for this launch, in the pool for the following
+// ones -- and then lets the chunk's consumer go on.  Every chunk is held by exactly one CTA of the grid, so nobody else
+// reads or writes these words during the launch.
 // Eight consecutive lanes own one 64-element group; the 8-lane shuffles never straddle K and V (D / 8 is a multiple
 // of 16).  The value codes are token-packed: one nibble of each of the row's D words is replaced.
 template <int G>
@@ -703,47 +722,61 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
       *reinterpret_cast<float4*>(reinterpret_cast<float*>(P.out) + (row0 + h) * Dv + d) = v;
     }
   };
-  for (int h = 0; h < n_rep; ++h) {
-    // weights: lane w looks at deposit w
+  // weights of the deposits, all heads side by side: lane w looks at deposit w
+  float wgt[4], Mh[4], Lh[4];
+  bool badh[4];
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
     const float* mine = merge_buf + ((size_t)(lane < NW ? lane : 0) * 4 + h) * kStride;
     const float2 ml = *reinterpret_cast<const float2*>(mine + Dv);
-    const float mw = lane < NW ? ml.x : -INFINITY, lw = lane < NW ? ml.y : 0.f;
+    const float mw = (lane < NW && h < n_rep) ? ml.x : -INFINITY, lw = (lane < NW && h < n_rep) ? ml.y : 0.f;
     float M = mw;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    const float wgt = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
-    float Lsum = wgt * lw;
+    wgt[h] = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
+    float L = wgt[h] * lw;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, o);
-    const bool bad = __any_sync(0xffffffffu, lw < 0.f);
-    if (bad) Lsum = 0.f;
-    const float inv = whole ? (Lsum > 0.f ? 1.f / Lsum : 0.f) : 1.f;
-    float4 acc[V];
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    badh[h] = __any_sync(0xffffffffu, lw < 0.f);
+    Mh[h] = M;
+    Lh[h] = badh[h] ? 0.f : L;
+  }
+  float4 acc[4][V];
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int w = 0; w < NW; ++w) {
-      const float ww = __shfl_sync(0xffffffffu, wgt, w);
+  for (int h = 0; h < 4; ++h)
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[h][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+  for (int w = 0; w < NW; ++w) {
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const float ww = __shfl_sync(0xffffffffu, wgt[h], w);
       const bool on = ww != 0.f;                         // an empty deposit holds stale bytes
       const float* dep = merge_buf + ((size_t)w * 4 + h) * kStride;
 #pragma unroll
       for (int v = 0; v < V; ++v) {
         const float4 x = *reinterpret_cast<const float4*>(dep + 128 * v + 4 * lane);
         const float bs = dep[Dv + 2 + ((128 * v + 4 * lane) >> 6)];
-        acc[v].x = fmaf(ww, on ? x.x + bs : 0.f, acc[v].x); acc[v].y = fmaf(ww, on ? x.y + bs : 0.f, acc[v].y);
-        acc[v].z = fmaf(ww, on ? x.z + bs : 0.f, acc[v].z); acc[v].w = fmaf(ww, on ? x.w + bs : 0.f, acc[v].w);
+        acc[h][v].x = fmaf(ww, on ? x.x + bs : 0.f, acc[h][v].x); acc[h][v].y = fmaf(ww, on ? x.y + bs : 0.f, acc[h][v].y);
+        acc[h][v].z = fmaf(ww, on ? x.z + bs : 0.f, acc[h][v].z); acc[h][v].w = fmaf(ww, on ? x.w + bs : 0.f, acc[h][v].w);
       }
     }
+  }
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    if (h >= n_rep) continue;
+    const float inv = whole ? (Lh[h] > 0.f ? 1.f / Lh[h] : 0.f) : 1.f;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-      acc[v].x *= inv; acc[v].y *= inv; acc[v].z *= inv; acc[v].w *= inv;
+      float4 o = acc[h][v];
+      o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
       const int d = 128 * v + 4 * lane;
-      if (whole) store4(h, d, acc[v]);
-      else *reinterpret_cast<float4*>(rec + (size_t)h * kRecStride(Dv) + d) = acc[v];
+      if (whole) store4(h, d, o);
+      else *reinterpret_cast<float4*>(rec + (size_t)h * kRecStride(Dv) + d) = o;
     }
     if (lane == 0) {
-      if (whole) { if (P.lse) P.lse[row0 + h] = Lsum > 0.f ? (M + log2f(Lsum)) / kLog2e : -INFINITY; }
-      else *reinterpret_cast<float2*>(rec + (size_t)h * kRecStride(Dv) + Dv) = make_float2(M, bad ? -1.f : Lsum);
+      if (whole) { if (P.lse) P.lse[row0 + h] = Lh[h] > 0.f ? (Mh[h] + log2f(Lh[h])) / kLog2e : -INFINITY; }
+      else *reinterpret_cast<float2*>(rec + (size_t)h * kRecStride(Dv) + Dv) = make_float2(Mh[h], badh[h] ? -1.f : Lh[h]);
     }
   }
   // the deposit buffer can be reused from here on
@@ -808,42 +841,42 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
   }
   const bool any_bad = __any_sync(0xffffffffu, badl);
   // pass 2: weighted sum of the records, RB at a time, all heads together (nothing is stored before the end)
-  float Mh[4], Lh[4];
+  float Mr[4], Lr[4];
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
-    Mh[h] = __shfl_sync(0xffffffffu, Ml, h);
-    Lh[h] = any_bad ? 0.f : __shfl_sync(0xffffffffu, Ll, h);
+    Mr[h] = __shfl_sync(0xffffffffu, Ml, h);
+    Lr[h] = any_bad ? 0.f : __shfl_sync(0xffffffffu, Ll, h);
   }
-  float4 acc[4][V];
+  float4 racc[4][V];
 #pragma unroll
   for (int h = 0; h < 4; ++h)
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[h][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) racc[h][v] = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int rb = 0; rb < R; rb += RB) {
     if (rb > 0) load_batch(rb);
 #pragma unroll
     for (int i = 0; i < RB; ++i)
 #pragma unroll
       for (int h = 0; h < 4; ++h) {
-        const float e = (rb + i >= R || mr[i][h] == -INFINITY) ? 0.f : fast_exp2(mr[i][h] - Mh[h]);
+        const float e = (rb + i >= R || mr[i][h] == -INFINITY) ? 0.f : fast_exp2(mr[i][h] - Mr[h]);
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-          acc[h][v].x = fmaf(e, xv[i][h][v].x, acc[h][v].x); acc[h][v].y = fmaf(e, xv[i][h][v].y, acc[h][v].y);
-          acc[h][v].z = fmaf(e, xv[i][h][v].z, acc[h][v].z); acc[h][v].w = fmaf(e, xv[i][h][v].w, acc[h][v].w);
+          racc[h][v].x = fmaf(e, xv[i][h][v].x, racc[h][v].x); racc[h][v].y = fmaf(e, xv[i][h][v].y, racc[h][v].y);
+          racc[h][v].z = fmaf(e, xv[i][h][v].z, racc[h][v].z); racc[h][v].w = fmaf(e, xv[i][h][v].w, racc[h][v].w);
         }
       }
   }
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
     if (h >= n_rep) continue;
-    const float inv = Lh[h] > 0.f ? 1.f / Lh[h] : 0.f;
+    const float inv = Lr[h] > 0.f ? 1.f / Lr[h] : 0.f;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-      float4 o = acc[h][v];
+      float4 o = racc[h][v];
       o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
       store4(h, 128 * v + 4 * lane, o);
     }
-    if (lane == 0 && P.lse) P.lse[row0 + h] = Lh[h] > 0.f ? (Mh[h] + log2f(Lh[h])) / kLog2e : -INFINITY;
+    if (lane == 0 && P.lse) P.lse[row0 + h] = Lr[h] > 0.f ? (Mr[h] + log2f(Lr[h])) / kLog2e : -INFINITY;
   }
 }
 
@@ -865,7 +898,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   // rows of query heads that do not exist (n_rep < 4) are never staged: they stay zero
   for (int i = threadIdx.x; i < kQBufs * 2 * G * 32; i += blockDim.x) (&sm.qfrag[0][0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); sm.released[s] = 0; sm.bad[s] = 0; }
+    for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); sm.released[s] = 0; sm.bad[s] = 0; sm.patched[s] = 0; }
     for (int i = 0; i < kQBufs; ++i) sm.q_tag[i] = 0;
     for (int i = 0; i < kMBufs; ++i) { sm.deposits[i] = 0; sm.epilogues[i] = 0; }
     sm.next_chunk = 0;
@@ -880,7 +913,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   if (rs.any_bad && cta == 0 && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
   const int n_chunks = (int)(rs.u_end - rs.u_begin);
   Walker wk;
-  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, rs);
+  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, rs, P.k_new != nullptr);
   Segment seg;
 
   const uint8_t* layer_base = P.pool + (uint64_t)P.layer * y.layer_bytes;
@@ -905,6 +938,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     // the pool is read only after it.
     static_assert(kSlots <= 32 && kOffCap >= 2 * 32 + kSlots, "table ring: a step of entries ahead of every reader");
     bool waited = false, bad_block = false, more = wk.next(seg);
+    int tq_head = 0, tq_tail = 0;            // patch queue: entries tq_head .. tq_tail-1 (indices taken modulo kTailQ)
     int kb = 0;                              // chunks of `seg` already planned
     int planned = 0;                         // chunks of the CTA that have their table entry
     int next_k = lane < kSlots ? lane : INT_MAX, round = 0;   // this lane's next chunk and its round in the slot
@@ -916,10 +950,16 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
         int lo = next_k;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-        while (more && planned + 32 <= lo + kOffCap) {
+        while (more && planned + 32 <= lo + kOffCap && tq_tail - tq_head < kTailQ) {
           const int cnt = seg.c1 - seg.c0;
+          if (kb == 0 && seg.tail_pos >= 0) {
+            // this segment ends with the agent's newest position: queue the patch, ask for the new rows
+            if (lane == 0) sm.tail_q[tq_tail % kTailQ] = make_int4(seg.k0 + seg.tail_pos, seg.a, seg.hk, (seg.n - 1) & 31);
+            ++tq_tail;
+            prefetch_new_token<G>(P.k_new, P.v_new, y.Hkv, seg.a, seg.hk, lane);
+          }
           if (kb + lane < cnt) {
-            const int c = seg.c1 - 1 - (kb + lane);   // a segment is walked from its last chunk to its first (see the consumers)
+            const int c = seg.chunk_at(kb + lane);
             const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
             uint32_t off = kOffBad;
             if (blk >= 0 && blk < P.n_blocks)
@@ -938,6 +978,24 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       // ---- issue: a short polling loop, left from time to time to plan further ----
       bool any_left = true;
       for (int it = 0; it < 64 && any_left; ++it) {
+        // the fused append: quantize the new token into the oldest queued chunk once that chunk has landed (the whole
+        // warp works on it; its consumer waits for sm.patched)
+        if (tq_head < tq_tail) {
+          const int4 t = sm.tail_q[tq_head % kTailQ];
+          const int tslot = t.x % kSlots, tround = t.x / kSlots;
+          const int issued = __shfl_sync(0xffffffffu, round, tslot);      // copies this slot's lane has issued so far
+          if (issued > tround && mbar_test_wait(&sm.full[tslot], (uint32_t)tround & 1u)) {
+            if (!sm.bad[tslot]) {
+              uint8_t* gchunk = const_cast<uint8_t*>(layer_base) + (uint64_t)sm.src_off[t.x % kOffCap] * 16u;
+              append_new_token<G>(sm.ring + (size_t)tslot * kChunkBytes, gchunk, y, P.k_new, P.v_new, t.y, t.z, t.w, lane);
+            }
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) *(volatile int*)&sm.patched[tslot] = tround + 1;
+            ++tq_head;
+            idle = 0;
+          }
+        }
         const bool can = next_k < planned && *my_released >= round;
         if (can) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the consumer's reads and patches of the slot come first
@@ -945,9 +1003,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
           next_k += kSlots;
           ++round;
         }
-        any_left = __any_sync(0xffffffffu, next_k < n_chunks);
+        any_left = __any_sync(0xffffffffu, next_k < n_chunks) || tq_head < tq_tail;
         if (__any_sync(0xffffffffu, can)) { idle = 0; continue; }
-        if (more && __all_sync(0xffffffffu, next_k >= planned)) break;   // nothing to issue before more is planned
+        if (more && tq_tail - tq_head < kTailQ && __all_sync(0xffffffffu, next_k >= planned)) break;   // plan further first
         ++idle;
         __nanosleep(200);
       }
@@ -988,7 +1046,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     for (int s = 0; s < kQBufs && w2.next(s2); ++s) {
       if (s % NW != warp) continue;
       stage_query<G>(sm.qfrag[s], sm.qsum[s], sm.kappa[s], P.q, y.Hq, n_rep, P.scale_log2, s2.a, s2.hk, lane);
-      if (P.k_new != nullptr && s2.c1 == ((s2.n + 31) >> 5)) prefetch_new_token<G>(P.k_new, P.v_new, y.Hkv, s2.a, s2.hk, lane);
       __threadfence_block();
       __syncwarp();
       if (lane == 0) *(volatile int*)&sm.q_tag[s] = s + 1;
@@ -1058,17 +1115,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     segment_epilogue<G, NW>(&sm.merge[b][0][0][0], &sm.epilogues[b], use, P, seg, cta, rs.part, lane);
   };
 
-  // Chunks are claimed one ahead: the claim of the following chunk is taken before this one is worked on, so that the
-  // shared-memory atomic's latency is off the path.
+  // A chunk is claimed only when the warp is free to work on it: a warp that is away in a segment's epilogue (a few
+  // microseconds when it merges a pair's records) must not sit on a claimed chunk meanwhile.
   bool out_of_chunks = false;
-  int k_ahead = 0;
-  if (lane == 0) k_ahead = atomicAdd(&sm.next_chunk, 1);
   for (;;) {
     int k = 0;
     if (!out_of_chunks) {
-      k = __shfl_sync(0xffffffffu, k_ahead, 0);
+      if (lane == 0) k = atomicAdd(&sm.next_chunk, 1);
+      k = __shfl_sync(0xffffffffu, k, 0);
       out_of_chunks = k >= n_chunks;
-      if (!out_of_chunks && lane == 0) k_ahead = atomicAdd(&sm.next_chunk, 1);
     }
     // move to the segment that holds chunk k (to the end of the list when out of chunks), leaving a
     // deposit in every segment passed
@@ -1090,7 +1145,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
         const int prev = cur - kQBufs;
         if (!aborted && !spin_until_ge(&sm.epilogues[prev % kMBufs], prev / kMBufs + 1, &sm.abort_flag)) aborted = true;
         stage_query<G>(sm.qfrag[qb], sm.qsum[qb], sm.kappa[qb], P.q, y.Hq, n_rep, P.scale_log2, seg.a, seg.hk, lane);
-        if (P.k_new != nullptr && seg.c1 == ((seg.n + 31) >> 5)) prefetch_new_token<G>(P.k_new, P.v_new, y.Hkv, seg.a, seg.hk, lane);
         __threadfence_block();
         __syncwarp();
         if (lane == 0) *(volatile int*)&sm.q_tag[qb] = cur + 1;
@@ -1118,18 +1172,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     if (sm.bad[slot]) {
       poisoned = true;
     } else {
-      // A segment is walked from its last chunk to its first: the order does not matter to the online softmax, and
-      // the chunk that may carry the fused append (the agent's newest position) then comes first, where its extra
-      // latency overlaps the other warps' chunks instead of ending the launch.
-      const int c = seg.c1 - 1 - (k - seg.k0);
-      if (P.k_new != nullptr && c == ((seg.n - 1) >> 5)) {
-        // the chunk of the agent's newest position: its block id has passed the producer's check
-        const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
-        uint8_t* gchunk = const_cast<uint8_t*>(head_block(P.pool, y, P.layer, blk, seg.hk)) + (size_t)(c & 7) * kChunkBytes;
-        append_new_token<G>(sm.ring + (size_t)slot * kChunkBytes, gchunk, y, P.k_new, P.v_new, seg.a, seg.hk,
-                            (seg.n - 1) & 31, lane);
-      }
-      process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, c * 32, seg.lo, seg.n, g, tid, qa, qs, kap, split_mask, st);
+      const int j = k - seg.k0;
+      // the chunk that receives the step's new token is usable once the planner warp has quantized the token into it
+      if (j == seg.tail_pos && !spin_until_ge(&sm.patched[slot], round + 1, &sm.abort_flag)) { aborted = true; continue; }
+      __threadfence_block();
+      process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, seg.chunk_at(j) * 32, seg.lo, seg.n, g, tid, qa, qs, kap,
+                       split_mask, st);
     }
     __syncwarp();
     if (lane == 0) { __threadfence_block(); *(volatile int*)&sm.released[slot] = round + 1; }
