@@ -154,6 +154,172 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Bulk form (a prefill phase: many new tokens per agent).  One warp owns one (octet, KV head) unit: the eight cache
+// positions that share position / 8, i.e. the eight nibbles of every token-packed V word it writes.  A lane owns one
+// of the eight positions and one 64-element group at a time (four groups per pass: K groups first, then V groups):
+// it loads its 64 elements as eight 16-byte words (all in flight before the arithmetic), takes minimum and maximum
+// with packed bf16 instructions (no cross-lane step at all), and quantizes them with ~11 instructions per element:
+// the quotient as t * (1/scale), rounded by adding 1.5 * 2^23 (the code is then in the low bits), and only a quotient
+// within 4e-6 of a tie goes through the division itself, so that the codes equal those of the fixed sequence bit for
+// bit.  K words go out as 8-byte stores.  V words are first exchanged between the eight lanes of a group (an 8 x 8
+// transposition of words by twelve shuffles), which leaves in each lane the 8 positions x 8 elements block of
+// nibbles that an in-register transposition turns into eight token-packed words.  Octets that are not full (an
+// unaligned start or end of the phase) take the same path with some lanes idle and read-modify-write the V words.
+// ---------------------------------------------------------------------------------------------
+__device__ inline void transpose_nibbles_8x8_regs(uint32_t (&r)[8]) {
+  // rows = registers, columns = nibbles: three rounds of block swaps
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) {
+    const uint32_t m = s == 1 ? 0x0F0F0F0Fu : s == 2 ? 0x00FF00FFu : 0x0000FFFFu;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (t & s) continue;
+      const uint32_t x = ((r[t] >> (4 * s)) ^ r[t + s]) & m;
+      r[t + s] ^= x;
+      r[t] ^= x << (4 * s);
+    }
+  }
+}
+
+// Code of one element by the division itself (the rare element whose quotient is within a few ulps of a tie).  A call, so
+// that the compiler keeps the division out of the common path.
+__device__ __noinline__ float exact_code(float x, float bf, float sf) {
+  return fminf(rintf(__fdiv_rn(__fsub_rn(x, bf), sf)), 15.0f);
+}
+
+__global__ void __launch_bounds__(kThreads, 3)
+quantize_append_bulk_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_agents, int max_blocks,
+                            const int32_t* __restrict__ tables, const int32_t* __restrict__ pos,
+                            const int32_t* __restrict__ new_offs, const uint16_t* __restrict__ k_new,
+                            const uint16_t* __restrict__ v_new, int32_t* flags, int units) {
+  __shared__ UnitInfo s_unit[kThreads / 32];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * (kThreads / 32) + warp;
+  const int u = gw / y.Hkv, hk = gw - u * y.Hkv;
+  if (u >= units) return;
+  find_unit(u, n_agents, max_blocks, n_blocks, tables, pos, new_offs, flags, gw == 0, &s_unit[warp]);
+  __syncwarp();
+  const UnitInfo un = s_unit[warp];
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (un.agent < 0) return;
+
+  const int s = lane & 7, gq0 = lane >> 3;             // position slot inside the octet, group inside a pass
+  const int k0 = un.first & 7;
+  const int i = s - k0;                                  // this lane's token of the unit
+  const bool tok = i >= 0 && i < un.cnt;
+  const int slot0 = un.first & 255 & ~7;                 // block slot of the octet's position 0
+  uint8_t* chunk = head_block(pool, y, layer, un.block, hk) + (size_t)(slot0 >> 5) * y.chunk_bytes;
+  const int tau = (slot0 & 31) + s;                      // chunk token of this lane's position
+  const int o = (slot0 & 31) >> 3;                       // token octet inside the chunk
+  const uint32_t nib_mask = un.cnt == 8 ? 0xFFFFFFFFu : (((1u << (4 * un.cnt)) - 1u) << (4 * k0));
+  const int n_groups = y.G + (y.alias ? 0 : y.Gv);
+  constexpr float kMagic = 12582912.0f;                  // 1.5 * 2^23: (q + kMagic) - kMagic is q rounded to nearest even
+  // t * inv is within 2 ulps (2e-6 at q < 16) of the quotient the fixed sequence rounds: beyond 4e-6 of a tie both round
+  // to the same code
+  constexpr float kTieZone = 0.499996f;
+
+  for (int pass = 0; pass * 4 < n_groups; ++pass) {
+    const int gq = pass * 4 + gq0;
+    const bool has = gq < n_groups;
+    const bool is_v = has && gq >= y.G;
+    const int gi = is_v ? gq - y.G : gq;
+    const bool active = has && tok;
+    uint4 raw[8];
+    if (active) {
+      const uint16_t* src = is_v ? v_new + ((size_t)(un.row0 + i) * y.Hkv + hk) * y.Dv + 64 * gi
+                                 : k_new + ((size_t)(un.row0 + i) * y.Hkv + hk) * y.D + 64 * gi;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) raw[j] = __ldg(reinterpret_cast<const uint4*>(src) + j);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) raw[j] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    // minimum and maximum of the 64 elements on packed bf16 (values are exact, so this is the binary32 result)
+    __nv_bfloat162 mn2 = *reinterpret_cast<const __nv_bfloat162*>(&raw[0].x), mx2 = mn2;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t wv[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&wv[e]);
+        mn2 = __hmin2(mn2, v);
+        mx2 = __hmax2(mx2, v);
+      }
+    }
+    const uint32_t mnb = *reinterpret_cast<const uint32_t*>(&mn2), mxb = *reinterpret_cast<const uint32_t*>(&mx2);
+    const float mn = fminf(__uint_as_float(mnb << 16), __uint_as_float(mnb & 0xffff0000u));
+    const float mx = fmaxf(__uint_as_float(mxb << 16), __uint_as_float(mxb & 0xffff0000u));
+    const GroupScale gs = group_scale(mn, mx);
+    uint32_t cw[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) cw[j] = 0u;
+    if (gs.sf != 0.0f) {
+      const float inv = __frcp_rn(gs.sf);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t wv[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+        // t = x - bias, q = t / scale (as t * inv), c = q rounded to nearest even by adding and subtracting 1.5 * 2^23;
+        // q <= 15 + a few ulps by construction of the scale, so no clamp is needed.  The eight codes are assembled in
+        // floating point (two exact 16-bit halves) instead of by shifts.
+        float c[8], far = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float x = (e & 1) ? __uint_as_float(wv[e >> 1] & 0xffff0000u) : __uint_as_float(wv[e >> 1] << 16);
+          const float q = __fmul_rn(__fsub_rn(x, gs.bf), inv);
+          c[e] = __fsub_rn(__fadd_rn(q, kMagic), kMagic);
+          far = fmaxf(far, fabsf(__fsub_rn(q, c[e])));
+        }
+        if (far > kTieZone) {                            // rare: some quotient is too close to a tie for t * inv to decide
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float x = (e & 1) ? __uint_as_float(wv[e >> 1] & 0xffff0000u) : __uint_as_float(wv[e >> 1] << 16);
+            const float q = __fmul_rn(__fsub_rn(x, gs.bf), inv);
+            if (fabsf(__fsub_rn(q, c[e])) > kTieZone) c[e] = exact_code(x, gs.bf, gs.sf);
+          }
+        }
+        const float lo = fmaf(fmaf(fmaf(c[3], 16.f, c[2]), 16.f, c[1]), 16.f, c[0]);
+        const float hi = fmaf(fmaf(fmaf(c[7], 16.f, c[6]), 16.f, c[5]), 16.f, c[4]);
+        const uint32_t w = __byte_perm(__float_as_uint(lo + 8388608.0f), __float_as_uint(hi + 8388608.0f), 0x5410);
+        cw[j] = w;
+      }
+    }
+    const uint32_t sb = (uint32_t)__half_as_ushort(gs.hs) | ((uint32_t)__half_as_ushort(gs.hb) << 16);
+    if (active && !is_v) {
+      // words w = 8 gi + 4 i2 + t sit in 16-byte pieces of four (group, half) words: this lane's pair is 8 bytes
+      uint32_t* kc = reinterpret_cast<uint32_t*>(chunk + y.off_kc);
+#pragma unroll
+      for (int t = 0; t < 4; ++t)
+        *reinterpret_cast<uint2*>(kc + k_word_offset(tau, 8 * gi + t, y.G)) = make_uint2(cw[t], cw[4 + t]);
+      reinterpret_cast<uint32_t*>(chunk + y.off_ksb)[sb_offset(tau, gi, y.G)] = sb;
+    }
+    if (pass * 4 + 3 < y.G) continue;                    // a pass of K groups only: nothing to transpose (warp-uniform)
+    if (active && is_v) reinterpret_cast<uint32_t*>(chunk + y.off_vsb)[sb_offset(tau, gi, y.Gv)] = sb;
+    // 8 x 8 transposition of words between the eight lanes of a group: afterwards lane s holds, in cw[t], word s
+    // (elements 8s .. 8s+7 of the group) of position t
+#pragma unroll
+    for (int b = 4; b > 0; b >>= 1) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (j & b) continue;
+        const uint32_t send = (s & b) ? cw[j] : cw[j | b];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, b);
+        if (s & b) cw[j] = recv; else cw[j | b] = recv;
+      }
+    }
+    transpose_nibbles_8x8_regs(cw);                      // cw[e]: element 8s + e of the group, nibble t = position t
+    if (is_v) {
+      uint32_t* vc = reinterpret_cast<uint32_t*>(chunk + y.off_vc);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        uint32_t* at = vc + v_word_offset(o, 64 * gi + 8 * s + e);
+        *at = nib_mask == 0xFFFFFFFFu ? cw[e] : ((*at & ~nib_mask) | (cw[e] & nib_mask));
+      }
+    }
+  }
+}
+
 template <int M>
 cudaError_t launch_m(const Layout& y, uint8_t* pool, int n_blocks, int layer, const q4kv_batch& b, const int32_t* pos,
                      const int32_t* new_offs, int units, const void* k_new, const void* v_new, int32_t* flags,
@@ -179,6 +345,22 @@ cudaError_t launch_quantize_append(const Layout& y, void* pool, int n_blocks, in
                                    const void* k_new, const void* v_new, int32_t* flags, cudaStream_t st) {
   if (total_new <= 0 || b.n_agents <= 0) return cudaSuccess;
   const int units = total_new / 8 + 2 * b.n_agents;        // >= sum over agents of ceil((pos%8+n)/8)
+  if (total_new >= 8 * b.n_agents) {
+    // a phase of many tokens per agent: one warp per (octet, KV head)
+    const long long warps = (long long)units * y.Hkv;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((warps + kThreads / 32 - 1) / (kThreads / 32)));
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, quantize_append_bulk_kernel, y, (uint8_t*)pool, n_blocks, layer, b.n_agents,
+                              b.max_blocks, b.block_tables, pos, new_offs, (const uint16_t*)k_new,
+                              (const uint16_t*)v_new, flags, units);
+  }
   return launch_m<1>(y, (uint8_t*)pool, n_blocks, layer, b, pos, new_offs, units, k_new, v_new, flags, st);
 }
 

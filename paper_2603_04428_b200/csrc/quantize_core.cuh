@@ -11,6 +11,19 @@ namespace q4kv {
 
 struct QuantOut { uint32_t word; __half2 sb; };
 
+// Scale and bias of one group from its minimum and maximum (the fixed binary32 sequence of the header comment).
+struct GroupScale { __half hs, hb; float sf, bf; };
+__device__ inline GroupScale group_scale(float mn, float mx) {
+  GroupScale gs;
+  gs.hb = __float2half_rd(mn);
+  if (__half2float(gs.hb) == 0.0f) gs.hb = __ushort_as_half((unsigned short)0);   // -0 -> +0
+  gs.bf = __half2float(gs.hb);
+  const float r = __fsub_rn(mx, gs.bf);
+  gs.hs = __float2half_ru(__fdiv_rn(r, 15.0f));
+  gs.sf = __half2float(gs.hs);
+  return gs;
+}
+
 // x[8]: eight consecutive elements owned by this lane; the 8 lanes of a group cooperate.
 __device__ inline QuantOut quantize_eight(const float x[8]) {
   float mn = x[0], mx = x[0];
@@ -21,12 +34,9 @@ __device__ inline QuantOut quantize_eight(const float x[8]) {
     mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   }
-  __half hb = __float2half_rd(mn);
-  if (__half2float(hb) == 0.0f) hb = __ushort_as_half((unsigned short)0);   // -0 -> +0
-  const float bf = __half2float(hb);
-  const float r = __fsub_rn(mx, bf);
-  const __half hs = __float2half_ru(__fdiv_rn(r, 15.0f));
-  const float sf = __half2float(hs);
+  const GroupScale gs = group_scale(mn, mx);
+  const __half hb = gs.hb, hs = gs.hs;
+  const float bf = gs.bf, sf = gs.sf;
   uint32_t w = 0;
   if (sf != 0.0f) {
     // code = clamp(rne(fl((x - b) / s))).  The eight IEEE divisions dominate this function, so the quotient is
