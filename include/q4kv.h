@@ -260,6 +260,41 @@ int q4kv_unpack(const q4kv_spec* spec, const void* src, size_t src_bytes, int32_
                 void* pool, int32_t n_blocks, const int32_t* block_table_row,
                 int32_t* status_flags, void* stream);
 
+
+/* ---- Persisted container and warm restore (Appendix "safetensors Q4 Format"; Section 3.2: the cache is persisted in
+ * its quantized form and restored without a dequantize step; the warm-cache rows of the time-to-first-token table) ----
+ *
+ * One agent's cache as a safetensors file: 8 bytes holding the little-endian length N of the header, N bytes of JSON,
+ * then the data section, which is exactly the buffer q4kv_pack writes.  The header lists, layer by layer and block by
+ * block, the tensors  L{l}_B{b}_K_weights (U32 [Hkv][256][d_qk/8]), L{l}_B{b}_K_scales, L{l}_B{b}_K_biases
+ * (F16 [Hkv][256][d_qk/64]) and the three V tensors likewise (absent when V aliases K), each with its byte range, and
+ * carries the spec and the token count under "__metadata__".  The text is canonical: the same cache gives the same
+ * bytes, and any safetensors reader can open the file.  All three calls below are host-only. */
+size_t q4kv_container_header_bytes(const q4kv_spec* spec, int32_t n_tokens);   /* 8 + N, a multiple of 64; 0: unsupported */
+/* dst: HOST memory of at least q4kv_container_header_bytes. */
+int q4kv_container_write_header(const q4kv_spec* spec, int32_t n_tokens, void* dst, size_t dst_bytes);
+/* src: HOST memory holding at least the header of a container written by this library (any other header is refused
+ * with Q4KV_EINVAL).  Returns the spec, the token count and the offset of the data section. */
+int q4kv_container_read_header(const void* src, size_t src_bytes, q4kv_spec* spec, int32_t* n_tokens, size_t* data_offset);
+
+/* Save: header into host_image (written at once by the calling thread), then q4kv_pack into dev_staging and one
+ * device-to-host copy of the packed bytes behind the header, both enqueued on `stream`.  After the stream has run them,
+ * host_image[0 .. header + packed) is the file.  dev_staging: DEVICE, at least q4kv_packed_bytes; host_image: HOST
+ * (pinned memory for a copy that overlaps other work), at least q4kv_container_header_bytes + q4kv_packed_bytes. */
+int q4kv_save(const q4kv_spec* spec, const void* pool, int32_t n_blocks, const int32_t* block_table_row, int32_t n_tokens,
+              void* dev_staging, size_t dev_staging_bytes, void* host_image, size_t host_image_bytes,
+              int32_t* status_flags, void* stream);
+
+/* Warm restore: the data section of a container, in HOST memory (pinned, 16-byte aligned), goes to the caller-chosen
+ * blocks of the pool in chunks of whole layers: one host-to-device copy per chunk on copy_stream, q4kv_unpack of that
+ * chunk on unpack_stream, the copy of the next chunk overlapping the scatter of this one.  dev_staging: DEVICE, at
+ * least one layer's packed bytes (q4kv_packed_bytes / n_layers); two layers' worth or more lets copies and scatters
+ * overlap.  The two streams may be the same.  The pool is complete when unpack_stream has run everything enqueued here;
+ * the call creates and destroys four CUDA events and allocates no memory. */
+int q4kv_restore(const q4kv_spec* spec, const void* host_packed, size_t packed_bytes, int32_t n_tokens, void* pool,
+                 int32_t n_blocks, const int32_t* block_table_row, void* dev_staging, size_t dev_staging_bytes,
+                 int32_t* status_flags, void* copy_stream, void* unpack_stream);
+
 #ifdef __cplusplus
 }
 #endif

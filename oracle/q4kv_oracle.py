@@ -338,3 +338,49 @@ def unpack(pool: Pool, table_row, n_tokens, buf: np.ndarray):
                 nbytes = t[l, b].nbytes
                 t[l, b] = buf[off:off + nbytes].view(t.dtype).reshape(t[l, b].shape)
                 off += nbytes
+
+
+# ----------------------------------------------------------------------------
+# persisted container (Appendix "safetensors Q4 Format")
+# ----------------------------------------------------------------------------
+def container_header(spec: Spec, n_tokens: int) -> bytes:
+    """Header of the safetensors file that holds one agent's cache: 8-byte little-endian length, then JSON.
+
+    Tensors are listed layer by layer and block by block under the paper's names
+    L{l}_B{b}_{K,V}_{weights,scales,biases}, in the order of the data section
+    (K codes, K scales, K biases, V codes, V scales, V biases), each with dtype,
+    shape [Hkv][256][...] and byte range; "__metadata__" carries the spec and the
+    token count as strings.  No blanks inside; padded with spaces so that the
+    data section starts at a multiple of 64 bytes.
+    """
+    s, T, H = spec, BLOCK_TOKENS, spec.n_kv_heads
+    nblk = -(-n_tokens // T)
+    meta = [("format", "q4kv-1"), ("n_layers", s.n_layers), ("n_q_heads", s.n_q_heads), ("n_kv_heads", s.n_kv_heads),
+            ("d_qk", s.d_qk), ("d_v", s.d_v), ("v_aliases_k", int(s.v_aliases_k)), ("group", GROUP),
+            ("block_tokens", T), ("sb_dtype", 0), ("n_tokens", n_tokens)]
+    parts = ['"__metadata__":{' + ",".join(f'"{k}":"{v}"' for k, v in meta) + "}"]
+    off = 0
+    for l in range(s.n_layers):
+        for b in range(nblk):
+            tensors = [("K", "weights", "U32", s.d_qk // 8, 4), ("K", "scales", "F16", s.d_qk // GROUP, 2),
+                       ("K", "biases", "F16", s.d_qk // GROUP, 2)]
+            if not s.v_aliases_k:
+                tensors += [("V", "weights", "U32", s.d_v // 8, 4), ("V", "scales", "F16", s.d_v // GROUP, 2),
+                            ("V", "biases", "F16", s.d_v // GROUP, 2)]
+            for kv, what, dt, last, esz in tensors:
+                nb = H * T * last * esz
+                parts.append(f'"L{l}_B{b}_{kv}_{what}":{{"dtype":"{dt}","shape":[{H},{T},{last}],'
+                             f'"data_offsets":[{off},{off + nb}]}}')
+                off += nb
+    assert off == s.packed_bytes(n_tokens)
+    js = ("{" + ",".join(parts) + "}").encode("ascii")
+    total = (8 + len(js) + 63) // 64 * 64
+    js = js + b" " * (total - 8 - len(js))
+    return len(js).to_bytes(8, "little") + js
+
+
+def container(pool: Pool, table_row, n_tokens) -> np.ndarray:
+    """The whole file image of one agent: header, then the packed buffer."""
+    head = np.frombuffer(container_header(pool.spec, n_tokens), dtype=np.uint8)
+    return np.concatenate([head, pack(pool, table_row, n_tokens)])
+

@@ -24,6 +24,7 @@ EXPORTS = [
     "q4kv_status_string", "q4kv_pool_bytes", "q4kv_packed_bytes", "q4kv_workspace_bytes",
     "q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack", "q4kv_unpack",
     "q4kv_decode_attention_static", "q4kv_append_decode_attention",
+    "q4kv_container_header_bytes", "q4kv_container_write_header", "q4kv_container_read_header", "q4kv_save", "q4kv_restore",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 WORKSPACE_HEADER_BYTES = 65536
@@ -83,6 +84,16 @@ def lib() -> ctypes.CDLL:
         L.q4kv_prefill_attention.restype = ctypes.c_int
         L.q4kv_prefill_attention.argtypes = [sp, vp, i32, i32, bp, vp, vp, i32, i32, i32, i32, vp, f32, vp, i32, vp,
                                              vp, sz, vp, vp]
+        L.q4kv_container_header_bytes.restype = sz
+        L.q4kv_container_header_bytes.argtypes = [sp, i32]
+        L.q4kv_container_write_header.restype = ctypes.c_int
+        L.q4kv_container_write_header.argtypes = [sp, i32, vp, sz]
+        L.q4kv_container_read_header.restype = ctypes.c_int
+        L.q4kv_container_read_header.argtypes = [vp, sz, sp, ctypes.POINTER(i32), ctypes.POINTER(sz)]
+        L.q4kv_save.restype = ctypes.c_int
+        L.q4kv_save.argtypes = [sp, vp, i32, vp, i32, vp, sz, vp, sz, vp, vp]
+        L.q4kv_restore.restype = ctypes.c_int
+        L.q4kv_restore.argtypes = [sp, vp, sz, i32, vp, i32, vp, vp, sz, vp, vp, vp]
         L.q4kv_pack.restype = ctypes.c_int
         L.q4kv_pack.argtypes = [sp, vp, i32, vp, i32, vp, sz, vp, vp]
         L.q4kv_unpack.restype = ctypes.c_int
@@ -185,3 +196,44 @@ def q4kv_pack(spec, pool, n_blocks, block_table_row, n_tokens, dst, status_flags
 def q4kv_unpack(spec, src, n_tokens, pool, n_blocks, block_table_row, status_flags=None):
     _check(lib().q4kv_unpack(ctypes.byref(spec), _ptr(src), src.numel() * src.element_size(), n_tokens, _ptr(pool),
                              n_blocks, _ptr(block_table_row), _ptr(status_flags), _stream()), "q4kv_unpack")
+
+
+def q4kv_container_header_bytes(spec: Spec, n_tokens: int) -> int:
+    return lib().q4kv_container_header_bytes(ctypes.byref(spec), n_tokens)
+
+
+def q4kv_container_write_header(spec: Spec, n_tokens: int) -> bytes:
+    """The container header (host only) as bytes."""
+    n = q4kv_container_header_bytes(spec, n_tokens)
+    buf = ctypes.create_string_buffer(n)
+    _check(lib().q4kv_container_write_header(ctypes.byref(spec), n_tokens, buf, n), "q4kv_container_write_header")
+    return buf.raw
+
+
+def q4kv_container_read_header(data: bytes):
+    """(spec, n_tokens, data_offset) of a container whose first bytes are `data` (host only)."""
+    spec = Spec()
+    nt, off = ctypes.c_int32(0), ctypes.c_size_t(0)
+    buf = ctypes.create_string_buffer(bytes(data), len(data))
+    _check(lib().q4kv_container_read_header(buf, len(data), ctypes.byref(spec), ctypes.byref(nt), ctypes.byref(off)),
+           "q4kv_container_read_header")
+    return spec, nt.value, off.value
+
+
+def q4kv_save(spec, pool, n_blocks, block_table_row, n_tokens, dev_staging, host_image, status_flags=None):
+    """host_image: a pinned CPU uint8 tensor; complete once the current stream has run."""
+    assert not host_image.is_cuda and host_image.is_contiguous()
+    _check(lib().q4kv_save(ctypes.byref(spec), _ptr(pool), n_blocks, _ptr(block_table_row), n_tokens, _ptr(dev_staging),
+                           dev_staging.numel(), host_image.data_ptr(), host_image.numel(), _ptr(status_flags), _stream()),
+           "q4kv_save")
+
+
+def q4kv_restore(spec, host_packed, n_tokens, pool, n_blocks, block_table_row, dev_staging, status_flags=None,
+                 copy_stream=None, unpack_stream=None):
+    """host_packed: a pinned CPU uint8 tensor holding the container's data section."""
+    assert not host_packed.is_cuda and host_packed.is_contiguous()
+    cs = copy_stream.cuda_stream if copy_stream is not None else _stream()
+    us = unpack_stream.cuda_stream if unpack_stream is not None else _stream()
+    _check(lib().q4kv_restore(ctypes.byref(spec), host_packed.data_ptr(), host_packed.numel(), n_tokens, _ptr(pool), n_blocks,
+                              _ptr(block_table_row), _ptr(dev_staging), dev_staging.numel(), _ptr(status_flags), cs, us),
+           "q4kv_restore")

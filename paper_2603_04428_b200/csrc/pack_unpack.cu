@@ -54,10 +54,10 @@ __device__ inline void transpose_nibbles_8x8(uint32_t (&a)[8]) {
 template <bool kPack>
 __global__ void __launch_bounds__(kThreads)
 pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restrict__ row, int n_tokens,
-                   uint8_t* buf, int32_t* flags) {
+                   uint8_t* buf, int32_t* flags, int layer0) {
   extern __shared__ __align__(16) uint8_t stage_all[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int lb = blockIdx.x / y.Hkv, hk = blockIdx.x % y.Hkv, layer = blockIdx.y;
+  const int lb = blockIdx.x / y.Hkv, hk = blockIdx.x % y.Hkv, layer = layer0 + blockIdx.y;   // buf starts at layer0
   const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
   const int phys = row[lb];
   const bool bad = phys < 0 || phys >= n_blocks;
@@ -68,7 +68,7 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
   const int slot0 = warp * kChunkTokens;
   const int nv = max(0, min(kChunkTokens, n_tokens - lb * kBlockTokens - slot0));   // tokens of this chunk that exist
   uint8_t* chunk = bad ? nullptr : head_block(pool, y, layer, phys, hk) + (size_t)warp * y.chunk_bytes;
-  uint8_t* pb = buf + ((uint64_t)layer * nblk + lb) * persisted_block_bytes(y);
+  uint8_t* pb = buf + ((uint64_t)blockIdx.y * nblk + lb) * persisted_block_bytes(y);
   const PersistedOffsets po = persisted_offsets(y);
   const int kw = y.D / 8, vw = y.Dv / 8;
   uint8_t* st = stage_all + (size_t)warp * y.chunk_bytes;
@@ -152,7 +152,7 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
 namespace {
 template <bool kPack>
 cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_t* row, int n_tokens, uint8_t* buf,
-                      int32_t* flags, cudaStream_t st) {
+                      int32_t* flags, cudaStream_t st, int layer0, int layer_count) {
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -163,9 +163,9 @@ cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-  dim3 grid(nblk * y.Hkv, y.L);
+  dim3 grid(nblk * y.Hkv, layer_count);
   pack_unpack_kernel<kPack><<<grid, kThreads, (size_t)kChunksPerBlock * y.chunk_bytes, st>>>(y, pool, n_blocks, row, n_tokens,
-                                                                                              buf, flags);
+                                                                                              buf, flags, layer0);
   return cudaGetLastError();
 }
 }  // namespace
@@ -173,13 +173,20 @@ cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_
 cudaError_t launch_pack(const Layout& y, const void* pool, int n_blocks, const int32_t* row, int n_tokens,
                         void* dst, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  return launch_pu<true>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags, st);
+  return launch_pu<true>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags, st, 0, y.L);
 }
 
 cudaError_t launch_unpack(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
                           const int32_t* row, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st);
+  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, 0, y.L);
+}
+
+// layers [layer0, layer0 + layer_count) only; src points at the persisted bytes of layer0
+cudaError_t launch_unpack_layers(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
+                                 const int32_t* row, int32_t* flags, cudaStream_t st, int layer0, int layer_count) {
+  if (n_tokens <= 0 || layer_count <= 0) return cudaSuccess;
+  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, layer0, layer_count);
 }
 
 }  // namespace q4kv

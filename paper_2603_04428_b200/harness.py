@@ -120,3 +120,34 @@ class DeviceCache:
     def unpack(self, agent, n_tokens, buf):
         src = dev(buf) if isinstance(buf, np.ndarray) else buf
         B.q4kv_unpack(self.spec, src, n_tokens, self.pool, self.n_blocks, self.tables[agent], self.flags)
+
+    # ---- persisted container and warm restore ----------------------------------------------------
+    def save(self, agent, n_tokens) -> torch.Tensor:
+        """The agent's file image (header + packed bytes) in pinned host memory."""
+        hb = B.q4kv_container_header_bytes(self.spec, n_tokens)
+        pb = B.q4kv_packed_bytes(self.spec, n_tokens)
+        stage = torch.empty(pb, dtype=torch.uint8, device="cuda")
+        image = torch.empty(hb + pb, dtype=torch.uint8).pin_memory()
+        B.q4kv_save(self.spec, self.pool, self.n_blocks, self.tables[agent], n_tokens, stage, image, self.flags)
+        torch.cuda.current_stream().synchronize()
+        return image
+
+    def restore(self, agent, image: torch.Tensor, staging_layers: int = 0):
+        """Scatter a file image (pinned host uint8 tensor) into the agent's blocks; returns the token count."""
+        spec, n_tokens, off = B.q4kv_container_read_header(bytes(image[:min(image.numel(), 1 << 22)].numpy()))
+        pb = B.q4kv_packed_bytes(self.spec, n_tokens)
+        packed = image[off:off + pb]
+        if packed.data_ptr() % 16:
+            packed = packed.clone().pin_memory()
+        layer_bytes = pb // self.spec.n_layers
+        n_stage = staging_layers or min(self.spec.n_layers, 8)
+        stage = torch.empty(n_stage * layer_bytes, dtype=torch.uint8, device="cuda")
+        copy_stream = torch.cuda.Stream()
+        cur = torch.cuda.current_stream()
+        copy_stream.wait_stream(cur)
+        B.q4kv_restore(self.spec, packed, n_tokens, self.pool, self.n_blocks, self.tables[agent], stage, self.flags,
+                       copy_stream=copy_stream, unpack_stream=cur)
+        cur.synchronize()
+        copy_stream.synchronize()
+        return n_tokens
+

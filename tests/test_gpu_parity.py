@@ -707,6 +707,39 @@ def test_prefill_bad_block_and_bad_length(H):
     p.dc.flags.zero_()
 
 
+
+# ---- persisted container and warm restore --------------------------------------------------------
+@pytest.mark.parametrize("name,lens", [("gqa128", [700, 33]), ("mla", [300, 256]), ("asym", [17, 513])])
+def test_saved_file_image_equals_the_oracles_and_restores_into_other_blocks(H, name, lens, tmp_path):
+    """q4kv_save writes exactly the oracle's file image (canonical header + packed bytes); the image, written to a file
+    and read back, is restored by q4kv_restore into another cache's blocks (chunked copies overlapping the scatter),
+    after which that cache packs to the same bytes and attends to the same result."""
+    p = Pair(H, SPECS[name], lens, seed=61).fill()
+    s = p.ospec
+    images = []
+    for a, n in enumerate(lens):
+        img = p.dc.save(a, n)
+        ref = O.container(p.opool, p.tabs[a], n)
+        assert img.numel() == ref.size and np.array_equal(img.numpy(), ref), f"agent {a}"
+        f = tmp_path / f"agent{a}.safetensors"
+        f.write_bytes(img.numpy().tobytes())
+        images.append(f)
+    # a second cache with other physical blocks
+    p2 = Pair(H, SPECS[name], lens, seed=62)
+    for a, n in enumerate(lens):
+        raw = np.fromfile(images[a], dtype=np.uint8)
+        img = torch.from_numpy(raw).pin_memory()
+        for stage_layers in (1, 2):                                   # one staging half, then two
+            assert p2.dc.restore(a, img, staging_layers=stage_layers) == n
+            assert np.array_equal(p2.dc.pack(a, n).cpu().numpy(), O.pack(p.opool, p.tabs[a], n))
+    q = p.q(7, len(lens))
+    scale = 1.0 / math.sqrt(192 if name == "mla" else s.d_qk)
+    ref, _ = O.decode_attention(p.opool, 0, p.tabs, lens, 0, f32(q), scale)
+    out, _ = p2.dc.decode(0, lens, 0, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert p.dc.read_flags() == 0 and p2.dc.read_flags() == 0
+
+
 # ---- anomalies are reported, not faulted on -----------------------------------------------------
 def test_bad_block_id_and_bad_length_raise_flags_and_zero_output(H):
     from paper_2603_04428_b200 import binding as B
