@@ -295,6 +295,41 @@ int q4kv_restore(const q4kv_spec* spec, const void* host_packed, size_t packed_b
                  int32_t n_blocks, const int32_t* block_table_row, void* dev_staging, size_t dev_staging_bytes,
                  int32_t* status_flags, void* copy_stream, void* unpack_stream);
 
+/* ---- Block pool bookkeeping (Section 3.1 "Block Pool with Per-Agent Isolation") ----
+ * Host-side policy only; no device memory is touched.  Every block belongs to at most one agent (isolation); agents
+ * are kept in least-recently-used order.  When q4kv_allocator_reserve reports Q4KV_EWORKSPACE the pool is full: ask
+ * q4kv_allocator_pick_victim for the least recently used agent that is not pinned, persist it (q4kv_save), release
+ * it, and reserve again.  Not thread-safe: serialise the calls on one allocator. */
+typedef struct q4kv_allocator q4kv_allocator;
+q4kv_allocator* q4kv_allocator_create(int32_t n_blocks);            /* NULL: n_blocks <= 0 or no host memory */
+void q4kv_allocator_destroy(q4kv_allocator* allocator);
+int32_t q4kv_allocator_free_blocks(const q4kv_allocator* allocator);
+int32_t q4kv_allocator_agent_blocks(const q4kv_allocator* allocator, int64_t agent_id);   /* 0: unknown agent */
+/* Make the agent's block list cover n_tokens (it only grows; earlier blocks keep their place), mark the agent most
+ * recently used, and write its block-table row to table_row (HOST, max_blocks entries, -1 past the last block). */
+int q4kv_allocator_reserve(q4kv_allocator* allocator, int64_t agent_id, int32_t n_tokens, int32_t* table_row,
+                           int32_t max_blocks);
+int q4kv_allocator_touch(q4kv_allocator* allocator, int64_t agent_id);                    /* most recently used */
+int q4kv_allocator_pin(q4kv_allocator* allocator, int64_t agent_id, int32_t pinned);      /* pinned agents are never victims */
+int q4kv_allocator_pick_victim(const q4kv_allocator* allocator, int64_t* agent_id);       /* Q4KV_EWORKSPACE: none */
+int q4kv_allocator_release(q4kv_allocator* allocator, int64_t agent_id);                  /* its blocks become free */
+
+/* ---- Dense-batch shim (Section 3.4: BatchQuantizedKVCache.merge / extract) ----
+ * The paper stacks caches of different lengths into one left-padded batch.  This library attends through block tables
+ * and needs no such copy; these two calls serve code that holds, or wants, the dense form of ONE layer:
+ *   K_codes u32 [A][Hkv][T][d_qk/8] | K_scales f16 [A][Hkv][T][d_qk/64] | K_biases | V_codes | V_scales | V_biases
+ * (no V tensors when v_aliases_k), one tensor after the other, agent a's kv_lens[a] tokens in rows T - kv_lens[a] ..
+ * T - 1 and zero bytes in the padding rows before them.  merge: dense -> the agents' pool blocks (cache positions
+ * 0 .. kv_lens[a] - 1); extract: the reverse.  kv_lens: DEVICE [A]; a length above T or above max_blocks * 256 raises
+ * Q4KV_FLAG_BAD_LENGTH and skips the agent.  dense: DEVICE, at least q4kv_dense_bytes(spec, A, T). */
+size_t q4kv_dense_bytes(const q4kv_spec* spec, int32_t n_agents, int32_t T);
+int q4kv_merge_dense(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer, const q4kv_batch* batch,
+                     const int32_t* kv_lens, int32_t T, const void* dense, size_t dense_bytes, int32_t* status_flags,
+                     void* stream);
+int q4kv_extract_dense(const q4kv_spec* spec, const void* pool, int32_t n_blocks, int32_t layer, const q4kv_batch* batch,
+                       const int32_t* kv_lens, int32_t T, void* dense, size_t dense_bytes, int32_t* status_flags,
+                       void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -384,3 +384,38 @@ def container(pool: Pool, table_row, n_tokens) -> np.ndarray:
     head = np.frombuffer(container_header(pool.spec, n_tokens), dtype=np.uint8)
     return np.concatenate([head, pack(pool, table_row, n_tokens)])
 
+
+# ----------------------------------------------------------------------------
+# dense left-padded batch of one layer (Section 3.4: merge / extract)
+# ----------------------------------------------------------------------------
+def extract_dense(pool: Pool, layer, block_tables, kv_lens, T) -> np.ndarray:
+    """The paper's merged cache of one layer as bytes: K codes [A][Hkv][T][D/8] u32, K scales, K biases
+    [A][Hkv][T][D/64] f16, then the V tensors (absent when V aliases K), one after the other; agent a's
+    tokens sit in rows T - len_a .. T - 1, the padding rows before them are zero."""
+    s, A = pool.spec, len(kv_lens)
+    outs = [np.zeros((A,) + t.shape[2:3] + (T,) + t.shape[4:], dtype=t.dtype) for t in pool.tensors()]
+    for a, n in enumerate(kv_lens):
+        assert 0 <= n <= T
+        for j in range(n):
+            b, slot = int(block_tables[a][j // BLOCK_TOKENS]), j % BLOCK_TOKENS
+            for o, t in zip(outs, pool.tensors()):
+                o[a, :, T - n + j] = t[layer, b, :, slot]
+    return np.concatenate([o.reshape(-1).view(np.uint8) for o in outs])
+
+
+def merge_dense(pool: Pool, layer, block_tables, kv_lens, T, dense: np.ndarray):
+    """Inverse of extract_dense: the rows of a dense left-padded batch go to cache positions 0 .. len_a - 1."""
+    s, A = pool.spec, len(kv_lens)
+    dense = np.asarray(dense, dtype=np.uint8)
+    off = 0
+    for t in pool.tensors():
+        shape = (A,) + t.shape[2:3] + (T,) + t.shape[4:]
+        nb = int(np.prod(shape)) * t.dtype.itemsize
+        d = dense[off:off + nb].view(t.dtype).reshape(shape)
+        off += nb
+        for a, n in enumerate(kv_lens):
+            for j in range(n):
+                b, slot = int(block_tables[a][j // BLOCK_TOKENS]), j % BLOCK_TOKENS
+                t[layer, b, :, slot] = d[a, :, T - n + j]
+    assert off == dense.size
+

@@ -25,6 +25,9 @@ EXPORTS = [
     "q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack", "q4kv_unpack",
     "q4kv_decode_attention_static", "q4kv_append_decode_attention",
     "q4kv_container_header_bytes", "q4kv_container_write_header", "q4kv_container_read_header", "q4kv_save", "q4kv_restore",
+    "q4kv_allocator_create", "q4kv_allocator_destroy", "q4kv_allocator_free_blocks", "q4kv_allocator_agent_blocks",
+    "q4kv_allocator_reserve", "q4kv_allocator_touch", "q4kv_allocator_pin", "q4kv_allocator_pick_victim",
+    "q4kv_allocator_release", "q4kv_dense_bytes", "q4kv_merge_dense", "q4kv_extract_dense",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 WORKSPACE_HEADER_BYTES = 65536
@@ -94,6 +97,31 @@ def lib() -> ctypes.CDLL:
         L.q4kv_save.argtypes = [sp, vp, i32, vp, i32, vp, sz, vp, sz, vp, vp]
         L.q4kv_restore.restype = ctypes.c_int
         L.q4kv_restore.argtypes = [sp, vp, sz, i32, vp, i32, vp, vp, sz, vp, vp, vp]
+        i64 = ctypes.c_int64
+        L.q4kv_allocator_create.restype = vp
+        L.q4kv_allocator_create.argtypes = [i32]
+        L.q4kv_allocator_destroy.restype = None
+        L.q4kv_allocator_destroy.argtypes = [vp]
+        L.q4kv_allocator_free_blocks.restype = i32
+        L.q4kv_allocator_free_blocks.argtypes = [vp]
+        L.q4kv_allocator_agent_blocks.restype = i32
+        L.q4kv_allocator_agent_blocks.argtypes = [vp, i64]
+        L.q4kv_allocator_reserve.restype = ctypes.c_int
+        L.q4kv_allocator_reserve.argtypes = [vp, i64, i32, ctypes.POINTER(i32), i32]
+        L.q4kv_allocator_touch.restype = ctypes.c_int
+        L.q4kv_allocator_touch.argtypes = [vp, i64]
+        L.q4kv_allocator_pin.restype = ctypes.c_int
+        L.q4kv_allocator_pin.argtypes = [vp, i64, i32]
+        L.q4kv_allocator_pick_victim.restype = ctypes.c_int
+        L.q4kv_allocator_pick_victim.argtypes = [vp, ctypes.POINTER(i64)]
+        L.q4kv_allocator_release.restype = ctypes.c_int
+        L.q4kv_allocator_release.argtypes = [vp, i64]
+        L.q4kv_dense_bytes.restype = sz
+        L.q4kv_dense_bytes.argtypes = [sp, i32, i32]
+        L.q4kv_merge_dense.restype = ctypes.c_int
+        L.q4kv_merge_dense.argtypes = [sp, vp, i32, i32, bp, vp, i32, vp, sz, vp, vp]
+        L.q4kv_extract_dense.restype = ctypes.c_int
+        L.q4kv_extract_dense.argtypes = [sp, vp, i32, i32, bp, vp, i32, vp, sz, vp, vp]
         L.q4kv_pack.restype = ctypes.c_int
         L.q4kv_pack.argtypes = [sp, vp, i32, vp, i32, vp, sz, vp, vp]
         L.q4kv_unpack.restype = ctypes.c_int
@@ -237,3 +265,60 @@ def q4kv_restore(spec, host_packed, n_tokens, pool, n_blocks, block_table_row, d
     _check(lib().q4kv_restore(ctypes.byref(spec), host_packed.data_ptr(), host_packed.numel(), n_tokens, _ptr(pool), n_blocks,
                               _ptr(block_table_row), _ptr(dev_staging), dev_staging.numel(), _ptr(status_flags), cs, us),
            "q4kv_restore")
+
+
+class Allocator:
+    """Thin holder of a q4kv_allocator (host-side block bookkeeping with LRU order)."""
+
+    def __init__(self, n_blocks: int):
+        self._h = lib().q4kv_allocator_create(n_blocks)
+        if not self._h:
+            raise Q4KVError(EINVAL, "q4kv_allocator_create")
+
+    def close(self):
+        if self._h:
+            lib().q4kv_allocator_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def free_blocks(self) -> int:
+        return lib().q4kv_allocator_free_blocks(self._h)
+
+    def agent_blocks(self, agent_id: int) -> int:
+        return lib().q4kv_allocator_agent_blocks(self._h, agent_id)
+
+    def reserve(self, agent_id: int, n_tokens: int, max_blocks: int):
+        row = (ctypes.c_int32 * max_blocks)()
+        _check(lib().q4kv_allocator_reserve(self._h, agent_id, n_tokens, row, max_blocks), "q4kv_allocator_reserve")
+        return list(row)
+
+    def touch(self, agent_id: int):
+        _check(lib().q4kv_allocator_touch(self._h, agent_id), "q4kv_allocator_touch")
+
+    def pin(self, agent_id: int, pinned: bool):
+        _check(lib().q4kv_allocator_pin(self._h, agent_id, int(pinned)), "q4kv_allocator_pin")
+
+    def pick_victim(self) -> int:
+        v = ctypes.c_int64(0)
+        _check(lib().q4kv_allocator_pick_victim(self._h, ctypes.byref(v)), "q4kv_allocator_pick_victim")
+        return v.value
+
+    def release(self, agent_id: int):
+        _check(lib().q4kv_allocator_release(self._h, agent_id), "q4kv_allocator_release")
+
+
+def q4kv_dense_bytes(spec: Spec, n_agents: int, T: int) -> int:
+    return lib().q4kv_dense_bytes(ctypes.byref(spec), n_agents, T)
+
+
+def q4kv_merge_dense(spec, pool, n_blocks, layer, bt: Batch, kv_lens, T, dense, status_flags=None):
+    _check(lib().q4kv_merge_dense(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt), _ptr(kv_lens), T,
+                                  _ptr(dense), dense.numel() * dense.element_size(), _ptr(status_flags), _stream()),
+           "q4kv_merge_dense")
+
+
+def q4kv_extract_dense(spec, pool, n_blocks, layer, bt: Batch, kv_lens, T, dense, status_flags=None):
+    _check(lib().q4kv_extract_dense(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt), _ptr(kv_lens), T,
+                                    _ptr(dense), dense.numel() * dense.element_size(), _ptr(status_flags), _stream()),
+           "q4kv_extract_dense")

@@ -123,6 +123,8 @@ cudaError_t launch_unpack(const Layout& y, const void* src, int n_tokens, void* 
                           const int32_t* row, int32_t* flags, cudaStream_t st);
 cudaError_t launch_unpack_layers(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
                                  const int32_t* row, int32_t* flags, cudaStream_t st, int layer0, int layer_count);
+cudaError_t launch_dense_exchange(const Layout& y, void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                                  const int32_t* kv_lens, int T, void* dense, bool to_pool, int32_t* flags, cudaStream_t st);
 cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                                      const int32_t* kv_lens, const int32_t* q_offs, int total_q, int max_q_len,
                                      int max_kv_len, int window, const void* q, float scale, void* out,

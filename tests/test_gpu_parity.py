@@ -740,6 +740,35 @@ def test_saved_file_image_equals_the_oracles_and_restores_into_other_blocks(H, n
     assert p.dc.read_flags() == 0 and p2.dc.read_flags() == 0
 
 
+
+@pytest.mark.parametrize("name,lens,T", [("gqa128", [300, 5, 0, 256, 33], 320), ("mla", [70, 513], 520), ("asym", [17, 290], 290)])
+def test_dense_batch_extract_and_merge_match_the_oracle(H, name, lens, T):
+    """The paper's merge / extract as a shim: a layer's caches as one left-padded dense batch, bytes equal to the
+    oracle's, and merged back into other blocks (partly filled chunks keep their neighbours' slots) to the same cache."""
+    from paper_2603_04428_b200 import binding as B
+    p = Pair(H, SPECS[name], lens, seed=63).fill()
+    s = p.ospec
+    A = len(lens)
+    lens_d = H.dev(np.asarray(lens, dtype=np.int32))
+    nbytes = B.q4kv_dense_bytes(p.dc.spec, A, T)
+    layer = s.n_layers - 1
+    dense = torch.full((nbytes,), 0xAB, dtype=torch.uint8, device="cuda")
+    B.q4kv_extract_dense(p.dc.spec, p.dc.pool, p.dc.n_blocks, layer, p.dc.bt, lens_d, T, dense, p.dc.flags)
+    ref = O.extract_dense(p.opool, layer, p.tabs, lens, T)
+    assert ref.size == nbytes and np.array_equal(dense.cpu().numpy(), ref)
+    # merge into a cache that already holds other tokens: positions >= len keep what was there
+    longer = [n + 40 for n in lens]
+    p2 = Pair(H, SPECS[name], longer, seed=64).fill()
+    B.q4kv_merge_dense(p2.dc.spec, p2.dc.pool, p2.dc.n_blocks, layer, p2.dc.bt, lens_d, T, dense, p2.dc.flags)
+    O.merge_dense(p2.opool, layer, p2.tabs, lens, T, ref)
+    p2.check_packed_equal()                                      # every layer, all longer[a] positions
+    # a length beyond the dense row count is flagged and skipped
+    bad = H.dev(np.asarray([T + 1] + lens[1:], dtype=np.int32))
+    B.q4kv_extract_dense(p.dc.spec, p.dc.pool, p.dc.n_blocks, layer, p.dc.bt, bad, T, dense, p.dc.flags)
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    p.dc.flags.zero_()
+
+
 # ---- anomalies are reported, not faulted on -----------------------------------------------------
 def test_bad_block_id_and_bad_length_raise_flags_and_zero_output(H):
     from paper_2603_04428_b200 import binding as B
