@@ -206,6 +206,20 @@ class DeviceWorkload:
                                        self.q[l], w.softmax_scale,
                                        self.out[l], B.OUT_F32, None, self.ws, dc.flags)
 
+    def layers_supported(self):
+        w = self.w
+        return fused_update_and_fetch(w) and not w.v_aliases_k and w.n_layers <= 64
+
+    def layers_step(self):
+        """The whole step as ONE launch: update-and-fetch of all layers (for callers that hold every layer's rows)."""
+        w, dc, B = self.w, self.dc, self.B
+        if not hasattr(self, "ws_layers"):
+            self.ws_layers = self.torch.zeros(B.q4kv_workspace_bytes_layers(dc.spec, w.n_agents, self.max_kv, w.n_layers),
+                                              dtype=self.torch.uint8, device="cuda")
+        B.q4kv_decode_attention_layers(dc.spec, dc.pool, dc.n_blocks, 0, w.n_layers, dc.bt, self.lens1, self.max_kv,
+                                       [w.layer_window(l) for l in range(w.n_layers)], self.k_new, self.v_new, self.q,
+                                       w.softmax_scale, self.out, B.OUT_F32, None, self.ws_layers, dc.flags)
+
     def step(self):
         for l in range(self.w.n_layers):
             if self.fused:
@@ -424,7 +438,13 @@ def measure(w, args, local, dist=None, full=True):
             gl_layers = [l for l in range(L) if w.layer_window(l) == 0]
             gl_fn = dw.fused_layer if dw.fused else dw.attend_layer
             gl_s = per_launch_s(lambda i: gl_fn(gl_layers[i % len(gl_layers)]))
+        lb_s = None
+        if dw.layers_supported():
+            for _ in range(3):
+                dw.layers_step()
+            lb_s = float(np.median(timed_batches(torch, dw.layers_step, 1, min_total_s=args.min_seconds / 2)))
         clocks = sampler.stop()
+        res.update(lb_s=lb_s)
         res.update(t_step=t_step, k=k, n_batches=len(batches), region_s=float(np.sum(batches)), att_s=att_s, app_s=app_s,
                    gl_s=gl_s, clocks=clocks, graph=graph is not None, fused=dw.fused)
         if full:
@@ -480,6 +500,12 @@ def roofline_of(w, res):
                 "frac": ach / tf_sust, "frac_of_burst": ach / tf_burst, "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS}
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
     roof["avg_launch_us"] = att_s * 1e6
+    if res.get("lb_s"):
+        # the same step as one launch for all layers (q4kv_decode_attention_layers): the per-kernel rate at this
+        # batch size when the caller has every layer's rows at hand; labelled, beside the per-layer number
+        ach = step_units / res["lb_s"] / 1e9
+        roof["layer_batched"] = {"kernel": "q4kv_decode_attention_layers (all layers in one launch)", "ms_per_step": res["lb_s"] * 1e3,
+                                 "achieved": ach, "frac": ach / hbm_peak, "agent_steps_per_s": w.n_agents / res["lb_s"]}
     return step_units, roof
 
 

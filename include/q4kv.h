@@ -196,6 +196,26 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
                                  void* workspace, size_t workspace_bytes,
                                  int32_t* status_flags, void* stream);
 
+/* Update-and-fetch (or plain decode attention) for SEVERAL layers in one launch (Section 3.4; the same update_and_fetch,
+ * batched over layers as well as agents).  For callers that hold the queries -- and, for the update, the new K/V rows --
+ * of layers layer_begin .. layer_begin + layer_count - 1 at once (a replayed step, a speculative pass, a test harness):
+ * the kernel's work list then runs over layers x agents x KV heads, so that small batches still fill the GPU.  Equivalent
+ * to layer_count calls of q4kv_append_decode_attention (k_new, v_new given) or q4kv_decode_attention (both NULL), layer by
+ * layer.
+ *   windows  HOST [layer_count]: the sliding window of each layer (0: none)
+ *   k_new    bf16 [layer_count][A][n_kv_heads][d_qk], v_new likewise with d_v; both NULL: nothing is appended
+ *   q        bf16 [layer_count][A][n_q_heads][d_qk];  out [layer_count][A][n_q_heads][d_v];  lse [layer_count][A][n_q_heads]
+ *   workspace  at least q4kv_workspace_bytes_layers(spec, A, max_kv_len, layer_count) bytes, header zeroed as for
+ *              q4kv_decode_attention
+ * Covered specs: d_qk = d_v in {128, 256}, at most four query heads per KV head, V not aliasing K, at most 64 layers
+ * per call; anything else returns Q4KV_EUNSUPPORTED (call layer by layer then). */
+size_t q4kv_workspace_bytes_layers(const q4kv_spec* spec, int32_t n_agents, int32_t max_kv_len, int32_t layer_count);
+int q4kv_decode_attention_layers(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer_begin,
+                                 int32_t layer_count, const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                                 const int32_t* windows, const void* k_new, const void* v_new, const void* q,
+                                 float softmax_scale, void* out, int32_t out_dtype, float* lse,
+                                 void* workspace, size_t workspace_bytes, int32_t* status_flags, void* stream);
+
 /* Decode attention without a caller-supplied workspace.  The paper has no counterpart: this entry
  * point exists for hosts that cannot allocate device memory when they call -- a runtime that
  * carved up all of its device memory at start-up, a plugin that must not touch its host's

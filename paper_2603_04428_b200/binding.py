@@ -23,7 +23,8 @@ OUT_F32, OUT_BF16 = 0, 1
 EXPORTS = [
     "q4kv_status_string", "q4kv_pool_bytes", "q4kv_packed_bytes", "q4kv_workspace_bytes",
     "q4kv_quantize_append", "q4kv_decode_attention", "q4kv_prefill_attention", "q4kv_pack", "q4kv_unpack",
-    "q4kv_decode_attention_static", "q4kv_append_decode_attention",
+    "q4kv_decode_attention_static", "q4kv_append_decode_attention", "q4kv_decode_attention_layers",
+    "q4kv_workspace_bytes_layers",
     "q4kv_container_header_bytes", "q4kv_container_write_header", "q4kv_container_read_header", "q4kv_save", "q4kv_restore",
     "q4kv_allocator_create", "q4kv_allocator_destroy", "q4kv_allocator_free_blocks", "q4kv_allocator_agent_blocks",
     "q4kv_allocator_reserve", "q4kv_allocator_touch", "q4kv_allocator_pin", "q4kv_allocator_pick_victim",
@@ -82,6 +83,11 @@ def lib() -> ctypes.CDLL:
         L.q4kv_append_decode_attention.restype = ctypes.c_int
         L.q4kv_append_decode_attention.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, vp, vp, f32, vp, i32, vp, vp,
                                                    sz, vp, vp]
+        L.q4kv_workspace_bytes_layers.restype = sz
+        L.q4kv_workspace_bytes_layers.argtypes = [sp, i32, i32, i32]
+        L.q4kv_decode_attention_layers.restype = ctypes.c_int
+        L.q4kv_decode_attention_layers.argtypes = [sp, vp, i32, i32, i32, bp, vp, i32, ctypes.POINTER(i32), vp, vp, vp, f32, vp,
+                                                   i32, vp, vp, sz, vp, vp]
         L.q4kv_decode_attention_static.restype = ctypes.c_int
         L.q4kv_decode_attention_static.argtypes = [sp, vp, i32, i32, bp, vp, i32, i32, vp, f32, vp, i32, vp, vp, vp]
         L.q4kv_prefill_attention.restype = ctypes.c_int
@@ -322,3 +328,18 @@ def q4kv_extract_dense(spec, pool, n_blocks, layer, bt: Batch, kv_lens, T, dense
     _check(lib().q4kv_extract_dense(ctypes.byref(spec), _ptr(pool), n_blocks, layer, ctypes.byref(bt), _ptr(kv_lens), T,
                                     _ptr(dense), dense.numel() * dense.element_size(), _ptr(status_flags), _stream()),
            "q4kv_extract_dense")
+
+
+def q4kv_workspace_bytes_layers(spec: Spec, n_agents: int, max_kv_len: int, layer_count: int) -> int:
+    return lib().q4kv_workspace_bytes_layers(ctypes.byref(spec), n_agents, max_kv_len, layer_count)
+
+
+def q4kv_decode_attention_layers(spec, pool, n_blocks, layer_begin, layer_count, bt: Batch, kv_lens, max_kv_len, windows,
+                                 k_new, v_new, q, softmax_scale, out, out_dtype, lse, workspace, status_flags=None):
+    """Decode attention (k_new, v_new None) or update-and-fetch for layer_count layers in one launch; windows: a host list."""
+    w = (ctypes.c_int32 * layer_count)(*[int(x) for x in windows])
+    _check(lib().q4kv_decode_attention_layers(ctypes.byref(spec), _ptr(pool), n_blocks, layer_begin, layer_count,
+                                              ctypes.byref(bt), _ptr(kv_lens), max_kv_len, w, _ptr(k_new), _ptr(v_new),
+                                              _ptr(q), softmax_scale, _ptr(out), out_dtype, _ptr(lse), _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream()),
+           "q4kv_decode_attention_layers")

@@ -151,17 +151,42 @@ __device__ inline uint32_t f32x2_to_h2_rn(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+constexpr int kMaxLayersPerCall = 64;
+struct DecodeParams {
+  Layout y;
+  const uint8_t* pool;
+  int n_blocks, layer, n_agents, max_blocks, len_cap;
+  // Several layers in one launch (the layer-batched entry): the work list runs over "virtual agents" v = li * n_real + a
+  // (layer li of the call, real agent a).  q, out, lse, the new rows, the arrival counters and the partial records are
+  // all indexed by v; lengths and block tables by a; the window and the pool layer by li.  n_agents = layer_count * n_real.
+  int n_real, layer_count;
+  int windows[kMaxLayersPerCall];   // sliding window of each layer of the call (0: none)
+  const int32_t* tables;
+  const int32_t* kv_lens;
+  const uint16_t* q;          // bf16 [layer_count][A][Hq][D]
+  float scale_log2;           // softmax_scale * log2(e)
+  int32_t* tickets;           // [A*Hkv], zero between calls
+  float* partials;            // [A*Hkv + grid][n_rep][Dv + 4]
+  void* out;
+  int out_dtype;
+  float* lse;
+  int32_t* flags;
+  const uint16_t* k_new;      // fused append: bf16 [A][Hkv][D] rows of the token at position kv_len - 1 (null: none)
+  const uint16_t* v_new;
+};
+
 // ---------------------------------------------------------------------------------------------
 // Work list: chunks of all (agent, KV head) pairs, agent-major, then head, then chunk
 // ---------------------------------------------------------------------------------------------
 struct AgentRange { int n, lo, cf, nc; };   // keys [lo, n); chunks cf .. cf+nc-1
 
 // len_cap: the host's bound on every length (at most max_blocks * 256); longer or negative lengths are rejected
-__device__ inline AgentRange agent_range(const int32_t* __restrict__ kv_lens, int a, int window, int len_cap,
-                                         bool& bad) {
+__device__ inline AgentRange agent_range(const DecodeParams& P, int a, bool& bad) {
   AgentRange r;
-  r.n = kv_lens[a];
-  bad = r.n < 0 || r.n > len_cap;
+  const int li = P.layer_count > 1 ? a / P.n_real : 0;
+  const int window = P.windows[li];
+  r.n = P.kv_lens[a - li * P.n_real];
+  bad = r.n < 0 || r.n > P.len_cap;
   if (bad) r.n = 0;
   r.lo = window > 0 ? max(0, r.n - window) : 0;
   r.cf = r.lo >> 5;
@@ -185,9 +210,9 @@ struct Partition {
 // first unit.  One pass over the agents when there are at most 32 of them.
 struct RangeStart { uint32_t U, u_begin, u_end, agent_start; int n_ctas, agent; bool any_bad; Partition part; };
 
-__device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int n_agents, int Hkv, int window,
-                                        int len_cap, int cta, int grid) {
+__device__ inline RangeStart find_range(const DecodeParams& P, int cta, int grid) {
   const int lane = threadIdx.x & 31;
+  const int n_agents = P.n_agents, Hkv = P.y.Hkv;
   RangeStart rs;
   rs.any_bad = false;
   rs.agent = -1;
@@ -197,7 +222,7 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
     const int a = base + lane;
     uint32_t cnt = 0;
     bool bad = false;
-    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, len_cap, bad).nc * Hkv);
+    if (a < n_agents) cnt = (uint32_t)(agent_range(P, a, bad).nc * Hkv);
     rs.any_bad |= __any_sync(0xffffffffu, bad);
     uint32_t inc = cnt;
 #pragma unroll
@@ -229,7 +254,7 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
     const int a = base + lane;
     uint32_t cnt = 0;
     bool bad = false;
-    if (a < n_agents) cnt = (uint32_t)(agent_range(kv_lens, a, window, len_cap, bad).nc * Hkv);
+    if (a < n_agents) cnt = (uint32_t)(agent_range(P, a, bad).nc * Hkv);
     uint32_t inc = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -255,7 +280,8 @@ __device__ inline RangeStart find_range(const int32_t* __restrict__ kv_lens, int
 // places back in the walk (to place tail_pos), so that the consumers have other chunks to work on meanwhile.
 constexpr int kTailPos = 14;
 struct Segment {
-  int a, hk, c0, c1;      // logical chunk indices [c0, c1) of the agent
+  int a, hk, c0, c1;      // (virtual) agent, KV head, logical chunk indices [c0, c1) of the agent
+  int ar, li;             // real agent (lengths, block table) and layer of the call (pool layer)
   int n, lo;              // key range of the agent
   int cf, nc;             // the pair's whole chunk range
   int k0;                 // running chunk counter of the CTA at c0
@@ -272,22 +298,21 @@ struct Segment {
 };
 
 struct Walker {
-  const int32_t* kv_lens;
-  int n_agents, Hkv, window, len_cap;
+  const DecodeParams* P;
+  int n_agents, Hkv;
   uint32_t u, u_end;
   int k, a, hk, c;
   bool fused;               // the launch appends one token per agent
   AgentRange r;
 
-  __device__ void init(const int32_t* kv_lens_, int n_agents_, int Hkv_, int window_, int len_cap_,
-                       const RangeStart& rs, bool fused_) {
-    kv_lens = kv_lens_; n_agents = n_agents_; Hkv = Hkv_; window = window_; len_cap = len_cap_; fused = fused_;
+  __device__ void init(const DecodeParams& P_, const RangeStart& rs) {
+    P = &P_; n_agents = P_.n_agents; Hkv = P_.y.Hkv; fused = P_.k_new != nullptr;
     u = rs.u_begin; u_end = rs.u_end; k = 0;
     a = rs.agent; hk = 0; c = 0;
     r.n = 0; r.lo = 0; r.cf = 0; r.nc = 0;
     if (u < u_end && a >= 0) {
       bool bad;
-      r = agent_range(kv_lens, a, window, len_cap, bad);
+      r = agent_range(*P, a, bad);
       const uint32_t rem = u - rs.agent_start;
       hk = (int)(rem / (uint32_t)r.nc);
       c = r.cf + (int)(rem - (uint32_t)hk * (uint32_t)r.nc);
@@ -298,6 +323,7 @@ struct Walker {
     const int pair_end = r.cf + r.nc;
     const uint32_t left = u_end - u;
     const int c1 = (uint32_t)(pair_end - c) <= left ? pair_end : c + (int)left;
+    s.li = P->layer_count > 1 ? a / P->n_real : 0; s.ar = a - s.li * P->n_real;
     s.a = a; s.hk = hk; s.c0 = c; s.c1 = c1; s.n = r.n; s.lo = r.lo; s.cf = r.cf; s.nc = r.nc; s.k0 = k; s.u0 = u;
     s.set_tail(fused);
     const int cnt = c1 - c;
@@ -310,7 +336,7 @@ struct Walker {
         do {
           ++a;
           if (a >= n_agents) { a = -1; break; }
-          r = agent_range(kv_lens, a, window, len_cap, bad);
+          r = agent_range(*P, a, bad);
         } while (r.nc == 0);
       }
       if (a >= 0) c = r.cf;
@@ -324,24 +350,6 @@ struct Walker {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-struct DecodeParams {
-  Layout y;
-  const uint8_t* pool;
-  int n_blocks, layer, n_agents, max_blocks, len_cap;
-  const int32_t* tables;
-  const int32_t* kv_lens;
-  int window;
-  const uint16_t* q;          // bf16 [A][Hq][D]
-  float scale_log2;           // softmax_scale * log2(e)
-  int32_t* tickets;           // [A*Hkv], zero between calls
-  float* partials;            // [A*Hkv + grid][n_rep][Dv + 4]
-  void* out;
-  int out_dtype;
-  float* lse;
-  int32_t* flags;
-  const uint16_t* k_new;      // fused append: bf16 [A][Hkv][D] rows of the token at position kv_len - 1 (null: none)
-  const uint16_t* v_new;
-};
 
 __host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
 constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
@@ -909,11 +917,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   __syncthreads();
 
   // ---- this CTA's unit range (every warp computes it for itself; these inputs are not written by any kernel) ----
-  const RangeStart rs = find_range(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, cta, gridDim.x);
+  const RangeStart rs = find_range(P, cta, gridDim.x);
   if (rs.any_bad && cta == 0 && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
   const int n_chunks = (int)(rs.u_end - rs.u_begin);
   Walker wk;
-  wk.init(P.kv_lens, P.n_agents, y.Hkv, P.window, P.len_cap, rs, P.k_new != nullptr);
+  wk.init(P, rs);
   Segment seg;
 
   const uint8_t* layer_base = P.pool + (uint64_t)P.layer * y.layer_bytes;
@@ -960,10 +968,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
           }
           if (kb + lane < cnt) {
             const int c = seg.chunk_at(kb + lane);
-            const int blk = P.tables[(size_t)seg.a * P.max_blocks + (c >> 3)];
+            const int blk = P.tables[(size_t)seg.ar * P.max_blocks + (c >> 3)];
             uint32_t off = kOffBad;
             if (blk >= 0 && blk < P.n_blocks)
-              off = (uint32_t)(((uint64_t)blk * y.block_bytes + (uint64_t)seg.hk * y.head_block_bytes +
+              off = (uint32_t)(((uint64_t)seg.li * y.layer_bytes + (uint64_t)blk * y.block_bytes + (uint64_t)seg.hk * y.head_block_bytes +
                                 (uint64_t)(c & 7) * kChunkBytes) >> 4);
             else
               bad_block = true;
@@ -1033,7 +1041,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   // agents without any key (kv_len == 0 or a rejected length): zeros, lse = -inf
   for (int a = cta * NW + warp; a < P.n_agents; a += gridDim.x * NW) {
     bool bad_len;
-    if (agent_range(P.kv_lens, a, P.window, P.len_cap, bad_len).nc > 0) continue;
+    if (agent_range(P, a, bad_len).nc > 0) continue;
     for (int i = lane; i < y.Hq * Dv; i += 32) store_out(P, (size_t)a * y.Hq * Dv + i, 0.f);
     if (P.lse) for (int i = lane; i < y.Hq; i += 32) P.lse[(size_t)a * y.Hq + i] = -INFINITY;
   }
@@ -1229,32 +1237,43 @@ bool decode_mma_supported(const Layout& y) {
   return !y.alias && y.D == y.Dv && (y.D == 128 || y.D == 256) && y.n_rep <= 4;
 }
 
-// the kernel counts work units in 32 bits and keeps one arrival counter per (agent, KV head) pair in the
-// workspace header
-bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks) {
-  return (long long)n_agents * y.Hkv * (max_blocks * 8ll) < (1ll << 30) && (long long)n_agents * y.Hkv <= kMaxTicketPairs;
+// the kernel counts work units in 32 bits and keeps one arrival counter per (layer of the call, agent, KV head) in
+// the workspace header; chunk offsets inside the call's layers are kept in 16-byte units in 32 bits
+bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks, int layer_count) {
+  const long long v = (long long)n_agents * layer_count;
+  return layer_count >= 1 && layer_count <= kMaxLayersPerCall && v * y.Hkv * (max_blocks * 8ll) < (1ll << 30) &&
+         v * y.Hkv <= kMaxTicketPairs && (unsigned long long)layer_count * y.layer_bytes < (1ull << 36);
 }
 
-// bytes behind the workspace header: one record per pair and per CTA of the largest grid
-size_t decode_mma_workspace_bytes(const Layout& y, int n_agents) {
-  const size_t pairs = (size_t)n_agents * y.Hkv;
+// bytes behind the workspace header: one record per (layer, agent, KV head) and per CTA of the largest grid
+size_t decode_mma_workspace_bytes(const Layout& y, int n_agents, int layer_count) {
+  const size_t pairs = (size_t)n_agents * layer_count * y.Hkv;
   return (pairs + kMaxGrid) * y.n_rep * kRecStride(y.Dv) * sizeof(float);
 }
 
+// layer_count == 1: `windows` points at the one window.  Otherwise q, out, lse and the new rows hold layer_count
+// consecutive per-layer arrays and the launch covers layers layer .. layer + layer_count - 1.
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
-                              const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
-                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
-                              const void* k_new, const void* v_new) {
-  if (b.n_agents <= 0) return cudaSuccess;
+                              const int32_t* kv_lens, int max_kv_len, const int32_t* windows, int layer_count,
+                              const void* q, float scale, void* out, int out_dtype, float* lse, void* ws, int32_t* flags,
+                              cudaStream_t st, const void* k_new, const void* v_new) {
+  if (b.n_agents <= 0 || layer_count <= 0) return cudaSuccess;
   DecodeParams P;
-  P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
-  P.max_blocks = b.max_blocks; P.len_cap = max_kv_len; P.tables = b.block_tables; P.kv_lens = kv_lens; P.window = window;
+  P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents * layer_count;
+  P.n_real = b.n_agents; P.layer_count = layer_count;
+  long long units = 0;
+  for (int i = 0; i < kMaxLayersPerCall; ++i) {
+    P.windows[i] = i < layer_count ? windows[i] : 0;
+    if (i < layer_count) {
+      const int span = (windows[i] > 0 && windows[i] + 32 < max_kv_len) ? windows[i] + 32 : max_kv_len;
+      units += (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
+    }
+  }
+  P.max_blocks = b.max_blocks; P.len_cap = max_kv_len; P.tables = b.block_tables; P.kv_lens = kv_lens;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e;
   P.tickets = (int32_t*)ws; P.partials = (float*)((uint8_t*)ws + kWorkspaceHeaderBytes);
   P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
   P.k_new = (const uint16_t*)k_new; P.v_new = (const uint16_t*)v_new;
-  const int span = (window > 0 && window + 32 < max_kv_len) ? window + 32 : max_kv_len;
-  const long long units = (long long)b.n_agents * y.Hkv * ((span + 31) / 32 + 1);
   const int n_sm = sm_count();
   const int grid = (int)(units < n_sm ? (units < 1 ? 1 : units) : n_sm);
   return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128>(P, grid, true, st)

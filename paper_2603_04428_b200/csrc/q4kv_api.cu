@@ -125,7 +125,7 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
     e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out, out_dtype,
                           lse, records, status_flags, (cudaStream_t)stream);
   else if (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
-    e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out,
+    e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, &window, 1, q, softmax_scale, out,
                           out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
   else
     e = launch_attention_generic(y, pool, n_blocks, layer, *batch, kv_lens, nullptr, 0, 1, max_kv_len, window, q,
@@ -165,8 +165,46 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
   }
   if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks)) return Q4KV_EUNSUPPORTED;
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
-  const cudaError_t e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,
+  const cudaError_t e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, &window, 1, q, softmax_scale,
                                           out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream, k_new, v_new);
+  return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
+}
+
+size_t q4kv_workspace_bytes_layers(const q4kv_spec* spec, int32_t n_agents, int32_t max_kv_len, int32_t layer_count) {
+  if (check_spec(spec) != Q4KV_OK || n_agents < 0 || max_kv_len < 0 || layer_count < 1) return 0;
+  const Layout y = make_layout(*spec, 1);
+  if (!decode_mma_supported(y)) return 0;
+  const size_t one = workspace_need(y, n_agents > 0 ? n_agents : 1, max_kv_len > 0 ? max_kv_len : 1, 0);
+  const size_t all = kWorkspaceHeaderBytes + decode_mma_workspace_bytes(y, n_agents > 0 ? n_agents : 1, layer_count);
+  return all > one ? all : one;
+}
+
+int q4kv_decode_attention_layers(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer_begin,
+                                 int32_t layer_count, const q4kv_batch* batch, const int32_t* kv_lens, int32_t max_kv_len,
+                                 const int32_t* windows, const void* k_new, const void* v_new, const void* q,
+                                 float softmax_scale, void* out, int32_t out_dtype, float* lse,
+                                 void* workspace, size_t workspace_bytes, int32_t* status_flags, void* stream) {
+  int rc = check_spec(spec);
+  if (rc) return rc;
+  if ((rc = check_batch(batch))) return rc;
+  if (!pool || n_blocks <= 0 || layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > spec->n_layers ||
+      max_kv_len < 0 || !windows)
+    return Q4KV_EINVAL;
+  for (int i = 0; i < layer_count; ++i)
+    if (windows[i] < 0) return Q4KV_EINVAL;
+  if (out_dtype != Q4KV_OUT_F32 && out_dtype != Q4KV_OUT_BF16) return Q4KV_EINVAL;
+  if (batch->n_agents == 0) return Q4KV_OK;
+  if (!kv_lens || !q || !out || !workspace || ((k_new == nullptr) != (v_new == nullptr))) return Q4KV_EINVAL;
+  if (!aligned16(pool) || !aligned16(q) || !aligned16(out) || !aligned16(workspace) || !aligned16(k_new) || !aligned16(v_new))
+    return Q4KV_EINVAL;
+  const int cap = batch->max_blocks * kBlockTokens;
+  if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
+  const Layout y = make_layout(*spec, n_blocks);
+  if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks, layer_count)) return Q4KV_EUNSUPPORTED;
+  if (workspace_bytes < kWorkspaceHeaderBytes + decode_mma_workspace_bytes(y, batch->n_agents, layer_count)) return Q4KV_EWORKSPACE;
+  const cudaError_t e = launch_decode_mma(y, pool, n_blocks, layer_begin, *batch, kv_lens, max_kv_len, windows, layer_count, q,
+                                          softmax_scale, out, out_dtype, lse, workspace, status_flags, (cudaStream_t)stream,
+                                          k_new, v_new);
   return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
 }
 

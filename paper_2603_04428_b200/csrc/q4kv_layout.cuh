@@ -132,13 +132,13 @@ cudaError_t launch_attention_generic(const Layout& y, const void* pool, int n_bl
 
 // tensor-core decode path (GQA shapes with d_qk = d_v in {128, 256}, at most 4 query heads per KV head)
 bool decode_mma_supported(const Layout& y);
-bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks);
+bool decode_mma_fits(const Layout& y, int n_agents, int max_blocks, int layer_count = 1);
 int sm_count();   // SMs of the current device (148 when no device can be asked)
-size_t decode_mma_workspace_bytes(const Layout& y, int n_agents);
+size_t decode_mma_workspace_bytes(const Layout& y, int n_agents, int layer_count = 1);
 cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
-                              const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale,
-                              void* out, int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
-                              const void* k_new = nullptr, const void* v_new = nullptr);
+                              const int32_t* kv_lens, int max_kv_len, const int32_t* windows, int layer_count,
+                              const void* q, float scale, void* out, int out_dtype, float* lse, void* ws, int32_t* flags,
+                              cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr);
 
 // tensor-core prefill path (d_qk = d_v = 128, at most 4 query heads per KV head)
 bool prefill_mma_supported(const Layout& y);

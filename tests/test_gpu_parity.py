@@ -563,6 +563,50 @@ def test_length_beyond_the_stated_maximum_is_flagged_on_every_kernel(H, name):
     p.dc.flags.zero_()
 
 
+
+@pytest.mark.parametrize("spec_args,lens,windows,fused", [
+    ((3, 8, 2, 128, 128, False), [1000, 700, 0, 33, 257], [0, 0, 0], False),
+    ((4, 8, 2, 128, 128, False), [1000, 700, 64], [300, 0, 300, 0], True),        # window and global layers in one launch
+    ((2, 4, 2, 256, 256, False), [1500, 41, 2049], [1024, 0], True),
+])
+def test_layer_batched_decode_equals_the_oracle_layer_by_layer(H, spec_args, lens, windows, fused):
+    """q4kv_decode_attention_layers: all layers of a step in one launch (work list over layers x agents x KV heads),
+    with and without the fused append, against the oracle layer by layer; the pool ends up with the appended rows."""
+    from paper_2603_04428_b200 import binding as B
+    L = spec_args[0]
+    p = Pair(H, spec_args, lens, seed=71, extra_tokens=1).fill()
+    s = p.ospec
+    A = len(lens)
+    scale = 1.0 / math.sqrt(s.d_qk)
+    new_lens = [n + 1 if (fused and n > 0) else n for n in lens]
+    q_all = np.stack([p.q(80 + l, A) for l in range(L)])
+    kb = np.stack([synth.kv_bf16(71, 500 + l, A, s.n_kv_heads, s.d_qk) for l in range(L)])
+    vb = np.stack([synth.kv_bf16(71, 600 + l, A, s.n_kv_heads, s.d_v) for l in range(L)])
+    live = [a for a in range(A) if lens[a] > 0]
+    refs, lses = [], []
+    for l in range(L):
+        if fused:
+            offs = np.concatenate([[0], np.cumsum([1 if a in live else 0 for a in range(A)])]).astype(np.int32)
+            O.quantize_append(p.opool, l, p.tabs, lens, offs, f32(kb[l][live]), f32(vb[l][live]))
+        r, ls = O.decode_attention(p.opool, l, p.tabs, new_lens, windows[l], f32(q_all[l]), scale)
+        refs.append(r); lses.append(ls)
+    out = torch.full((L, A, s.n_q_heads, s.d_v), float("nan"), device="cuda")
+    lse = torch.full((L, A, s.n_q_heads), float("nan"), device="cuda")
+    need = B.q4kv_workspace_bytes_layers(p.dc.spec, A, p.dc.bt.max_blocks * 256, L)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    lens_d = H.dev(np.asarray(new_lens, dtype=np.int32))
+    for rounds in range(2 if not fused else 1):                 # the workspace header is left at zero: a second call works
+        B.q4kv_decode_attention_layers(p.dc.spec, p.dc.pool, p.dc.n_blocks, 0, L, p.dc.bt, lens_d, 0, windows,
+                                       H.bf16_dev(kb) if fused else None, H.bf16_dev(vb) if fused else None,
+                                       H.bf16_dev(q_all), scale, out, B.OUT_F32, lse, ws, p.dc.flags)
+        for l in range(L):
+            assert_attention_close(out[l].cpu().numpy(), refs[l], f"layer {l}")
+            assert_lse_close(lse[l].cpu().numpy(), lses[l])
+    assert int(ws[:B.WORKSPACE_HEADER_BYTES].max()) == 0
+    p.lens = new_lens
+    p.check_packed_equal()
+
+
 # ---- prefill attention --------------------------------------------------------------------------
 @pytest.mark.parametrize("name,prefix,chunk,window", [
     ("gqa64", [300, 70], 40, 0),
