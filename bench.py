@@ -375,9 +375,12 @@ def peaks():
 NOMINAL_BF16_TFLOPS = 2250.0
 
 # DRAM bytes (read + write) of one launch of each workload's dominant kernel, from one profiler capture of that
-# kernel; None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"llama31_8b_decode": None, "gemma3_12b_ragged_decode": None, "dsv2lite_mla_decode": None,
-                     "llama31_8b_chunked_prefill": None, "pack": None, "unpack": None, "append_8x1024": None}
+# kernel; None where no capture of the current kernel exists.  The decode and prefill captures ran the workload with
+# fewer layers (the launch itself is the full-size one, so nothing is scaled); the config-3 figure is a global layer's
+# launch, the MLA figure the attention kernel without its merge launch (4.88 MB more when its records miss L2).
+NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23_969_707, "gemma3_12b_ragged_decode": 364_673_280,
+                     "dsv2lite_mla_decode": 21_437_824, "llama31_8b_chunked_prefill": 240_176_000,
+                     "pack": 254_027_000, "unpack": None, "append_8x1024": 33_632_256}
 
 
 def measure(w, args, local, dist=None, full=True):

@@ -33,9 +33,11 @@
 //     query is scaled per row by a power of two into binary16, so nothing is rounded before the
 //     products, which are exact.  (The 8-bit float forms of mma.sync are not used: on this part
 //     each costs two f16 tensor instructions plus conversions and adds.)
-//   * Scores come out as [8 rows x 8 tokens] fragments whose lane ownership is the B-operand
-//     ownership of the P.V product, so probabilities never move between lanes.  Rows 0..3 are
-//     the query heads and rows 4..7 repeat them; rows 4..7 go on to carry the low half of a
+//   * In the score product the key codes are the A operand (16 tokens x 16 head-dim elements) and the
+//     query the B operand (eight columns: the query heads 0..3 and their repeats), so a KV head's
+//     codes are unpacked once for all its query heads.  The probabilities times the token's value
+//     scale are transposed across the warp (movmatrix) into the B operand of the value product,
+//     whose A operand is the token-packed value words.  Columns 4..7 carry the low half of a
 //     two-term binary16 split of p*s, which makes the value product accurate to ~2^-22 at no
 //     extra MMA.
 #include <climits>
