@@ -55,15 +55,47 @@ def _f16_round_up(x32: np.ndarray) -> np.ndarray:
     return h.astype(np.float16)
 
 
+def _bf16_round_down(x32: np.ndarray) -> np.ndarray:
+    """binary32 -> bfloat16 bit patterns (uint16), rounding toward -infinity.
+
+    bfloat16 is the upper half of binary32, so dropping the lower 16 bits rounds toward zero; a negative value that
+    lost bits moves one step further from zero."""
+    u = np.ascontiguousarray(x32, dtype=np.float32).view(np.uint32)
+    top = u >> np.uint32(16)
+    lost = (u & np.uint32(0xFFFF)) != 0
+    neg = (u >> np.uint32(31)) != 0
+    return (top + (lost & neg)).astype(np.uint16)
+
+
+def _bf16_round_up(x32: np.ndarray) -> np.ndarray:
+    """binary32 -> bfloat16 bit patterns (uint16), rounding toward +infinity."""
+    u = np.ascontiguousarray(x32, dtype=np.float32).view(np.uint32)
+    top = u >> np.uint32(16)
+    lost = (u & np.uint32(0xFFFF)) != 0
+    neg = (u >> np.uint32(31)) != 0
+    return (top + (lost & ~neg)).astype(np.uint16)
+
+
+def sb_values(a: np.ndarray) -> np.ndarray:
+    """Scales or biases as float64 numbers: float16 arrays hold binary16 values, uint16 arrays bfloat16 bit patterns."""
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    assert a.dtype == np.float16
+    return a.astype(np.float64)
+
+
 # ----------------------------------------------------------------------------
 # quantizer (Section 3.2 format; arithmetic = this library's fixed reading)
 # ----------------------------------------------------------------------------
-def quantize_rows(x32: np.ndarray):
+def quantize_rows(x32: np.ndarray, sb_dtype: int = 0):
     """Quantize rows of binary32 values (already exact images of bf16 inputs).
 
     x32: [..., D] float32, D a multiple of 64, finite, |x| <= 65504.
-    Returns (codes uint8 [..., D] in 0..15, scale float16 [..., D/64],
-             bias float16 [..., D/64]).
+    Returns (codes uint8 [..., D] in 0..15, scale [..., D/64], bias [..., D/64]);
+    scale and bias are float16 arrays for sb_dtype 0 (binary16) and uint16 arrays of
+    bfloat16 bit patterns for sb_dtype 1 (Section 3.2 and Appendix A name both types);
+    the sequence is the same with the 16-bit roundings taken in that type.
     Per group of 64 consecutive elements:
         bias  = round_down_f16(min x)            (a zero result is stored as +0)
         r     = f32(max x - f32(bias))
@@ -78,12 +110,18 @@ def quantize_rows(x32: np.ndarray):
     xg = x32.reshape(x32.shape[:-1] + (D // GROUP, GROUP))
     mn = xg.min(axis=-1)
     mx = xg.max(axis=-1)
-    bias = _f16_round_down(mn)
-    bias = np.where(bias == np.float16(0), np.float16(0), bias).astype(np.float16)
-    bias32 = bias.astype(np.float32)
+    if sb_dtype == 0:
+        bias = _f16_round_down(mn)
+        bias = np.where(bias == np.float16(0), np.float16(0), bias).astype(np.float16)
+    else:
+        assert sb_dtype == 1
+        bias = _bf16_round_down(mn)
+        bias = np.where(bias == np.uint16(0x8000), np.uint16(0), bias).astype(np.uint16)
+    bias32 = sb_values(bias).astype(np.float32)          # exact: both 16-bit types embed in binary32
     r = (mx - bias32).astype(np.float32)
-    scale = _f16_round_up((r / np.float32(15.0)).astype(np.float32))
-    scale32 = scale.astype(np.float32)
+    r15 = (r / np.float32(15.0)).astype(np.float32)
+    scale = _f16_round_up(r15) if sb_dtype == 0 else _bf16_round_up(r15)
+    scale32 = sb_values(scale).astype(np.float32)
     safe = np.where(scale32 == 0, np.float32(1.0), scale32)
     t = ((xg - bias32[..., None]).astype(np.float32) / safe[..., None]).astype(np.float32)
     c = np.clip(np.rint(t), 0, 15)
@@ -111,10 +149,10 @@ def unpack_codes(words: np.ndarray) -> np.ndarray:
 
 
 def dequantize(codes: np.ndarray, scale: np.ndarray, bias: np.ndarray) -> np.ndarray:
-    """x_hat = code * scale + bias in float64 (exact: 4-bit x 11-bit + 11-bit)."""
+    """x_hat = code * scale + bias in float64 (4-bit x 11-bit + 11-bit; exact, or at most one rounding of the sum)."""
     D = codes.shape[-1]
     cg = codes.reshape(codes.shape[:-1] + (D // GROUP, GROUP)).astype(np.float64)
-    xh = cg * scale.astype(np.float64)[..., None] + bias.astype(np.float64)[..., None]
+    xh = cg * sb_values(scale)[..., None] + sb_values(bias)[..., None]
     return xh.reshape(codes.shape)
 
 
@@ -124,12 +162,14 @@ def dequantize(codes: np.ndarray, scale: np.ndarray, bias: np.ndarray) -> np.nda
 class Spec:
     """Architectural parameters of one model's cache (the paper's ModelCacheSpec)."""
 
-    def __init__(self, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False):
+    def __init__(self, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False, sb_dtype=0):
         assert n_q_heads % n_kv_heads == 0 and d_qk % GROUP == 0 and d_v % GROUP == 0
+        assert sb_dtype in (0, 1)                        # scale / bias type: 0 binary16, 1 bfloat16
         if v_aliases_k:
             assert d_v <= d_qk
         self.n_layers, self.n_q_heads, self.n_kv_heads = n_layers, n_q_heads, n_kv_heads
         self.d_qk, self.d_v, self.v_aliases_k = d_qk, d_v, bool(v_aliases_k)
+        self.sb_dtype = sb_dtype
 
     @property
     def n_rep(self):
@@ -155,19 +195,21 @@ class Pool:
     Per layer l and physical block b (Appendix A, groups along head_dim):
         Kc [Hkv][256][D/8] uint32, Ks/Kb [Hkv][256][D/64] float16,
         Vc [Hkv][256][Dv/8] uint32, Vs/Vb [Hkv][256][Dv/64] float16 (absent when V aliases K).
+    With bfloat16 scales and biases (sb_dtype 1) the four 16-bit arrays are uint16 bit patterns.
     """
 
     def __init__(self, spec: Spec, n_blocks: int, fill: int = 0):
         s, T = spec, BLOCK_TOKENS
         self.spec, self.n_blocks = spec, n_blocks
         L, H = s.n_layers, s.n_kv_heads
+        sb = np.float16 if s.sb_dtype == 0 else np.uint16
         self.Kc = np.full((L, n_blocks, H, T, s.d_qk // 8), fill, dtype=np.uint32)
-        self.Ks = np.zeros((L, n_blocks, H, T, s.d_qk // GROUP), dtype=np.float16)
-        self.Kb = np.zeros((L, n_blocks, H, T, s.d_qk // GROUP), dtype=np.float16)
+        self.Ks = np.zeros((L, n_blocks, H, T, s.d_qk // GROUP), dtype=sb)
+        self.Kb = np.zeros((L, n_blocks, H, T, s.d_qk // GROUP), dtype=sb)
         if not s.v_aliases_k:
             self.Vc = np.full((L, n_blocks, H, T, s.d_v // 8), fill, dtype=np.uint32)
-            self.Vs = np.zeros((L, n_blocks, H, T, s.d_v // GROUP), dtype=np.float16)
-            self.Vb = np.zeros((L, n_blocks, H, T, s.d_v // GROUP), dtype=np.float16)
+            self.Vs = np.zeros((L, n_blocks, H, T, s.d_v // GROUP), dtype=sb)
+            self.Vb = np.zeros((L, n_blocks, H, T, s.d_v // GROUP), dtype=sb)
 
     def tensors(self):
         t = [self.Kc, self.Ks, self.Kb]
@@ -185,10 +227,10 @@ def quantize_append(pool: Pool, layer, block_tables, pos, new_offs, k_new32, v_n
     """
     s = pool.spec
     A = len(pos)
-    kc, ks, kb = quantize_rows(k_new32)
+    kc, ks, kb = quantize_rows(k_new32, s.sb_dtype)
     kw = pack_codes(kc)
     if not s.v_aliases_k:
-        vc, vs, vb = quantize_rows(v_new32)
+        vc, vs, vb = quantize_rows(v_new32, s.sb_dtype)
         vw = pack_codes(vc)
     for a in range(A):
         for i, row in enumerate(range(new_offs[a], new_offs[a + 1])):
@@ -357,16 +399,17 @@ def container_header(spec: Spec, n_tokens: int) -> bytes:
     nblk = -(-n_tokens // T)
     meta = [("format", "q4kv-1"), ("n_layers", s.n_layers), ("n_q_heads", s.n_q_heads), ("n_kv_heads", s.n_kv_heads),
             ("d_qk", s.d_qk), ("d_v", s.d_v), ("v_aliases_k", int(s.v_aliases_k)), ("group", GROUP),
-            ("block_tokens", T), ("sb_dtype", 0), ("n_tokens", n_tokens)]
+            ("block_tokens", T), ("sb_dtype", s.sb_dtype), ("n_tokens", n_tokens)]
     parts = ['"__metadata__":{' + ",".join(f'"{k}":"{v}"' for k, v in meta) + "}"]
     off = 0
+    sbt = "F16" if s.sb_dtype == 0 else "BF16"
     for l in range(s.n_layers):
         for b in range(nblk):
-            tensors = [("K", "weights", "U32", s.d_qk // 8, 4), ("K", "scales", "F16", s.d_qk // GROUP, 2),
-                       ("K", "biases", "F16", s.d_qk // GROUP, 2)]
+            tensors = [("K", "weights", "U32", s.d_qk // 8, 4), ("K", "scales", sbt, s.d_qk // GROUP, 2),
+                       ("K", "biases", sbt, s.d_qk // GROUP, 2)]
             if not s.v_aliases_k:
-                tensors += [("V", "weights", "U32", s.d_v // 8, 4), ("V", "scales", "F16", s.d_v // GROUP, 2),
-                            ("V", "biases", "F16", s.d_v // GROUP, 2)]
+                tensors += [("V", "weights", "U32", s.d_v // 8, 4), ("V", "scales", sbt, s.d_v // GROUP, 2),
+                            ("V", "biases", sbt, s.d_v // GROUP, 2)]
             for kv, what, dt, last, esz in tensors:
                 nb = H * T * last * esz
                 parts.append(f'"L{l}_B{b}_{kv}_{what}":{{"dtype":"{dt}","shape":[{H},{T},{last}],'

@@ -1022,6 +1022,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       if (!any_left) break;                  // every chunk has been issued
       if (idle > (kSpinLimit >> 2) || *(volatile int*)&sm.abort_flag) {
         if (lane == 0) { sm.abort_flag = 1; raise_flag(P.flags, Q4KV_FLAG_INTERNAL); }
+        // giving up: each lane lets the last copy it issued into its slot land before the CTA lets go of shared memory
+        if (lane < kSlots && round > 0)
+          for (uint32_t i = 0; i < 4096u && !mbar_try_wait(&sm.full[lane], (uint32_t)(round - 1) & 1u); ++i) {}
         break;
       }
     }

@@ -61,7 +61,7 @@ struct ExchangeView {
 // chunk c of the head-block through its own shared-memory copy of the chunk (dynamic smem: 8 * chunk_bytes).  Every
 // global access is a full 16- or 32-byte piece of a contiguous run: the pool chunk is one contiguous range, and each
 // head-dim-packed tensor's part of a chunk is too.
-template <bool kPack>
+template <bool kPack, bool kDense>
 __global__ void __launch_bounds__(kThreads)
 pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restrict__ row, int n_tokens,
                    uint8_t* buf, int32_t* flags, ExchangeView xv) {
@@ -72,7 +72,7 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
   int layer;
   uint8_t *b_kc, *b_ks, *b_kb, *b_vc, *b_vs, *b_vb;      // tensor bases; row index of this head-block's slot 0 below
   uint64_t row0;
-  if (xv.mode == 0) {
+  if (!kDense) {
     layer = xv.layer0 + blockIdx.y;                      // buf starts at layer0
     const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     uint8_t* pb = buf + ((uint64_t)blockIdx.y * nblk + lb) * persisted_block_bytes(y);
@@ -95,7 +95,7 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
     // may be "negative" for the first block of a short agent; only rows of existing tokens are ever touched
     row0 = ((uint64_t)a * y.Hkv + hk) * xv.T + (uint64_t)(xv.T - n_tokens) + (uint64_t)lb * kBlockTokens;
   }
-  const bool whole_blocks = xv.mode == 0;                // the persisted buffer holds whole blocks: rows past the end are zero bytes
+  constexpr bool whole_blocks = !kDense;                // the persisted buffer holds whole blocks: rows past the end are zero bytes
   const int phys = row[lb];
   const bool bad = phys < 0 || phys >= n_blocks;
   if (bad) {
@@ -198,7 +198,7 @@ pack_unpack_kernel(Layout y, uint8_t* pool, int n_blocks, const int32_t* __restr
 }  // namespace
 
 namespace {
-template <bool kPack>
+template <bool kPack, bool kDense>
 cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_t* row, int n_tokens, uint8_t* buf,
                       int32_t* flags, cudaStream_t st, const ExchangeView& xv, int grid_y) {
   static bool configured[64] = {};
@@ -206,13 +206,13 @@ cudaError_t launch_pu(const Layout& y, uint8_t* pool, int n_blocks, const int32_
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(pack_unpack_kernel<kPack>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    e = cudaFuncSetAttribute(pack_unpack_kernel<kPack, kDense>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   const int nblk = (n_tokens + kBlockTokens - 1) / kBlockTokens;   // mode 1: n_tokens is T, the dense row count
   dim3 grid(nblk * y.Hkv, grid_y);
-  pack_unpack_kernel<kPack><<<grid, kThreads, (size_t)kChunksPerBlock * y.chunk_bytes, st>>>(y, pool, n_blocks, row, n_tokens,
+  pack_unpack_kernel<kPack, kDense><<<grid, kThreads, (size_t)kChunksPerBlock * y.chunk_bytes, st>>>(y, pool, n_blocks, row, n_tokens,
                                                                                               buf, flags, xv);
   return cudaGetLastError();
 }
@@ -226,20 +226,20 @@ ExchangeView persisted_view(int layer0) {
 cudaError_t launch_pack(const Layout& y, const void* pool, int n_blocks, const int32_t* row, int n_tokens,
                         void* dst, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  return launch_pu<true>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags, st, persisted_view(0), y.L);
+  return launch_pu<true, false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)dst, flags, st, persisted_view(0), y.L);
 }
 
 cudaError_t launch_unpack(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
                           const int32_t* row, int32_t* flags, cudaStream_t st) {
   if (n_tokens <= 0) return cudaSuccess;
-  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, persisted_view(0), y.L);
+  return launch_pu<false, false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, persisted_view(0), y.L);
 }
 
 // layers [layer0, layer0 + layer_count) only; src points at the persisted bytes of layer0
 cudaError_t launch_unpack_layers(const Layout& y, const void* src, int n_tokens, void* pool, int n_blocks,
                                  const int32_t* row, int32_t* flags, cudaStream_t st, int layer0, int layer_count) {
   if (n_tokens <= 0 || layer_count <= 0) return cudaSuccess;
-  return launch_pu<false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, persisted_view(layer0), layer_count);
+  return launch_pu<false, false>(y, (uint8_t*)pool, n_blocks, row, n_tokens, (uint8_t*)src, flags, st, persisted_view(layer0), layer_count);
 }
 
 // the dense left-padded batch of one layer <-> the pool (to_pool: the paper's merge; else extract, into a zeroed buffer)
@@ -248,8 +248,8 @@ cudaError_t launch_dense_exchange(const Layout& y, void* pool, int n_blocks, int
   if (b.n_agents <= 0 || T <= 0) return cudaSuccess;
   ExchangeView xv;
   xv.mode = 1; xv.layer0 = layer; xv.T = T; xv.max_blocks = b.max_blocks; xv.n_agents = b.n_agents; xv.lens = kv_lens;
-  if (to_pool) return launch_pu<false>(y, (uint8_t*)pool, n_blocks, b.block_tables, T, (uint8_t*)dense, flags, st, xv, b.n_agents);
-  return launch_pu<true>(y, (uint8_t*)pool, n_blocks, b.block_tables, T, (uint8_t*)dense, flags, st, xv, b.n_agents);
+  if (to_pool) return launch_pu<false, true>(y, (uint8_t*)pool, n_blocks, b.block_tables, T, (uint8_t*)dense, flags, st, xv, b.n_agents);
+  return launch_pu<true, true>(y, (uint8_t*)pool, n_blocks, b.block_tables, T, (uint8_t*)dense, flags, st, xv, b.n_agents);
 }
 
 }  // namespace q4kv

@@ -390,7 +390,16 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
       if (old == kWarps * (round + 1) - 1 && k + kSlots < n_chunks) issue(k + kSlots);
     }
   }
-  if (aborted && lane == 0) raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
+  if (aborted && lane == 0) {
+    raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
+    // giving up: the copies already issued into the ring land before this warp lets go of shared memory.  Slot s has
+    // received one copy per completed round of releases plus the first one.
+    for (int s = 0; s < kSlots && s < n_chunks; ++s) {
+      const int later = (n_chunks - 1 - s) / kSlots;                       // refills this slot can ever get
+      const int issued = 1 + min(*(volatile int*)&sm.released[s] / kWarps, later);
+      for (uint32_t i = 0; i < 4096u && !mbar_try_wait(&sm.full[s], (uint32_t)(issued - 1) & 1u); ++i) {}
+    }
+  }
 
   // ---- normalise and write this warp's rows ----
   if (h >= n_rep) return;
