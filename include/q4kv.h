@@ -36,11 +36,13 @@
  *   - The library reads no environment variable; every choice is an argument.
  *
  * Q4 format (Section 3.2): groups of 64 consecutive head-dim elements; per
- * group one binary16 scale and one binary16 bias; 4-bit codes, value =
- * code*scale + bias.  The quantizer's arithmetic is fixed (single binary32
- * operations in this order) so that results are reproducible bit for bit:
- *     bias  = round_toward_minus_inf_f16(min x)      (a zero is stored as +0)
- *     scale = round_toward_plus_inf_f16( f32( f32(max x - bias) / 15 ) )
+ * group one 16-bit scale and one 16-bit bias, both binary16 (sb_dtype 0) or
+ * both bfloat16 (sb_dtype 1; Section 3.2 and Appendix A name both types);
+ * 4-bit codes, value = code*scale + bias.  The quantizer's arithmetic is fixed
+ * (single binary32 operations in this order) so that results are reproducible
+ * bit for bit; the two roundings to 16 bits are taken in the cache's type:
+ *     bias  = round_toward_minus_inf_16(min x)       (a zero is stored as +0)
+ *     scale = round_toward_plus_inf_16( f32( f32(max x - bias) / 15 ) )
  *     code  = clamp( round_half_even( f32( f32(x - bias) / scale ) ), 0, 15 ),
  *             all codes 0 when scale == 0.
  * Inputs must be finite with |x| <= 65504.
@@ -73,7 +75,9 @@ typedef struct {
                             (shared latent of MLA in absorbed form); requires d_v <= d_qk           */
   int32_t group;         /* quantization group, must be 64                                          */
   int32_t block_tokens;  /* tokens per pool block, must be 256                                      */
-  int32_t sb_dtype;      /* scale/bias type: 0 = binary16 (only value supported)                    */
+  int32_t sb_dtype;      /* scale/bias type: 0 = binary16, 1 = bfloat16.  A bfloat16 cache is always
+                            attended by the kernels that multiply the codes exactly (as with
+                            exact_products = 1): its scales can lie outside binary16's range          */
   int32_t exact_products;/* 0: attention kernels may expand the cache into binary16 tiles (one rounding
                             of every dequantized value, see "Accuracy" below); 1: always multiply the
                             4-bit codes exactly.  Ignored by append, pack and unpack.               */
@@ -108,12 +112,14 @@ enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
  *     four query heads per KV head; prefill with d = 128 and exact_products = 1; the shape-agnostic
  *     kernels every other case falls back to): the products are exact, sums are float32, the
  *     probabilities enter the value product as a two-term binary16 pair or as float32.  Error
- *     at most 2e-5 * M + 1e-5, i.e. within 2e-3 for any cache with M <= 64.
+ *     at most 2e-5 * M + 1e-5, i.e. within 2e-3 for any cache with M <= 64.  (An absolute bound:
+ *     the tensor-core kernels carry probability x scale in binary16, so contributions of groups
+ *     whose scale is below 2^-24 vanish; only bfloat16 caches can hold such scales.)
  *   - Kernels that expand the cache into binary16 tiles (prefill with d_qk = d_v = 128 and 1, 2 or 4
  *     query heads per KV head; decode on the MLA-latent cache: V aliasing K, d_qk 576, d_v 512, one
  *     KV head, at most 16 query heads) round every dequantized value once to binary16, a relative
  *     error of 2^-11 at most, and the probabilities likewise.  They are chosen only when
- *     exact_products == 0 and softmax_scale <= 2/sqrt(d_qk).  Their error is at most
+ *     exact_products == 0, sb_dtype == 0 and softmax_scale <= 2/sqrt(d_qk).  Their error is at most
  *     2^-10 * M * (1 + softmax_scale * ||q||_1 * M): the value and probability roundings, plus what
  *     the rounded keys do to the softmax weights.  On caches of unit-variance values (M about 5) the
  *     roundings average out over the attended keys and the measured error is below 3e-4; a cache
@@ -184,8 +190,8 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
  *                 (v_new is ignored, and may be NULL, when V aliases K)
  * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256} with at
  * most four query heads per KV head and V not aliasing K; and the MLA-latent cache (V aliasing K,
- * d_qk 576, d_v 512, one KV head, at most 16 query heads) with exact_products == 0 and
- * softmax_scale^2 * d_qk <= 4.
+ * d_qk 576, d_v 512, one KV head, at most 16 query heads) with exact_products == 0, binary16
+ * scales and biases, and softmax_scale^2 * d_qk <= 4.
  * Anything else returns Q4KV_EUNSUPPORTED and the caller makes the two calls.  Two agents must
  * not share the block that is written. */
 int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,

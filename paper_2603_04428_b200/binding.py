@@ -46,8 +46,8 @@ class Spec(ctypes.Structure):
         "exact_products")]
 
     @classmethod
-    def make(cls, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False, exact_products=False):
-        return cls(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), 64, 256, 0,
+    def make(cls, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k=False, exact_products=False, sb_dtype=0):
+        return cls(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), 64, 256, int(sb_dtype),
                    int(bool(exact_products)))
 
 

@@ -14,6 +14,12 @@ namespace q4kv {
 
 namespace {
 
+// a (scale, bias) pair of the cache as two binary32 numbers: binary16 or bfloat16 halves
+__device__ inline float2 sb_pair(uint32_t u, bool bf16) {
+  if (bf16) return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+  return __half22float2(*reinterpret_cast<const __half2*>(&u));
+}
+
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kMaxDvPerLane = 16;      // Dv <= 512
@@ -69,7 +75,7 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
   const int item = blockIdx.x, h = blockIdx.y, split = blockIdx.z;
   const int hk = h / y.n_rep;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int D = y.D, Dv = y.Dv, G = y.G, kw = D / 8;
+  const int D = y.D, Dv = y.Dv, G = y.G;
   const int nd = Dv / 32;
 
   ItemInfo it;
@@ -106,14 +112,14 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
     float s = 0.f;
     {
       const uint32_t* kc = reinterpret_cast<const uint32_t*>(chunk + y.off_kc);
-      const __half2* ksb = reinterpret_cast<const __half2*>(chunk + y.off_ksb);
+      const uint32_t* ksb = reinterpret_cast<const uint32_t*>(chunk + y.off_ksb);
       for (int p = 0; p < 2 * G; ++p) {
         const int gi = p >> 1, i2 = p & 1;
         const int w = 8 * gi + 4 * i2 + t;
         float sc = 0.f, bi = 0.f;
         uint32_t word = 0;
         if (valid) {
-          const float2 f = __half22float2(ksb[sb_offset(tau0 + k, gi, G)]);
+          const float2 f = sb_pair(ksb[sb_offset(tau0 + k, gi, G)], y.sb_bf16 != 0);
           sc = f.x; bi = f.y;
           word = kc[k_word_offset(tau0 + k, w, G)];
         }
@@ -161,7 +167,7 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
       }
     } else {
       const uint32_t* vc = reinterpret_cast<const uint32_t*>(chunk + y.off_vc);
-      const __half2* vsb = reinterpret_cast<const __half2*>(chunk + y.off_vsb);
+      const uint32_t* vsb = reinterpret_cast<const uint32_t*>(chunk + y.off_vsb);
 #pragma unroll
       for (int i = 0; i < kMaxDvPerLane; ++i) {
         if (i >= nd) break;
@@ -171,7 +177,7 @@ attn_generic_kernel(Layout y, const uint8_t* __restrict__ pool, int n_blocks, in
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           if (p[kk] != 0.f) {     // invalid tokens may hold garbage scale bits
-            const float2 f = __half22float2(vsb[sb_offset(tau0 + kk, gi, y.Gv)]);
+            const float2 f = sb_pair(vsb[sb_offset(tau0 + kk, gi, y.Gv)], y.sb_bf16 != 0);
             a = fmaf(p[kk], fmaf((float)((word >> (4 * kk)) & 15u), f.x, f.y), a);
           }
         }

@@ -45,7 +45,7 @@ std::string header_json(const q4kv_spec& s, int n_tokens) {
                 s.block_tokens, s.sb_dtype, n_tokens);
   std::string js = buf;
   js.reserve(js.size() + (size_t)s.n_layers * nblk * 6 * 100);
-  const char* sbt = "F16";
+  const char* sbt = s.sb_dtype == 1 ? "BF16" : "F16";
   uint64_t off = 0;
   const uint64_t rows = (uint64_t)y.Hkv * kBlockTokens;
   for (int l = 0; l < s.n_layers; ++l)
@@ -67,7 +67,7 @@ size_t padded_header_bytes(size_t json_bytes) { return (8 + json_bytes + 63) & ~
 
 bool spec_ok(const q4kv_spec* s) {
   return s && s->n_layers > 0 && s->n_q_heads > 0 && s->n_kv_heads > 0 && s->d_qk > 0 && s->d_v > 0 && s->group == 64 &&
-         s->block_tokens == 256 && s->sb_dtype == 0 && s->d_qk % 64 == 0 && s->d_v % 64 == 0 &&
+         s->block_tokens == 256 && (s->sb_dtype == 0 || s->sb_dtype == 1) && s->d_qk % 64 == 0 && s->d_v % 64 == 0 &&
          s->n_q_heads % s->n_kv_heads == 0 && s->d_qk <= 1024 && s->d_v <= 512 && (!s->v_aliases_k || s->d_v <= s->d_qk);
 }
 

@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[e] = 0.f;
       }
-      const QuantOut qo = quantize_eight(x);             // eight lanes per group of 64; 72 words = 9 whole groups
+      const QuantOut qo = quantize_eight(x, false);             // eight lanes per group of 64; 72 words = 9 whole groups
       if (w < kD / 8) {
         sm.new_words[w] = qo.word;
         if ((w & 7) == 0) sm.new_sb[w >> 3] = *reinterpret_cast<const uint32_t*>(&qo.sb);

@@ -119,18 +119,6 @@ __device__ inline void bulk_load(void* dst_smem, const void* src, uint32_t bytes
 __device__ inline void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ inline void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// D = A(16x16 f16, rows 8..15 zero) * B(16x8 f16); only rows 0..7 of D are meaningful
-__device__ inline void mma_f16_rows8_first(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
-}
-// D += A(16x16 f16, rows 8..15 zero) * B(16x8 f16)
-__device__ inline void mma_f16_rows8(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
-}
 __device__ inline void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -141,7 +129,6 @@ __device__ inline float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
-__device__ inline float2 h2_to_f2(uint32_t u) { return __half22float2(*reinterpret_cast<__half2*>(&u)); }
 // half2(lo = a, hi = b), both rounded toward zero
 __device__ inline uint32_t f32x2_to_h2_rz(float a, float b) {
   uint32_t r;
@@ -487,7 +474,7 @@ __device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, c
 #pragma unroll
       for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(u[i] << 16); x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
     }
-    const QuantOut qo = quantize_eight(x);
+    const QuantOut qo = quantize_eight(x, y.sb_bf16 != 0);
     const uint32_t sb = *reinterpret_cast<const uint32_t*>(&qo.sb);
     if (!is_v) {
       const uint32_t at = y.off_kc + 4u * k_word_offset(tau, w, G);
@@ -544,7 +531,7 @@ __device__ inline uint32_t transpose_8x8_b16(uint32_t a) {
 //   2 tid + 1.  The probabilities, multiplied by the token's value scale, are packed two columns to a register and
 //   transposed across the warp (movmatrix) into the B operand of the value product, whose A operand is the token-packed
 //   value words; columns 4..7 carry the low half of the two-term split of p * s.
-template <int G>
+template <int G, bool kBf>
 __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
                                               const uint4* qb, const float (&qs)[2][G], const float (&kap)[2],
                                               uint32_t split_mask, WarpState<G>& st) {
@@ -589,13 +576,13 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
       float ks[G], kb[G];
       if (G == 2) {
         const uint2 v = *reinterpret_cast<const uint2*>(ksb + (i * 8 + g) * 8);
-        const float2 f0 = h2_to_f2(v.x), f1 = h2_to_f2(v.y);
+        const float2 f0 = sb_to_f2<kBf>(v.x), f1 = sb_to_f2<kBf>(v.y);
         ks[0] = f0.x; kb[0] = f0.y; ks[1] = f1.x; kb[1] = f1.y;
       } else {
         const uint4 v = *reinterpret_cast<const uint4*>(ksb + (i * 8 + g) * 16);
         const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(u[gi]); ks[gi] = f.x; kb[gi] = f.y; }
+        for (int gi = 0; gi < 4; ++gi) { const float2 f = sb_to_f2<kBf>(u[gi]); ks[gi] = f.x; kb[gi] = f.y; }
       }
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
@@ -649,13 +636,13 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
     float vs[Gv], vb[Gv];
     if (G == 2) {
       const uint2 v = *reinterpret_cast<const uint2*>(vsb + (i * 8 + g) * 8);
-      const float2 f0 = h2_to_f2(v.x), f1 = h2_to_f2(v.y);
+      const float2 f0 = sb_to_f2<kBf>(v.x), f1 = sb_to_f2<kBf>(v.y);
       vs[0] = f0.x; vb[0] = f0.y; vs[1] = f1.x; vb[1] = f1.y;
     } else {
       const uint4 v = *reinterpret_cast<const uint4*>(vsb + (i * 8 + g) * 16);
       const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int gi = 0; gi < 4; ++gi) { const float2 f = h2_to_f2(u[gi]); vs[gi] = f.x; vb[gi] = f.y; }
+      for (int gi = 0; gi < 4; ++gi) { const float2 f = sb_to_f2<kBf>(u[gi]); vs[gi] = f.x; vb[gi] = f.y; }
     }
     if (edge) {
       const int pos = pos0 + 4 * g + i;
@@ -890,7 +877,7 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
   }
 }
 
-template <int G, int NW>
+template <int G, int NW, bool kBf>
 __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __grid_constant__ DecodeParams P) {
   constexpr int D = 64 * G, Dv = D, Gv = G;
   using S = Smem<G, NW>;
@@ -1189,7 +1176,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       // the chunk that receives the step's new token is usable once the planner warp has quantized the token into it
       if (j == seg.tail_pos && !spin_until_ge(&sm.patched[slot], round + 1, &sm.abort_flag)) { aborted = true; continue; }
       __threadfence_block();
-      process_chunk<G>(sm.ring + (size_t)slot * kChunkBytes, seg.chunk_at(j) * 32, seg.lo, seg.n, g, tid, qa, qs, kap,
+      process_chunk<G, kBf>(sm.ring + (size_t)slot * kChunkBytes, seg.chunk_at(j) * 32, seg.lo, seg.n, g, tid, qa, qs, kap,
                        split_mask, st);
     }
     __syncwarp();
@@ -1198,7 +1185,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   if (aborted && lane == 0) raise_flag(P.flags, Q4KV_FLAG_INTERNAL);
 }
 
-template <int G, int NW>
+template <int G, int NW, bool kBf>
 cudaError_t launch_g(const DecodeParams& P, int grid, bool pdl, cudaStream_t st) {
   static bool configured[64] = {};     // the attribute is per function and device: set it once for each
   const size_t smem = sizeof(Smem<G, NW>);
@@ -1206,7 +1193,7 @@ cudaError_t launch_g(const DecodeParams& P, int grid, bool pdl, cudaStream_t st)
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(decode_mma_kernel<G, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(decode_mma_kernel<G, NW, kBf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -1220,7 +1207,7 @@ cudaError_t launch_g(const DecodeParams& P, int grid, bool pdl, cudaStream_t st)
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, NW>, P);
+  return cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, NW, kBf>, P);
 }
 
 }  // namespace
@@ -1281,8 +1268,11 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
   P.k_new = (const uint16_t*)k_new; P.v_new = (const uint16_t*)v_new;
   const int n_sm = sm_count();
   const int grid = (int)(units < n_sm ? (units < 1 ? 1 : units) : n_sm);
-  return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128>(P, grid, true, st)
-                  : launch_g<4, Q4KV_DECODE_WARPS_D256>(P, grid, true, st);
+  if (y.sb_bf16)
+    return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128, true>(P, grid, true, st)
+                    : launch_g<4, Q4KV_DECODE_WARPS_D256, true>(P, grid, true, st);
+  return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128, false>(P, grid, true, st)
+                  : launch_g<4, Q4KV_DECODE_WARPS_D256, false>(P, grid, true, st);
 }
 
 }  // namespace q4kv

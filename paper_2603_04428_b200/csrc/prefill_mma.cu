@@ -21,6 +21,7 @@
 //   * The score fragment of two adjacent key tiles is the A fragment of the value product, as in any
 //     register-resident flash attention, so probabilities never leave their lane.
 #include "q4kv_layout.cuh"
+#include "quantize_core.cuh"
 
 namespace q4kv {
 
@@ -118,7 +119,7 @@ struct PrefillSmem {
   int abort_flag;
 };
 
-template <int R>
+template <int R, bool kBf>
 __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_constant__ PrefillParams P) {
   constexpr int D = 128, Dv = 128, G = 2;
   using S = PrefillSmem<R>;
@@ -276,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 sb = ksb4[i * 4 + tid];
-          const float2 e0g0 = h2_to_f2(sb.x), e0g1 = h2_to_f2(sb.y), e1g0 = h2_to_f2(sb.z), e1g1 = h2_to_f2(sb.w);
+          const float2 e0g0 = sb_to_f2<kBf>(sb.x), e0g1 = sb_to_f2<kBf>(sb.y), e1g0 = sb_to_f2<kBf>(sb.z), e1g1 = sb_to_f2<kBf>(sb.w);
 #pragma unroll
           for (int r = 0; r < 2; ++r) {
             const float t0 = fmaf(acc[i][1][2 * r], e0g1.x, acc[i][0][2 * r] * e0g0.x);
@@ -336,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 sb = vsb4[i * 4 + tid];
-          float2 v[2][G] = {{h2_to_f2(sb.x), h2_to_f2(sb.y)}, {h2_to_f2(sb.z), h2_to_f2(sb.w)}};   // [e][group] = (scale, bias)
+          float2 v[2][G] = {{sb_to_f2<kBf>(sb.x), sb_to_f2<kBf>(sb.y)}, {sb_to_f2<kBf>(sb.z), sb_to_f2<kBf>(sb.w)}};   // [e][group] = (scale, bias)
           if (tail) {
 #pragma unroll
             for (int e = 0; e < 2; ++e)
@@ -438,7 +439,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
     }
 }
 
-template <int R>
+template <int R, bool kBf>
 cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   static bool configured[64] = {};
   const size_t smem = sizeof(PrefillSmem<R>);
@@ -446,7 +447,7 @@ cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(prefill_mma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(prefill_mma_kernel<R, kBf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -460,7 +461,7 @@ cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, prefill_mma_kernel<R>, P);
+  return cudaLaunchKernelEx(&cfg, prefill_mma_kernel<R, kBf>, P);
 }
 
 }  // namespace
@@ -477,7 +478,7 @@ cudaError_t launch_prefill_mma(const Layout& y, const void* pool, int n_blocks, 
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
   constexpr int R = 2;
   const dim3 grid((max_q_len + 32 * R - 1) / (32 * R), y.Hkv, b.n_agents);
-  return launch_r<R>(P, grid, st);
+  return y.sb_bf16 ? launch_r<R, true>(P, grid, st) : launch_r<R, false>(P, grid, st);
 }
 
 }  // namespace q4kv

@@ -11,7 +11,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 int check_spec(const q4kv_spec* s) {
   if (!s) return Q4KV_EINVAL;
   if (s->n_layers <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->d_qk <= 0 || s->d_v <= 0) return Q4KV_EINVAL;
-  if (s->group != 64 || s->block_tokens != 256 || s->sb_dtype != 0) return Q4KV_EUNSUPPORTED;
+  if (s->group != 64 || s->block_tokens != 256 || (s->sb_dtype != 0 && s->sb_dtype != 1)) return Q4KV_EUNSUPPORTED;
   if (s->exact_products != 0 && s->exact_products != 1) return Q4KV_EINVAL;
   if (s->d_qk % 64 || s->d_v % 64 || s->n_q_heads % s->n_kv_heads) return Q4KV_EUNSUPPORTED;
   if (s->d_qk > 1024 || s->d_v > 512) return Q4KV_EUNSUPPORTED;
@@ -44,9 +44,11 @@ size_t workspace_need(const Layout& y, int n_agents, int max_kv_len, int total_q
 
 // The kernels that expand the cache into binary16 tiles round each dequantized element once; they are taken only when
 // the spec allows it and the softmax scale is at most 2 / sqrt(d_qk) (the error a rounded key leaves in a score grows
-// with the scale).  Everything else multiplies the codes exactly.
+// with the scale).  Everything else multiplies the codes exactly.  A bfloat16 scale or bias can lie outside binary16's
+// range, so those caches never take the tile kernels.
 bool tiles_allowed(const q4kv_spec* s, float softmax_scale) {
-  return s->exact_products == 0 && softmax_scale > 0.f && softmax_scale * softmax_scale * (float)s->d_qk <= 4.f;
+  return s->exact_products == 0 && s->sb_dtype == 0 && softmax_scale > 0.f &&
+         softmax_scale * softmax_scale * (float)s->d_qk <= 4.f;
 }
 
 }  // namespace

@@ -49,6 +49,7 @@ constexpr int kMaxTicketPairs = (int)(kWorkspaceHeaderBytes / sizeof(int32_t));
 
 struct Layout {
   int L, Hq, Hkv, D, Dv, G, Gv, alias, n_rep;
+  int sb_bf16;            // scales and biases are bfloat16 (else binary16)
   // byte offsets inside a chunk
   uint32_t off_kc, off_ksb, off_vc, off_vsb, chunk_bytes, head_block_bytes;
   uint64_t block_bytes;   // all KV heads
@@ -60,6 +61,7 @@ __host__ __device__ inline Layout make_layout(const q4kv_spec& s, int n_blocks) 
   y.L = s.n_layers; y.Hq = s.n_q_heads; y.Hkv = s.n_kv_heads; y.D = s.d_qk; y.Dv = s.d_v;
   y.G = s.d_qk / kGroup; y.Gv = s.d_v / kGroup; y.alias = s.v_aliases_k ? 1 : 0;
   y.n_rep = s.n_q_heads / s.n_kv_heads;
+  y.sb_bf16 = s.sb_dtype == 1 ? 1 : 0;
   y.off_kc = 0;
   y.off_ksb = kChunkTokens * (y.D / 2);
   y.off_vc = y.off_ksb + kChunkTokens * 4 * y.G;

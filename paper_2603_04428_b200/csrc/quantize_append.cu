@@ -114,7 +114,7 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
     }
 #pragma unroll
     for (int r = 0; r < M; ++r) {
-      const QuantOut o = quantize_eight(x[r]);
+      const QuantOut o = quantize_eight(x[r], y.sb_bf16 != 0);
       if (!live[r]) continue;
       const UnitInfo un = s_unit[r];
       const int slot0 = un.first & 255;                 // the octet lies inside one 32-token chunk
@@ -124,10 +124,10 @@ quantize_append_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, int n_a
         uint8_t* vcodes = vcodes_all + (size_t)r * 8 * y.Dv;
 #pragma unroll
         for (int e = 0; e < 8; ++e) vcodes[i * y.Dv + 8 * w + e] = (o.word >> (4 * e)) & 15u;
-        if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_vsb)[sb_offset(tau, w >> 3, y.Gv)] = o.sb;
+        if ((w & 7) == 0) reinterpret_cast<uint32_t*>(chunk + y.off_vsb)[sb_offset(tau, w >> 3, y.Gv)] = o.sb;
       } else {
         reinterpret_cast<uint32_t*>(chunk + y.off_kc)[k_word_offset(tau, w, y.G)] = o.word;
-        if ((w & 7) == 0) reinterpret_cast<__half2*>(chunk + y.off_ksb)[sb_offset(tau, w >> 3, y.G)] = o.sb;
+        if ((w & 7) == 0) reinterpret_cast<uint32_t*>(chunk + y.off_ksb)[sb_offset(tau, w >> 3, y.G)] = o.sb;
       }
     }
   }
@@ -251,7 +251,7 @@ quantize_append_bulk_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, in
     const uint32_t mnb = *reinterpret_cast<const uint32_t*>(&mn2), mxb = *reinterpret_cast<const uint32_t*>(&mx2);
     const float mn = fminf(__uint_as_float(mnb << 16), __uint_as_float(mnb & 0xffff0000u));
     const float mx = fmaxf(__uint_as_float(mxb << 16), __uint_as_float(mxb & 0xffff0000u));
-    const GroupScale gs = group_scale(mn, mx);
+    const GroupScale gs = group_scale(mn, mx, y.sb_bf16 != 0);
     uint32_t cw[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) cw[j] = 0u;
@@ -285,7 +285,7 @@ quantize_append_bulk_kernel(Layout y, uint8_t* pool, int n_blocks, int layer, in
         cw[j] = w;
       }
     }
-    const uint32_t sb = (uint32_t)__half_as_ushort(gs.hs) | ((uint32_t)__half_as_ushort(gs.hb) << 16);
+    const uint32_t sb = gs.hs | (gs.hb << 16);
     if (active && !is_v) {
       // words w = 8 gi + 4 i2 + t sit in 16-byte pieces of four (group, half) words: this lane's pair is 8 bytes
       uint32_t* kc = reinterpret_cast<uint32_t*>(chunk + y.off_kc);

@@ -1,31 +1,60 @@
 // The quantizer of Section 3.2 as a device function shared by the kernels that write the cache: affine 4-bit
-// codes over groups of 64, binary16 scale and bias.  Every arithmetic step is a single rounded binary32 operation
-// in a fixed order, so that codes, scales and biases are reproducible bit for bit:
-//   bias = RD_f16(min) (-0 -> +0), scale = RU_f16((max - bias) / 15), code = clamp(rne((x - bias) / scale), 0, 15),
-//   all codes 0 when scale = 0.
+// codes over groups of 64, 16-bit scale and bias (binary16, or bfloat16: the section names both).  Every arithmetic
+// step is a single rounded binary32 operation in a fixed order, so that codes, scales and biases are reproducible
+// bit for bit:
+//   bias = RD_16(min) (-0 -> +0), scale = RU_16((max - bias) / 15), code = clamp(rne((x - bias) / scale), 0, 15),
+//   all codes 0 when scale = 0; RD_16 / RU_16 round toward -inf / +inf into the 16-bit type.
 #pragma once
 #include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace q4kv {
 
-struct QuantOut { uint32_t word; __half2 sb; };
+struct QuantOut { uint32_t word; uint32_t sb; };         // sb: scale in the low 16 bits, bias in the high 16 bits
 
-// Scale and bias of one group from its minimum and maximum (the fixed binary32 sequence of the header comment).
-struct GroupScale { __half hs, hb; float sf, bf; };
-__device__ inline GroupScale group_scale(float mn, float mx) {
+// bfloat16 is the upper half of binary32: dropping the lower half rounds toward zero, and a value that lost bits on
+// the far side of zero from the rounding direction moves one step away from zero.
+__device__ inline uint32_t bf16_bits_rd(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u >> 16) + (((u & 0xFFFFu) != 0u && (u >> 31) != 0u) ? 1u : 0u);
+}
+__device__ inline uint32_t bf16_bits_ru(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u >> 16) + (((u & 0xFFFFu) != 0u && (u >> 31) == 0u) ? 1u : 0u);
+}
+
+// Scale and bias of one group from its minimum and maximum (the fixed binary32 sequence of the header comment):
+// their 16-bit patterns and their values.
+struct GroupScale { uint32_t hs, hb; float sf, bf; };
+__device__ inline GroupScale group_scale(float mn, float mx, bool bf16) {
   GroupScale gs;
-  gs.hb = __float2half_rd(mn);
-  if (__half2float(gs.hb) == 0.0f) gs.hb = __ushort_as_half((unsigned short)0);   // -0 -> +0
-  gs.bf = __half2float(gs.hb);
-  const float r = __fsub_rn(mx, gs.bf);
-  gs.hs = __float2half_ru(__fdiv_rn(r, 15.0f));
-  gs.sf = __half2float(gs.hs);
+  if (bf16) {
+    gs.hb = bf16_bits_rd(mn);
+    if ((gs.hb & 0x7FFFu) == 0u) gs.hb = 0u;                                      // -0 -> +0
+    gs.bf = __uint_as_float(gs.hb << 16);
+    gs.hs = bf16_bits_ru(__fdiv_rn(__fsub_rn(mx, gs.bf), 15.0f));
+    gs.sf = __uint_as_float(gs.hs << 16);
+  } else {
+    __half hb = __float2half_rd(mn);
+    if (__half2float(hb) == 0.0f) hb = __ushort_as_half((unsigned short)0);       // -0 -> +0
+    gs.hb = __half_as_ushort(hb);
+    gs.bf = __half2float(hb);
+    const __half hs = __float2half_ru(__fdiv_rn(__fsub_rn(mx, gs.bf), 15.0f));
+    gs.hs = __half_as_ushort(hs);
+    gs.sf = __half2float(hs);
+  }
   return gs;
 }
 
+// A (scale, bias) pair of the cache as two binary32 numbers.
+template <bool kBf16>
+__device__ __forceinline__ float2 sb_to_f2(uint32_t u) {
+  if (kBf16) return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+  return __half22float2(*reinterpret_cast<const __half2*>(&u));
+}
+
 // x[8]: eight consecutive elements owned by this lane; the 8 lanes of a group cooperate.
-__device__ inline QuantOut quantize_eight(const float x[8]) {
+__device__ inline QuantOut quantize_eight(const float x[8], bool bf16) {
   float mn = x[0], mx = x[0];
 #pragma unroll
   for (int i = 1; i < 8; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
@@ -34,8 +63,7 @@ __device__ inline QuantOut quantize_eight(const float x[8]) {
     mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   }
-  const GroupScale gs = group_scale(mn, mx);
-  const __half hb = gs.hb, hs = gs.hs;
+  const GroupScale gs = group_scale(mn, mx, bf16);
   const float bf = gs.bf, sf = gs.sf;
   uint32_t w = 0;
   if (sf != 0.0f) {
@@ -57,7 +85,7 @@ __device__ inline QuantOut quantize_eight(const float x[8]) {
   }
   QuantOut o;
   o.word = w;
-  o.sb = __halves2half2(hs, hb);
+  o.sb = gs.hs | (gs.hb << 16);
   return o;
 }
 

@@ -23,8 +23,8 @@ def bf16_dev(bits: np.ndarray) -> torch.Tensor:
 
 class DeviceCache:
     def __init__(self, n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k, n_blocks, block_tables: np.ndarray,
-                 fill_byte: int | None = 0xFF, exact_products: bool = False):
-        self.spec = B.Spec.make(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k, exact_products)
+                 fill_byte: int | None = 0xFF, exact_products: bool = False, sb_dtype: int = 0):
+        self.spec = B.Spec.make(n_layers, n_q_heads, n_kv_heads, d_qk, d_v, v_aliases_k, exact_products, sb_dtype)
         self.n_blocks = int(n_blocks)
         nbytes = B.q4kv_pool_bytes(self.spec, self.n_blocks)
         assert nbytes > 0, "unsupported spec"
@@ -135,6 +135,10 @@ class DeviceCache:
     def restore(self, agent, image: torch.Tensor, staging_layers: int = 0):
         """Scatter a file image (pinned host uint8 tensor) into the agent's blocks; returns the token count."""
         spec, n_tokens, off = B.q4kv_container_read_header(bytes(image[:min(image.numel(), 1 << 22)].numpy()))
+        same = all(getattr(spec, f) == getattr(self.spec, f) for f in (
+            "n_layers", "n_q_heads", "n_kv_heads", "d_qk", "d_v", "v_aliases_k", "group", "block_tokens", "sb_dtype"))
+        if not same:
+            raise B.Q4KVError(-1, "restore: the image was written for another cache spec")
         pb = B.q4kv_packed_bytes(self.spec, n_tokens)
         packed = image[off:off + pb]
         if packed.data_ptr() % 16:

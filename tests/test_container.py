@@ -59,17 +59,18 @@ def test_oracle_container_opens_with_the_safetensors_package(args, n_tokens):
 
 @pytest.mark.parametrize("args,n_tokens", [((32, 32, 8, 128, 128, False), 4096), ((2, 8, 2, 128, 128, False), 300),
                                            ((27, 16, 1, 576, 512, True), 1000), ((1, 4, 4, 192, 128, False), 1)])
-def test_library_header_equals_the_oracles_and_reads_back(args, n_tokens):
-    ospec = O.Spec(*args)
-    spec = B.Spec.make(*args)
+@pytest.mark.parametrize("sb_dtype", [0, 1])
+def test_library_header_equals_the_oracles_and_reads_back(args, n_tokens, sb_dtype):
+    ospec = O.Spec(*args, sb_dtype=sb_dtype)
+    spec = B.Spec.make(*args, sb_dtype=sb_dtype)
     want = O.container_header(ospec, n_tokens)
     got = B.q4kv_container_write_header(spec, n_tokens)
     assert B.q4kv_container_header_bytes(spec, n_tokens) == len(want)
     assert got == want
     back, nt, off = B.q4kv_container_read_header(want)
     assert nt == n_tokens and off == len(want)
-    assert (back.n_layers, back.n_q_heads, back.n_kv_heads, back.d_qk, back.d_v, back.v_aliases_k) == \
-        (args[0], args[1], args[2], args[3], args[4], int(args[5]))
+    assert (back.n_layers, back.n_q_heads, back.n_kv_heads, back.d_qk, back.d_v, back.v_aliases_k, back.sb_dtype) == \
+        (args[0], args[1], args[2], args[3], args[4], int(args[5]), sb_dtype)
     # a header that is not this library's canonical text is refused
     bad = bytearray(want)
     i = bad.index(b'"L0_B0_K_weights"')

@@ -52,15 +52,16 @@ class Pair:
     """The same cache on both sides: an oracle pool and a device pool behind one block table."""
 
     def __init__(self, H, spec_args, lens, seed, spare_blocks=3, extra_tokens=0, gain=1.0, outlier_frac=0.0,
-                 exact_products=False):
+                 exact_products=False, sb_dtype=0):
         L, Hq, Hkv, D, Dv, alias = spec_args
         self.H, self.lens, self.seed, self.gain, self.outlier_frac = H, list(lens), seed, gain, outlier_frac
-        self.ospec = O.Spec(L, Hq, Hkv, D, Dv, alias)
+        self.ospec = O.Spec(L, Hq, Hkv, D, Dv, alias, sb_dtype=sb_dtype)
         need = sum(-(-(n + extra_tokens) // 256) for n in lens)
         self.n_blocks = need + spare_blocks
         self.tabs = synth.block_tables(seed, 99, lens, self.n_blocks, extra_tokens=extra_tokens)
         self.opool = O.Pool(self.ospec, self.n_blocks, fill=0xFFFFFFFF)
-        self.dc = H.DeviceCache(L, Hq, Hkv, D, Dv, alias, self.n_blocks, self.tabs, exact_products=exact_products)
+        self.dc = H.DeviceCache(L, Hq, Hkv, D, Dv, alias, self.n_blocks, self.tabs, exact_products=exact_products,
+                                sb_dtype=sb_dtype)
 
     def kv(self, layer, agent, n):
         s = self.ospec
