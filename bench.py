@@ -7,7 +7,7 @@ agent, then decode attention of one query per agent over the whole Q4 cache.  On
 layers.  The metric is the achieved HBM bandwidth over the algorithmic bytes of the step (each
 needed Q4 row read once + q + out + new rows); agent-steps/s rides along.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4|5] [--impl reference]
 
 N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no collective.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
@@ -600,7 +600,7 @@ def main():
     }
     if rank == 0 and world == 1 and default_run and not args.no_all_configs:
         allc = {}
-        for idx in (2, 3, 4):
+        for idx in (2, 3, 4, 5):
             wi = synth.workload(idx)
             ri = measure(wi, args, local, None, full=False)
             units_i, roof_i = roofline_of(wi, ri)
@@ -713,7 +713,7 @@ def fused_update_and_fetch(w):
     if w.v_aliases_k:      # the MLA-latent cache (at the usual softmax scales)
         return (w.d_qk, w.d_v, w.n_kv_heads) == (576, 512, 1) and w.n_q_heads <= 16 and w.softmax_scale ** 2 * w.d_qk <= 4
     n_rep = w.n_q_heads // w.n_kv_heads
-    return w.d_qk == w.d_v and w.d_qk in (128, 256) and n_rep <= 4
+    return n_rep <= 4 and ((w.d_qk == w.d_v and w.d_qk in (128, 256)) or (w.d_qk, w.d_v) == (192, 128))
 
 
 def dw_launches(w, two_calls=False):

@@ -340,7 +340,10 @@ struct Walker {
 // The kernel
 // ---------------------------------------------------------------------------------------------
 
-__host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }   // acc[Dv], m, l, pad: 16-byte multiples
+__host__ __device__ constexpr int kRecStride(int Dv) { return Dv + 4; }
+// The kernel is instantiated by the number of key groups G: 2 and 4 are the symmetric shapes (d_qk = d_v = 64 G), 3 is
+// the asymmetric per-head MLA cache of Section 3.6 (d_qk 192, d_v 128).
+__host__ __device__ constexpr int value_groups(int G) { return G == 3 ? 2 : G; }   // acc[Dv], m, l, pad: 16-byte multiples
 constexpr int kQBufs = 4;      // query-fragment buffers (segments s, s+4, ... share one)
 constexpr int kOffCap = 256;   // entries of the planner's offset table (a ring over the CTA's chunk indices)
 constexpr int kTailQ = 8;      // chunks waiting for the planner's patch (planning stops while the queue is full)
@@ -359,9 +362,9 @@ constexpr int kSmemBudget = 232448 - 2048;   // 227 KB per CTA, less the small a
 
 template <int G, int NW>
 struct Smem {
-  static constexpr int D = 64 * G;
-  static constexpr int kChunkBytes = 32 * (D / 2 + 4 * G) * 2;
-  static constexpr int kMergeStride = D + 8;            // acc[Dv], m, l, bias[Gv], pad
+  static constexpr int D = 64 * G, Gv = value_groups(G), Dv = 64 * Gv;
+  static constexpr int kChunkBytes = 32 * (D / 2 + 4 * G + Dv / 2 + 4 * Gv);
+  static constexpr int kMergeStride = Dv + 8;           // acc[Dv], m, l, bias[Gv], pad
   static constexpr int kMBufs = (G == 4 && NW > 7) ? 1 : 2;                  // deposit buffers (consecutive segments alternate)
   static constexpr int kRingBudget = kSmemBudget - kMBufs * NW * 4 * kMergeStride * 4 - kQBufs * 2 * G * 32 * 16;
   static constexpr int kSlots = kRingBudget / kChunkBytes < 32 ? kRingBudget / kChunkBytes : 32;   // one producer lane per slot
@@ -388,17 +391,18 @@ struct Smem {
 // m, l and the bias sums are per column, partial over the lane's tokens.
 template <int G>
 struct WarpState {
-  float m[2], l_e[2], l_o[2], bias_e[2][G], bias_o[2][G];
-  float o[4 * G][4];
+  static constexpr int Gv = value_groups(G);
+  float m[2], l_e[2], l_o[2], bias_e[2][Gv], bias_o[2][Gv];
+  float o[4 * Gv][4];
   __device__ void reset() {
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
       m[c] = -INFINITY; l_e[c] = 0.f; l_o[c] = 0.f;
 #pragma unroll
-      for (int i = 0; i < G; ++i) { bias_e[c][i] = 0.f; bias_o[c][i] = 0.f; }
+      for (int i = 0; i < Gv; ++i) { bias_e[c][i] = 0.f; bias_o[c][i] = 0.f; }
     }
 #pragma unroll
-    for (int i = 0; i < 4 * G; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
+    for (int i = 0; i < 4 * Gv; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
   }
 };
 
@@ -414,10 +418,13 @@ __device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], f
                                          const uint16_t* __restrict__ q, int Hq, int n_rep, float scale_log2, int a,
                                          int hk, int lane) {
   constexpr int D = 64 * G;
-  for (int base = 0; base < n_rep * (D / 8); base += 32) {
+  // a row's D / 8 words sit in kRowLanes consecutive lanes (a power of two, so that the row maximum is a butterfly)
+  constexpr int kRowLanes = D / 8 <= 16 ? 16 : 32;
+  for (int base = 0; base < n_rep * kRowLanes; base += 32) {
     const int idx = base + lane;
-    const bool valid = idx < n_rep * (D / 8);
-    const int h = valid ? idx / (D / 8) : 0, w = idx % (D / 8);
+    const int h_raw = idx / kRowLanes, w = idx % kRowLanes;
+    const bool valid = h_raw < n_rep && w < D / 8;
+    const int h = valid ? h_raw : 0;
     const uint16_t* qrow = q + ((size_t)a * Hq + (size_t)hk * n_rep + h) * D;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (valid) v = *reinterpret_cast<const uint4*>(qrow + 8 * w);
@@ -430,7 +437,7 @@ __device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], f
 #pragma unroll
     for (int i = 0; i < 8; ++i) { mx = fmaxf(mx, fabsf(x[i])); sum += x[i]; }
 #pragma unroll
-    for (int o = D / 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = kRowLanes / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
 #pragma unroll
     for (int o = 4; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);   // 8 words per group
     if (!valid) continue;
@@ -455,27 +462,30 @@ __device__ __noinline__ void stage_query(uint4 (*qfrag)[32], float (*qsum)[G], f
 // ones -- and then lets the chunk's consumer go on.  Every chunk is held by exactly one CTA of the grid, so nobody else
 // reads or writes these words during the launch.
 // Eight consecutive lanes own one 64-element group; the 8-lane shuffles never straddle K and V (D / 8 is a multiple
-// of 16).  The value codes are token-packed: one nibble of each of the row's D words is replaced.
+// of 8).  The value codes are token-packed: one nibble of each of the row's d_v words is replaced.
 template <int G>
 __device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, const Layout& y,
                                               const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                                               int a, int hk, int tau, int lane) {
-  constexpr int D = 64 * G, W = D / 8;                   // words per row
-  const size_t row = ((size_t)a * y.Hkv + hk) * D;
+  constexpr int D = 64 * G, Gv = value_groups(G), Dv = 64 * Gv, W = D / 8, Wv = Dv / 8;   // words per K row, per V row
+  const size_t head = (size_t)a * y.Hkv + hk;
 #pragma unroll
-  for (int base = 0; base < 2 * W; base += 32) {
+  for (int base = 0; base < W + Wv; base += 32) {
     const int idx = base + lane;
+    const bool live = idx < W + Wv;                      // W + Wv need not be a multiple of 32: idle lanes quantize zeros
     const bool is_v = idx >= W;
-    const int w = idx % W;
+    const int w = is_v ? (idx - W) % Wv : idx;
     float x[8];
     {
-      const uint4 v = *reinterpret_cast<const uint4*>((is_v ? v_new : k_new) + row + 8 * w);
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (live) v = *reinterpret_cast<const uint4*>(is_v ? v_new + head * Dv + 8 * w : k_new + head * D + 8 * w);
       const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(u[i] << 16); x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
     }
     const QuantOut qo = quantize_eight(x, y.sb_bf16 != 0);
-    const uint32_t sb = *reinterpret_cast<const uint32_t*>(&qo.sb);
+    const uint32_t sb = qo.sb;
+    if (!live) continue;
     if (!is_v) {
       const uint32_t at = y.off_kc + 4u * k_word_offset(tau, w, G);
       *reinterpret_cast<uint32_t*>(chunk + at) = qo.word;
@@ -496,7 +506,7 @@ __device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, c
         *reinterpret_cast<uint32_t*>(gchunk + at) = nw;
       }
       if ((w & 7) == 0) {
-        const uint32_t sat = y.off_vsb + 4u * sb_offset(tau, w >> 3, G);
+        const uint32_t sat = y.off_vsb + 4u * sb_offset(tau, w >> 3, Gv);
         *reinterpret_cast<uint32_t*>(chunk + sat) = sb;
         *reinterpret_cast<uint32_t*>(gchunk + sat) = sb;
       }
@@ -509,9 +519,10 @@ __device__ __noinline__ void append_new_token(uint8_t* chunk, uint8_t* gchunk, c
 // chunk finds them in L2.
 template <int G>
 __device__ inline void prefetch_new_token(const uint16_t* k_new, const uint16_t* v_new, int Hkv, int a, int hk, int lane) {
-  constexpr int D = 64 * G, kLines = D * 2 / 128;        // 128-byte lines per row
-  if (lane < 2 * kLines) {
-    const uint16_t* p = (lane < kLines ? k_new : v_new) + ((size_t)a * Hkv + hk) * D + (lane % kLines) * 64;
+  constexpr int D = 64 * G, Dv = 64 * value_groups(G), kLines = D * 2 / 128, kLinesV = Dv * 2 / 128;   // 128-byte lines per row
+  if (lane < kLines + kLinesV) {
+    const size_t head = (size_t)a * Hkv + hk;
+    const uint16_t* p = lane < kLines ? k_new + head * D + lane * 64 : v_new + head * Dv + (lane - kLines) * 64;
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
   }
 }
@@ -535,7 +546,7 @@ template <int G, bool kBf>
 __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, int key_lo, int key_n, int g, int tid,
                                               const uint4* qb, const float (&qs)[2][G], const float (&kap)[2],
                                               uint32_t split_mask, WarpState<G>& st) {
-  constexpr int D = 64 * G, Dv = D, Gv = G;
+  constexpr int D = 64 * G, Gv = value_groups(G), Dv = 64 * Gv;
   const uint4* kc4 = reinterpret_cast<const uint4*>(chunk);
   const uint8_t* ksb = chunk + 32 * (D / 2);
   const uint4* vc4 = reinterpret_cast<const uint4*>(chunk + 32 * (D / 2) + 128 * G);
@@ -551,10 +562,10 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) { acc[pr][gi][0] = 0.f; acc[pr][gi][1] = 0.f; acc[pr][gi][2] = 0.f; acc[pr][gi][3] = 0.f; }
 #pragma unroll
-    for (int half = 0; half < G / 2; ++half) {           // groups 2*half, 2*half+1
+    for (int half = 0; half < G / 2; ++half) {           // groups 2*half, 2*half+1: a 16-byte piece per token row
       uint4 kw[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) kw[i] = kc4[((i * (G / 2) + half) * 8 + g) * 4 + tid];
+      for (int i = 0; i < 4; ++i) kw[i] = kc4[i * 16 * G + half * 32 + g * 4 + tid];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {                      // word p = 4*half + j: group 2*half + j/2
         const uint4 b = qb[(4 * half + j) * 32];
@@ -570,11 +581,34 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
         }
       }
     }
+    if (G & 1) {                                         // the last group of an odd count: an 8-byte piece per token row
+      uint2 kw[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        kw[i] = reinterpret_cast<const uint2*>(chunk)[(i * 64 * G + (G / 2) * 128) / 2 + g * 4 + tid];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const uint4 b = qb[(4 * (G / 2) + j) * 32];
+#pragma unroll
+        for (int pr = 0; pr < 2; ++pr) {
+          const uint32_t w0 = j == 0 ? kw[2 * pr].x : kw[2 * pr].y;
+          const uint32_t w1 = j == 0 ? kw[2 * pr + 1].x : kw[2 * pr + 1].y;
+          const uint32_t h0 = w0 >> 8, h1 = w1 >> 8;
+          float (&a)[4] = acc[pr][G - 1];
+          mma_f16(a, w0 & kMaskLo, w1 & kMaskLo, w0 & kMaskHi, w1 & kMaskHi, b.x, b.y);
+          mma_f16(a, h0 & kMaskLo, h1 & kMaskLo, h0 & kMaskHi, h1 & kMaskHi, b.z, b.w);
+        }
+      }
+    }
     // the token's scale meets the integer dot products, its bias the per-group query sums
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float ks[G], kb[G];
-      if (G == 2) {
+      if (G == 3) {
+        const uint32_t* v = reinterpret_cast<const uint32_t*>(ksb + (i * 8 + g) * 12);
+#pragma unroll
+        for (int gi = 0; gi < 3; ++gi) { const float2 f = sb_to_f2<kBf>(v[gi]); ks[gi] = f.x; kb[gi] = f.y; }
+      } else if (G == 2) {
         const uint2 v = *reinterpret_cast<const uint2*>(ksb + (i * 8 + g) * 8);
         const float2 f0 = sb_to_f2<kBf>(v.x), f1 = sb_to_f2<kBf>(v.y);
         ks[0] = f0.x; kb[0] = f0.y; ks[1] = f1.x; kb[1] = f1.y;
@@ -634,7 +668,7 @@ __device__ __forceinline__ void process_chunk(const uint8_t* chunk, int pos0, in
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     float vs[Gv], vb[Gv];
-    if (G == 2) {
+    if (Gv == 2) {
       const uint2 v = *reinterpret_cast<const uint2*>(vsb + (i * 8 + g) * 8);
       const float2 f0 = sb_to_f2<kBf>(v.x), f1 = sb_to_f2<kBf>(v.y);
       vs[0] = f0.x; vb[0] = f0.y; vs[1] = f1.x; vb[1] = f1.y;
@@ -700,7 +734,7 @@ __device__ inline void store_out(const DecodeParams& P, size_t index, float v) {
 template <int G, int NW>
 __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* epilogues_word, int use, const DecodeParams& P,
                                               const Segment& seg, int cta, const Partition& part, int lane) {
-  constexpr int Dv = 64 * G, V = Dv / 128;
+  constexpr int Dv = 64 * value_groups(G), V = Dv / 128;
   constexpr int kStride = Dv + 8;
   static_assert(NW <= 32, "one lane per deposit in the weight pass");
   const Layout& y = P.y;
@@ -799,7 +833,7 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
   const float* base = P.partials + (size_t)(pair + c_first) * rstride;
   // The records sit in L2, a microsecond away: all heads travel together, and the first batch of record loads is issued
   // before the (m, l) pass, so that a pair with few records costs two round trips in all.
-  constexpr int RB = G == 2 ? 5 : 2;
+  constexpr int RB = V == 1 ? 5 : 2;
   float mr[RB][4];
   float4 xv[RB][4][V];
   auto load_batch = [&](int rb) {
@@ -879,7 +913,7 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
 
 template <int G, int NW, bool kBf>
 __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __grid_constant__ DecodeParams P) {
-  constexpr int D = 64 * G, Dv = D, Gv = G;
+  constexpr int Gv = value_groups(G), Dv = 64 * Gv;
   using S = Smem<G, NW>;
   constexpr int kSlots = S::kSlots, kChunkBytes = S::kChunkBytes, kMBufs = S::kMBufs;
   static_assert(kSlots >= NW + 4, "the ring must hold the chunks in work and a few in flight");
@@ -1226,7 +1260,7 @@ int sm_count() {
 }
 
 bool decode_mma_supported(const Layout& y) {
-  return !y.alias && y.D == y.Dv && (y.D == 128 || y.D == 256) && y.n_rep <= 4;
+  return !y.alias && y.n_rep <= 4 && ((y.D == y.Dv && (y.D == 128 || y.D == 256)) || (y.D == 192 && y.Dv == 128));
 }
 
 // the kernel counts work units in 32 bits and keeps one arrival counter per (layer of the call, agent, KV head) in
@@ -1269,10 +1303,12 @@ cudaError_t launch_decode_mma(const Layout& y, const void* pool, int n_blocks, i
   const int n_sm = sm_count();
   const int grid = (int)(units < n_sm ? (units < 1 ? 1 : units) : n_sm);
   if (y.sb_bf16)
-    return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128, true>(P, grid, true, st)
-                    : launch_g<4, Q4KV_DECODE_WARPS_D256, true>(P, grid, true, st);
-  return y.G == 2 ? launch_g<2, Q4KV_DECODE_WARPS_D128, false>(P, grid, true, st)
-                  : launch_g<4, Q4KV_DECODE_WARPS_D256, false>(P, grid, true, st);
+    return y.G == 2   ? launch_g<2, Q4KV_DECODE_WARPS_D128, true>(P, grid, true, st)
+           : y.G == 3 ? launch_g<3, Q4KV_DECODE_WARPS_D128, true>(P, grid, true, st)
+                      : launch_g<4, Q4KV_DECODE_WARPS_D256, true>(P, grid, true, st);
+  return y.G == 2   ? launch_g<2, Q4KV_DECODE_WARPS_D128, false>(P, grid, true, st)
+         : y.G == 3 ? launch_g<3, Q4KV_DECODE_WARPS_D128, false>(P, grid, true, st)
+                    : launch_g<4, Q4KV_DECODE_WARPS_D256, false>(P, grid, true, st);
 }
 
 }  // namespace q4kv

@@ -125,7 +125,8 @@ class Workload:
 
 
 def workload(index: int) -> Workload:
-    """The five configurations, 0-based."""
+    """The five benchmark configurations, 0-based, and (index 5) the per-head MLA cache of Section 3.6 at the sizes of
+    configuration 4: keys of 192 dims (3 groups), values of 128 (2 groups), 16 KV heads."""
     seed = BASE_SEED + index
     if index == 0:
         return Workload("tiny_gqa_decode", 1, 8, 2, 128, 128, False, [1000, 700], 1,
@@ -143,4 +144,7 @@ def workload(index: int) -> Workload:
     if index == 4:
         return Workload("llama31_8b_chunked_prefill", 32, 32, 8, 128, 128, False, [8192] * 8, 1024,
                         softmax_scale=1.0 / math.sqrt(128), seed=seed, kind="prefill")
+    if index == 5:
+        return Workload("dsv2lite_perhead_mla_decode", 27, 16, 16, 192, 128, False, [16384] * 4, 1,
+                        softmax_scale=1.0 / math.sqrt(192), seed=seed)
     raise IndexError(index)

@@ -253,6 +253,7 @@ def test_config1_tiny_decode_append_and_roundtrip(H):
     ("mla", [600, 70], 0),
     ("asym", [400, 300], 0),
     ("asym", [400, 300], 100),
+    ("asym", [3000, 1, 31, 32, 33, 255, 256, 257, 0], 0),
 ])
 def test_decode_matches_oracle(H, name, lens, window):
     p = Pair(H, SPECS[name], lens, seed=31).fill()
@@ -271,6 +272,7 @@ def test_decode_matches_oracle(H, name, lens, window):
     ((1, 16, 8, 256, 256, False), [30000, 9000], 0),       # ~66 chunks per CTA through a 12-slot ring
     ((1, 32, 8, 128, 128, False), [40000, 23000], 0),      # ~106 chunks per CTA through a 32-slot ring
     ((1, 16, 8, 256, 256, False), [30000, 9000], 1024),
+    ((1, 16, 16, 192, 128, False), [20000, 5000], 0),      # d_qk 192 / d_v 128, one query head per KV head
 ])
 def test_decode_long_contexts_wrap_the_ring(H, spec_args, lens, window):
     """Every CTA streams several times its shared-memory ring: slot reuse, ragged split and merge across many CTAs."""
@@ -409,6 +411,8 @@ def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
     ("gqa256", [1500, 41, 2049], 1024),
     ("mla", [1000, 700, 0, 63, 64, 65, 129, 31, 32, 33], 0),       # the latent cache: 64-key block and chunk edges
     ("mla", [2500, 300, 4000], 200),
+    ("asym", [1000, 700, 0, 255, 256, 257, 31, 32, 33], 0),        # d_qk 192 / d_v 128: the per-head MLA cache
+    ("asym", [600, 90], 100),
 ])
 def test_update_and_fetch_in_one_launch(H, name, lens, window):
     """q4kv_append_decode_attention: same pool bytes as quantize-append, same attention as decode, step after step."""
@@ -569,6 +573,7 @@ def test_length_beyond_the_stated_maximum_is_flagged_on_every_kernel(H, name):
     ((3, 8, 2, 128, 128, False), [1000, 700, 0, 33, 257], [0, 0, 0], False),
     ((4, 8, 2, 128, 128, False), [1000, 700, 64], [300, 0, 300, 0], True),        # window and global layers in one launch
     ((2, 4, 2, 256, 256, False), [1500, 41, 2049], [1024, 0], True),
+    ((2, 16, 16, 192, 128, False), [700, 33, 300], [0, 0], True),     # the per-head MLA cache, 16 KV heads
 ])
 def test_layer_batched_decode_equals_the_oracle_layer_by_layer(H, spec_args, lens, windows, fused):
     """q4kv_decode_attention_layers: all layers of a step in one launch (work list over layers x agents x KV heads),
