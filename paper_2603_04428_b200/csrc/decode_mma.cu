@@ -365,7 +365,9 @@ struct Smem {
   static constexpr int D = 64 * G, Gv = value_groups(G), Dv = 64 * Gv;
   static constexpr int kChunkBytes = 32 * (D / 2 + 4 * G + Dv / 2 + 4 * Gv);
   static constexpr int kMergeStride = Dv + 8;           // acc[Dv], m, l, bias[Gv], pad
-  static constexpr int kMBufs = (G == 4 && NW > 7) ? 1 : 2;                  // deposit buffers (consecutive segments alternate)
+  // deposit buffers (consecutive segments alternate).  One at d = 256: its 30 KB are worth more as four ring slots (20
+  // instead of 16: the global layer of the ragged benchmark runs 1.2 % faster, bytes in flight being what limits it)
+  static constexpr int kMBufs = G == 4 ? 1 : 2;
   static constexpr int kRingBudget = kSmemBudget - kMBufs * NW * 4 * kMergeStride * 4 - kQBufs * 2 * G * 32 * 16;
   static constexpr int kSlots = kRingBudget / kChunkBytes < 32 ? kRingBudget / kChunkBytes : 32;   // one producer lane per slot
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
