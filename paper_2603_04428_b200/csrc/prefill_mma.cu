@@ -105,26 +105,26 @@ struct PrefillParams {
   int32_t* flags;
 };
 
-template <int R>
+template <int R, int G>
 struct PrefillSmem {
-  static constexpr int kChunkBytes = 4608;               // d = 128: 32 * (64 + 8) * 2
+  static constexpr int kChunkBytes = 2304 * G;           // 32 * (32 G + 4 G) * 2: 4608 at d = 128, 9216 at d = 256
   static constexpr int kRows = kWarps * R * 16;
   alignas(128) uint8_t ring[kSlots * kChunkBytes];
-  alignas(16) uint4 qfrag[kWarps][R][4][2][32];          // [warp][row tile][key word][half of the word][lane] = A registers
+  alignas(16) uint4 qfrag[kWarps][R][2 * G][2][32];      // [warp][row tile][key word][half of the word][lane] = A registers
   float kappa[kRows];                                    // scale_log2 * 2^(ex + 13) of each row
-  float qsum[kRows][2];                                  // scale_log2 * per-group sums of the true query row
+  float qsum[kRows][G];                                  // scale_log2 * per-group sums of the true query row
   alignas(8) uint64_t full[kSlots];
   int released[kSlots];                                  // warps that have finished with each slot (monotonic)
   int bad[kSlots];
   int abort_flag;
 };
 
-template <int R, bool kBf>
+template <int R, int G, bool kBf>
 __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_constant__ PrefillParams P) {
-  constexpr int D = 128, Dv = 128, G = 2;
-  using S = PrefillSmem<R>;
+  constexpr int D = 64 * G, Dv = D;
+  constexpr int kRowWords = D / 8;                       // 16 or 32: the words of a query row sit in that many consecutive lanes
+  using S = PrefillSmem<R, G>;
   constexpr int kChunkBytes = S::kChunkBytes;
-  constexpr int kTileQ = 32 * R;                         // queries per CTA
   extern __shared__ __align__(128) uint8_t smem_raw[];
   S& sm = *reinterpret_cast<S*>(smem_raw);
 
@@ -144,11 +144,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
   // ---- this CTA's queries and key range ----
   const int q0 = P.q_offs[a], q_len = P.q_offs[a + 1] - q0;
   const int kv_len = P.kv_lens[a];
-  const int i_min = qt * kTileQ;
+  // the eight warps are (head slot, query sub-tile) pairs: 4 x 2 for three or four query heads per KV head, 2 x 4 for
+  // two, 1 x 8 for one, so that no warp works on a head that does not exist
+  const int hs = n_rep > 2 ? 4 : n_rep;
+  const int tile_q = (kWarps / hs) * 16 * R;             // queries per CTA
+  const int i_min = qt * tile_q;
   if (i_min >= q_len) return;                            // uniform: no thread has passed a barrier yet
   const bool bad_len = kv_len < 0 || kv_len > P.max_blocks * kBlockTokens || q_len > kv_len;
   if (bad_len && threadIdx.x == 0) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
-  const int i_max = min(q_len, i_min + kTileQ) - 1;
+  const int i_max = min(q_len, i_min + tile_q) - 1;
   const int prefix = kv_len - q_len;                     // query i sits at position prefix + i
   const int c_end = bad_len ? 0 : (prefix + i_max) / 32 + 1;
   const int c_begin = (bad_len || P.window == 0) ? 0 : max(0, prefix + i_min - P.window + 1) >> 5;
@@ -174,10 +178,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
   if (warp == 0 && lane < kSlots && lane < n_chunks) issue(lane);
 
   // ---- stage the query rows: binary16 in A-fragment order, per-row factor and group sums ----
-  for (int item = threadIdx.x; item < S::kRows * 16; item += kThreads) {
-    const int row = item >> 4, w = item & 15;
+  for (int item = threadIdx.x; item < S::kRows * kRowWords; item += kThreads) {
+    const int row = item / kRowWords, w = item % kRowWords;
     const int wv = row / (16 * R), rt = (row >> 4) % R, rr = row & 15;
-    const int h = wv & 3, qhalf = wv >> 2;
+    const int h = wv % hs, qhalf = wv / hs;
     const int i = i_min + (qhalf * R + rt) * 16 + rr;
     const bool valid = i < q_len && h < n_rep && !bad_len;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -190,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
 #pragma unroll
     for (int j = 0; j < 8; ++j) { mx = fmaxf(mx, fabsf(x[j])); sum += x[j]; }
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));   // 16 lanes per row
+    for (int o = kRowWords / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));   // the lanes of a row
 #pragma unroll
     for (int o = 4; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);           // 8 words per group
     int ex = (int)((__float_as_uint(mx) >> 23) & 255u) - 127;
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
   __syncthreads();
 
   // ---- per-warp rows: head h, R tiles of 16 consecutive queries; a lane owns rows g and g+8 of each tile ----
-  const int h = warp & 3, qhalf = warp >> 2;
+  const int h = warp % hs, qhalf = warp / hs;
   float kap[R][2], qs[R][2][G], m_run[R][2], l_e[R][2], l_o[R][2], bias_e[R][2][G], bias_o[R][2][G];
   float o[R][Dv / 8][4];
 #pragma unroll
@@ -244,140 +248,320 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
       const int pos0 = (c_begin + k) * 32;
       const bool tail = pos0 + 32 > kv_len;              // slots past the cache end may hold stale bytes
 
-      uint32_t apv[R][G][2][4], apl[R][G][2][4];         // value-product A operands, high and low term: [tile][group][MMA][register]
-      bool active[R];
-#pragma unroll
-      for (int rt = 0; rt < R; ++rt) {
-        const int pq_lo = prefix + i_min + (qhalf * R + rt) * 16, pq_hi = pq_lo + 15;
-        active[rt] = pos0 <= pq_hi && (W == 0 || pos0 + 31 > pq_lo - W);
-        if (!active[rt]) continue;
-        const bool need_mask = pos0 + 31 > pq_lo || (W > 0 && pos0 <= pq_hi - W);
-        // ---- integer dot products per key tile and group ----
-        float acc[4][G][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int gi = 0; gi < G; ++gi) { acc[i][gi][0] = 0.f; acc[i][gi][1] = 0.f; acc[i][gi][2] = 0.f; acc[i][gi][3] = 0.f; }
-        uint4 kw[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kw[i] = kc4[(i * 8 + g) * 4 + tid];
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint4 a1 = sm.qfrag[warp][rt][ks][0][lane], a2 = sm.qfrag[warp][rt][ks][1][lane];
-#pragma unroll
+      // Two forms of the same step.  d = 128 (two 16-row tiles per warp): all groups' operands of the value product
+      // are built first.  d = 256 (one tile per warp, 128 accumulator registers per lane): keys and values are taken
+      // two groups and one group at a time, which keeps the live registers within the file.
+      if (G == 2) {
+        uint32_t apv[R][G][2][4], apl[R][G][2][4];         // value-product A operands, high and low term: [tile][group][MMA][register]
+        bool active[R];
+  #pragma unroll
+        for (int rt = 0; rt < R; ++rt) {
+          const int pq_lo = prefix + i_min + (qhalf * R + rt) * 16, pq_hi = pq_lo + 15;
+          active[rt] = pos0 <= pq_hi && (W == 0 || pos0 + 31 > pq_lo - W);
+          if (!active[rt]) continue;
+          const bool need_mask = pos0 + 31 > pq_lo || (W > 0 && pos0 <= pq_hi - W);
+          // ---- integer dot products per key tile and group ----
+          float acc[4][G][4];
+  #pragma unroll
+          for (int i = 0; i < 4; ++i)
+  #pragma unroll
+            for (int gi = 0; gi < G; ++gi) { acc[i][gi][0] = 0.f; acc[i][gi][1] = 0.f; acc[i][gi][2] = 0.f; acc[i][gi][3] = 0.f; }
+          uint4 kw[4];
+  #pragma unroll
+          for (int i = 0; i < 4; ++i) kw[i] = kc4[(i * 8 + g) * 4 + tid];
+  #pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint4 a1 = sm.qfrag[warp][rt][ks][0][lane], a2 = sm.qfrag[warp][rt][ks][1][lane];
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t w = ks == 0 ? kw[i].x : ks == 1 ? kw[i].y : ks == 2 ? kw[i].z : kw[i].w;
+              const uint32_t wh = w >> 8;
+              mma_f16(acc[i][ks >> 1], a1, w & kMaskLo, w & kMaskHi);
+              mma_f16(acc[i][ks >> 1], a2, wh & kMaskLo, wh & kMaskHi);
+            }
+          }
+          // ---- scores in log2 units, mask, online softmax ----
+          float s[4][2][2];                                // [tile][token e][row r]
+  #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const uint32_t w = ks == 0 ? kw[i].x : ks == 1 ? kw[i].y : ks == 2 ? kw[i].z : kw[i].w;
-            const uint32_t wh = w >> 8;
-            mma_f16(acc[i][ks >> 1], a1, w & kMaskLo, w & kMaskHi);
-            mma_f16(acc[i][ks >> 1], a2, wh & kMaskLo, wh & kMaskHi);
+            const uint4 sb = ksb4[i * 4 + tid];
+            const float2 e0g0 = sb_to_f2<kBf>(sb.x), e0g1 = sb_to_f2<kBf>(sb.y), e1g0 = sb_to_f2<kBf>(sb.z), e1g1 = sb_to_f2<kBf>(sb.w);
+  #pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              const float t0 = fmaf(acc[i][1][2 * r], e0g1.x, acc[i][0][2 * r] * e0g0.x);
+              const float t1 = fmaf(acc[i][1][2 * r + 1], e1g1.x, acc[i][0][2 * r + 1] * e1g0.x);
+              const float u0 = fmaf(qs[rt][r][1], e0g1.y, qs[rt][r][0] * e0g0.y);
+              const float u1 = fmaf(qs[rt][r][1], e1g1.y, qs[rt][r][0] * e1g0.y);
+              s[i][0][r] = fmaf(kap[rt][r], t0, u0);
+              s[i][1][r] = fmaf(kap[rt][r], t1, u1);
+            }
           }
-        }
-        // ---- scores in log2 units, mask, online softmax ----
-        float s[4][2][2];                                // [tile][token e][row r]
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 sb = ksb4[i * 4 + tid];
-          const float2 e0g0 = sb_to_f2<kBf>(sb.x), e0g1 = sb_to_f2<kBf>(sb.y), e1g0 = sb_to_f2<kBf>(sb.z), e1g1 = sb_to_f2<kBf>(sb.w);
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            const float t0 = fmaf(acc[i][1][2 * r], e0g1.x, acc[i][0][2 * r] * e0g0.x);
-            const float t1 = fmaf(acc[i][1][2 * r + 1], e1g1.x, acc[i][0][2 * r + 1] * e1g0.x);
-            const float u0 = fmaf(qs[rt][r][1], e0g1.y, qs[rt][r][0] * e0g0.y);
-            const float u1 = fmaf(qs[rt][r][1], e1g1.y, qs[rt][r][0] * e1g0.y);
-            s[i][0][r] = fmaf(kap[rt][r], t0, u0);
-            s[i][1][r] = fmaf(kap[rt][r], t1, u1);
+          if (need_mask) {
+  #pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              const int pq = pq_lo + g + 8 * r;
+  #pragma unroll
+              for (int i = 0; i < 4; ++i)
+  #pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const int pos = pos0 + 8 * tid + 4 * e + i;
+                  if (pos > pq || (W > 0 && pos <= pq - W)) s[i][e][r] = -INFINITY;
+                }
+            }
           }
-        }
-        if (need_mask) {
-#pragma unroll
+          float corr[2];
+  #pragma unroll
           for (int r = 0; r < 2; ++r) {
-            const int pq = pq_lo + g + 8 * r;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                const int pos = pos0 + 8 * tid + 4 * e + i;
-                if (pos > pq || (W > 0 && pos <= pq - W)) s[i][e][r] = -INFINITY;
+            float cm = fmaxf(fmaxf(fmaxf(s[0][0][r], s[0][1][r]), fmaxf(s[1][0][r], s[1][1][r])),
+                             fmaxf(fmaxf(s[2][0][r], s[2][1][r]), fmaxf(s[3][0][r], s[3][1][r])));
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+            float m_new = fmaxf(m_run[rt][r], cm);
+            if (m_new == -INFINITY) m_new = 0.f;
+            corr[r] = fast_exp2(m_run[rt][r] - m_new);
+            m_run[rt][r] = m_new;
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float off = (i & 1) ? m_new + 4.f : m_new;   // odd tiles: p / 16 (their value codes carry a factor 16)
+              s[i][0][r] = fast_exp2(s[i][0][r] - off);
+              s[i][1][r] = fast_exp2(s[i][1][r] - off);
+            }
+            l_e[rt][r] = fmaf(l_e[rt][r], corr[r], (s[0][0][r] + s[0][1][r]) + (s[2][0][r] + s[2][1][r]));
+            l_o[rt][r] = fmaf(l_o[rt][r], corr[r], (s[1][0][r] + s[1][1][r]) + (s[3][0][r] + s[3][1][r]));
+          }
+          if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+  #pragma unroll
+            for (int gi = 0; gi < G; ++gi) {
+              bias_e[rt][0][gi] *= corr[0]; bias_o[rt][0][gi] *= corr[0];
+              bias_e[rt][1][gi] *= corr[1]; bias_o[rt][1][gi] *= corr[1];
+            }
+  #pragma unroll
+            for (int nt = 0; nt < Dv / 8; ++nt) {
+              o[rt][nt][0] *= corr[0]; o[rt][nt][1] *= corr[0]; o[rt][nt][2] *= corr[1]; o[rt][nt][3] *= corr[1];
+            }
+          }
+          // ---- p * s_v per group as a two-term binary16 sum (high part + rounded remainder): the A operands of the
+          // value product, which is then good to ~2^-22 whatever the magnitude of the cached values ----
+  #pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 sb = vsb4[i * 4 + tid];
+            float2 v[2][G] = {{sb_to_f2<kBf>(sb.x), sb_to_f2<kBf>(sb.y)}, {sb_to_f2<kBf>(sb.z), sb_to_f2<kBf>(sb.w)}};   // [e][group] = (scale, bias)
+            if (tail) {
+  #pragma unroll
+              for (int e = 0; e < 2; ++e)
+                if (pos0 + 8 * tid + 4 * e + i >= kv_len) { v[e][0] = make_float2(0.f, 0.f); v[e][1] = make_float2(0.f, 0.f); }
+            }
+  #pragma unroll
+            for (int gi = 0; gi < G; ++gi)
+  #pragma unroll
+              for (int r = 0; r < 2; ++r) {
+                const float x0 = s[i][0][r] * v[0][gi].x, x1 = s[i][1][r] * v[1][gi].x;
+                const uint32_t hi = f32x2_to_h2(x0, x1);
+                const float2 hf = h2_to_f2(hi);
+                apv[rt][gi][i >> 1][(i & 1) * 2 + r] = hi;
+                apl[rt][gi][i >> 1][(i & 1) * 2 + r] = f32x2_to_h2(x0 - hf.x, x1 - hf.y);
+                const float b = fmaf(s[i][0][r], v[0][gi].y, s[i][1][r] * v[1][gi].y);
+                if (i & 1) bias_o[rt][r][gi] += b; else bias_e[rt][r][gi] += b;
               }
           }
         }
-        float corr[2];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          float cm = fmaxf(fmaxf(fmaxf(s[0][0][r], s[0][1][r]), fmaxf(s[1][0][r], s[1][1][r])),
-                           fmaxf(fmaxf(s[2][0][r], s[2][1][r]), fmaxf(s[3][0][r], s[3][1][r])));
-          cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-          cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-          float m_new = fmaxf(m_run[rt][r], cm);
-          if (m_new == -INFINITY) m_new = 0.f;
-          corr[r] = fast_exp2(m_run[rt][r] - m_new);
-          m_run[rt][r] = m_new;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float off = (i & 1) ? m_new + 4.f : m_new;   // odd tiles: p / 16 (their value codes carry a factor 16)
-            s[i][0][r] = fast_exp2(s[i][0][r] - off);
-            s[i][1][r] = fast_exp2(s[i][1][r] - off);
-          }
-          l_e[rt][r] = fmaf(l_e[rt][r], corr[r], (s[0][0][r] + s[0][1][r]) + (s[2][0][r] + s[2][1][r]));
-          l_o[rt][r] = fmaf(l_o[rt][r], corr[r], (s[1][0][r] + s[1][1][r]) + (s[3][0][r] + s[3][1][r]));
-        }
-        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-          for (int gi = 0; gi < G; ++gi) {
-            bias_e[rt][0][gi] *= corr[0]; bias_o[rt][0][gi] *= corr[0];
-            bias_e[rt][1][gi] *= corr[1]; bias_o[rt][1][gi] *= corr[1];
-          }
-#pragma unroll
-          for (int nt = 0; nt < Dv / 8; ++nt) {
-            o[rt][nt][0] *= corr[0]; o[rt][nt][1] *= corr[0]; o[rt][nt][2] *= corr[1]; o[rt][nt][3] *= corr[1];
-          }
-        }
-        // ---- p * s_v per group as a two-term binary16 sum (high part + rounded remainder): the A operands of the
-        // value product, which is then good to ~2^-22 whatever the magnitude of the cached values ----
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 sb = vsb4[i * 4 + tid];
-          float2 v[2][G] = {{sb_to_f2<kBf>(sb.x), sb_to_f2<kBf>(sb.y)}, {sb_to_f2<kBf>(sb.z), sb_to_f2<kBf>(sb.w)}};   // [e][group] = (scale, bias)
-          if (tail) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e)
-              if (pos0 + 8 * tid + 4 * e + i >= kv_len) { v[e][0] = make_float2(0.f, 0.f); v[e][1] = make_float2(0.f, 0.f); }
-          }
-#pragma unroll
-          for (int gi = 0; gi < G; ++gi)
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-              const float x0 = s[i][0][r] * v[0][gi].x, x1 = s[i][1][r] * v[1][gi].x;
-              const uint32_t hi = f32x2_to_h2(x0, x1);
-              const float2 hf = h2_to_f2(hi);
-              apv[rt][gi][i >> 1][(i & 1) * 2 + r] = hi;
-              apl[rt][gi][i >> 1][(i & 1) * 2 + r] = f32x2_to_h2(x0 - hf.x, x1 - hf.y);
-              const float b = fmaf(s[i][0][r], v[0][gi].y, s[i][1][r] * v[1][gi].y);
-              if (i & 1) bias_o[rt][r][gi] += b; else bias_e[rt][r][gi] += b;
+        // ---- value product on the codes ----
+        bool any_active = false;
+  #pragma unroll
+        for (int rt = 0; rt < R; ++rt) any_active |= active[rt];
+        if (any_active) {
+  #pragma unroll
+          for (int q4 = 0; q4 < Dv / 32; ++q4) {
+            const uint4 w4 = vc4[(q4 * 8 + g) * 4 + tid];
+            const uint32_t wd[4] = {w4.x, w4.y, w4.z, w4.w};
+            const int gi = q4 >> 1;
+  #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t wh = wd[j] >> 8;
+              const uint32_t be0 = wd[j] & kMaskLo, be1 = wd[j] & kMaskHi, bo0 = wh & kMaskLo, bo1 = wh & kMaskHi;
+  #pragma unroll
+              for (int rt = 0; rt < R; ++rt) {
+                if (!active[rt]) continue;
+                mma_f16(o[rt][4 * q4 + j], apv[rt][gi][0], be0, be1);
+                mma_f16(o[rt][4 * q4 + j], apv[rt][gi][1], bo0, bo1);
+                mma_f16(o[rt][4 * q4 + j], apl[rt][gi][0], be0, be1);
+                mma_f16(o[rt][4 * q4 + j], apl[rt][gi][1], bo0, bo1);
+              }
             }
+          }
         }
-      }
-      // ---- value product on the codes ----
-      bool any_active = false;
-#pragma unroll
-      for (int rt = 0; rt < R; ++rt) any_active |= active[rt];
-      if (any_active) {
-#pragma unroll
-        for (int q4 = 0; q4 < Dv / 32; ++q4) {
-          const uint4 w4 = vc4[(q4 * 8 + g) * 4 + tid];
-          const uint32_t wd[4] = {w4.x, w4.y, w4.z, w4.w};
-          const int gi = q4 >> 1;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t wh = wd[j] >> 8;
-            const uint32_t be0 = wd[j] & kMaskLo, be1 = wd[j] & kMaskHi, bo0 = wh & kMaskLo, bo1 = wh & kMaskHi;
-#pragma unroll
-            for (int rt = 0; rt < R; ++rt) {
-              if (!active[rt]) continue;
-              mma_f16(o[rt][4 * q4 + j], apv[rt][gi][0], be0, be1);
-              mma_f16(o[rt][4 * q4 + j], apv[rt][gi][1], bo0, bo1);
-              mma_f16(o[rt][4 * q4 + j], apl[rt][gi][0], be0, be1);
-              mma_f16(o[rt][4 * q4 + j], apl[rt][gi][1], bo0, bo1);
+      } else {
+        float prob[R][4][2][2];                            // probabilities of the active tiles: [tile][key tile][token e][row r]
+        bool active[R];
+  #pragma unroll
+        for (int rt = 0; rt < R; ++rt) {
+          const int pq_lo = prefix + i_min + (qhalf * R + rt) * 16, pq_hi = pq_lo + 15;
+          active[rt] = pos0 <= pq_hi && (W == 0 || pos0 + 31 > pq_lo - W);
+          if (!active[rt]) continue;
+          const bool need_mask = pos0 + 31 > pq_lo || (W > 0 && pos0 <= pq_hi - W);
+          // ---- integer dot products per key tile and group, two groups (one 16-byte piece per token row) at a time;
+          // the token's scale meets them, its bias the per-group query sums ----
+          float tsum[4][2][2], usum[4][2][2];              // [key tile][token e][row r]
+  #pragma unroll
+          for (int i = 0; i < 4; ++i)
+  #pragma unroll
+            for (int e = 0; e < 2; ++e) { tsum[i][e][0] = 0.f; tsum[i][e][1] = 0.f; usum[i][e][0] = 0.f; usum[i][e][1] = 0.f; }
+  #pragma unroll
+          for (int half = 0; half < G / 2; ++half) {
+            float acc[4][2][4];
+  #pragma unroll
+            for (int i = 0; i < 4; ++i)
+  #pragma unroll
+              for (int gi = 0; gi < 2; ++gi) { acc[i][gi][0] = 0.f; acc[i][gi][1] = 0.f; acc[i][gi][2] = 0.f; acc[i][gi][3] = 0.f; }
+            uint4 kw[4];
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) kw[i] = kc4[i * 16 * G + half * 32 + g * 4 + tid];
+  #pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint4 a1 = sm.qfrag[warp][rt][4 * half + ks][0][lane], a2 = sm.qfrag[warp][rt][4 * half + ks][1][lane];
+  #pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t w = ks == 0 ? kw[i].x : ks == 1 ? kw[i].y : ks == 2 ? kw[i].z : kw[i].w;
+                const uint32_t wh = w >> 8;
+                mma_f16(acc[i][ks >> 1], a1, w & kMaskLo, w & kMaskHi);
+                mma_f16(acc[i][ks >> 1], a2, wh & kMaskLo, wh & kMaskHi);
+              }
+            }
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              // (scale, bias) of tokens e = 0, 1 for the groups 2 half and 2 half + 1
+              float2 f[2][2];
+              if (G == 2) {
+                const uint4 sb = ksb4[i * 4 + tid];
+                f[0][0] = sb_to_f2<kBf>(sb.x); f[0][1] = sb_to_f2<kBf>(sb.y); f[1][0] = sb_to_f2<kBf>(sb.z); f[1][1] = sb_to_f2<kBf>(sb.w);
+              } else {
+  #pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const uint4 sb = ksb4[(i * 4 + tid) * 2 + e];
+                  f[e][0] = sb_to_f2<kBf>(half == 0 ? sb.x : sb.z); f[e][1] = sb_to_f2<kBf>(half == 0 ? sb.y : sb.w);
+                }
+              }
+  #pragma unroll
+              for (int e = 0; e < 2; ++e)
+  #pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                  tsum[i][e][r] = fmaf(acc[i][1][2 * r + e], f[e][1].x, fmaf(acc[i][0][2 * r + e], f[e][0].x, tsum[i][e][r]));
+                  usum[i][e][r] = fmaf(qs[rt][r][2 * half + 1], f[e][1].y, fmaf(qs[rt][r][2 * half], f[e][0].y, usum[i][e][r]));
+                }
+            }
+          }
+          // ---- scores in log2 units, mask, online softmax ----
+          float (&sc)[4][2][2] = prob[rt];
+  #pragma unroll
+          for (int i = 0; i < 4; ++i)
+  #pragma unroll
+            for (int e = 0; e < 2; ++e)
+  #pragma unroll
+              for (int r = 0; r < 2; ++r) sc[i][e][r] = fmaf(kap[rt][r], tsum[i][e][r], usum[i][e][r]);
+          if (need_mask) {
+  #pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              const int pq = pq_lo + g + 8 * r;
+  #pragma unroll
+              for (int i = 0; i < 4; ++i)
+  #pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const int pos = pos0 + 8 * tid + 4 * e + i;
+                  if (pos > pq || (W > 0 && pos <= pq - W)) sc[i][e][r] = -INFINITY;
+                }
+            }
+          }
+          float corr[2];
+  #pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            float cm = fmaxf(fmaxf(fmaxf(sc[0][0][r], sc[0][1][r]), fmaxf(sc[1][0][r], sc[1][1][r])),
+                             fmaxf(fmaxf(sc[2][0][r], sc[2][1][r]), fmaxf(sc[3][0][r], sc[3][1][r])));
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+            float m_new = fmaxf(m_run[rt][r], cm);
+            if (m_new == -INFINITY) m_new = 0.f;
+            corr[r] = fast_exp2(m_run[rt][r] - m_new);
+            m_run[rt][r] = m_new;
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float off = (i & 1) ? m_new + 4.f : m_new;   // odd tiles: p / 16 (their value codes carry a factor 16)
+              sc[i][0][r] = fast_exp2(sc[i][0][r] - off);
+              sc[i][1][r] = fast_exp2(sc[i][1][r] - off);
+            }
+            l_e[rt][r] = fmaf(l_e[rt][r], corr[r], (sc[0][0][r] + sc[0][1][r]) + (sc[2][0][r] + sc[2][1][r]));
+            l_o[rt][r] = fmaf(l_o[rt][r], corr[r], (sc[1][0][r] + sc[1][1][r]) + (sc[3][0][r] + sc[3][1][r]));
+          }
+          if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+  #pragma unroll
+            for (int gi = 0; gi < G; ++gi) {
+              bias_e[rt][0][gi] *= corr[0]; bias_o[rt][0][gi] *= corr[0];
+              bias_e[rt][1][gi] *= corr[1]; bias_o[rt][1][gi] *= corr[1];
+            }
+  #pragma unroll
+            for (int nt = 0; nt < Dv / 8; ++nt) {
+              o[rt][nt][0] *= corr[0]; o[rt][nt][1] *= corr[0]; o[rt][nt][2] *= corr[1]; o[rt][nt][3] *= corr[1];
+            }
+          }
+        }
+        // ---- value product on the codes, group by group: p * s_v as a two-term binary16 sum (high part + rounded
+        // remainder) is the A operand, which keeps the product good to ~2^-22 whatever the cached magnitudes ----
+        bool any_active = false;
+  #pragma unroll
+        for (int rt = 0; rt < R; ++rt) any_active |= active[rt];
+        if (any_active) {
+  #pragma unroll
+          for (int gi = 0; gi < G; ++gi) {
+            uint32_t apv[R][2][4], apl[R][2][4];           // [tile][MMA][register]
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float2 v[2];                                 // (scale, bias) of tokens e = 0, 1 for this group
+              if (G == 2) {
+                const uint4 sb = vsb4[i * 4 + tid];
+                v[0] = sb_to_f2<kBf>(gi == 0 ? sb.x : sb.y); v[1] = sb_to_f2<kBf>(gi == 0 ? sb.z : sb.w);
+              } else {
+  #pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const uint4 sb = vsb4[(i * 4 + tid) * 2 + e];
+                  v[e] = sb_to_f2<kBf>(gi == 0 ? sb.x : gi == 1 ? sb.y : gi == 2 ? sb.z : sb.w);
+                }
+              }
+              if (tail) {
+  #pragma unroll
+                for (int e = 0; e < 2; ++e)
+                  if (pos0 + 8 * tid + 4 * e + i >= kv_len) v[e] = make_float2(0.f, 0.f);
+              }
+  #pragma unroll
+              for (int rt = 0; rt < R; ++rt) {
+                if (!active[rt]) continue;
+  #pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                  const float x0 = prob[rt][i][0][r] * v[0].x, x1 = prob[rt][i][1][r] * v[1].x;
+                  const uint32_t hi = f32x2_to_h2(x0, x1);
+                  const float2 hf = h2_to_f2(hi);
+                  apv[rt][i >> 1][(i & 1) * 2 + r] = hi;
+                  apl[rt][i >> 1][(i & 1) * 2 + r] = f32x2_to_h2(x0 - hf.x, x1 - hf.y);
+                  const float b = fmaf(prob[rt][i][0][r], v[0].y, prob[rt][i][1][r] * v[1].y);
+                  if (i & 1) bias_o[rt][r][gi] += b; else bias_e[rt][r][gi] += b;
+                }
+              }
+            }
+  #pragma unroll
+            for (int q4 = 2 * gi; q4 < 2 * gi + 2; ++q4) {
+              const uint4 w4 = vc4[(q4 * 8 + g) * 4 + tid];
+              const uint32_t wd[4] = {w4.x, w4.y, w4.z, w4.w};
+  #pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint32_t wh = wd[j] >> 8;
+                const uint32_t be0 = wd[j] & kMaskLo, be1 = wd[j] & kMaskHi, bo0 = wh & kMaskLo, bo1 = wh & kMaskHi;
+  #pragma unroll
+                for (int rt = 0; rt < R; ++rt) {
+                  if (!active[rt]) continue;
+                  mma_f16(o[rt][4 * q4 + j], apv[rt][0], be0, be1);
+                  mma_f16(o[rt][4 * q4 + j], apv[rt][1], bo0, bo1);
+                  mma_f16(o[rt][4 * q4 + j], apl[rt][0], be0, be1);
+                  mma_f16(o[rt][4 * q4 + j], apl[rt][1], bo0, bo1);
+                }
+              }
             }
           }
         }
@@ -439,15 +623,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_mma_kernel(const __grid_c
     }
 }
 
-template <int R, bool kBf>
+template <int R, int G, bool kBf>
 cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   static bool configured[64] = {};
-  const size_t smem = sizeof(PrefillSmem<R>);
+  const size_t smem = sizeof(PrefillSmem<R, G>);
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(prefill_mma_kernel<R, kBf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(prefill_mma_kernel<R, G, kBf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -461,12 +645,12 @@ cudaError_t launch_r(const PrefillParams& P, dim3 grid, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, prefill_mma_kernel<R, kBf>, P);
+  return cudaLaunchKernelEx(&cfg, prefill_mma_kernel<R, G, kBf>, P);
 }
 
 }  // namespace
 
-bool prefill_mma_supported(const Layout& y) { return !y.alias && y.D == 128 && y.Dv == 128 && y.n_rep <= 4; }
+bool prefill_mma_supported(const Layout& y) { return !y.alias && y.D == y.Dv && (y.D == 128 || y.D == 256) && y.n_rep <= 4; }
 
 cudaError_t launch_prefill_mma(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                                const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
@@ -476,9 +660,15 @@ cudaError_t launch_prefill_mma(const Layout& y, const void* pool, int n_blocks, 
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.q_offs = q_offs; P.window = window;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
-  constexpr int R = 2;
-  const dim3 grid((max_q_len + 32 * R - 1) / (32 * R), y.Hkv, b.n_agents);
-  return y.sb_bf16 ? launch_r<R, true>(P, grid, st) : launch_r<R, false>(P, grid, st);
+  const int hs = y.n_rep > 2 ? 4 : y.n_rep;
+  const int tile1 = (kWarps / hs) * 16;                  // queries per CTA with one 16-row tile per warp
+  if (y.G == 4) {
+    // d = 256: one 16-row tile per warp (the accumulators of a tile are 128 registers per lane)
+    const dim3 grid((max_q_len + tile1 - 1) / tile1, y.Hkv, b.n_agents);
+    return y.sb_bf16 ? launch_r<1, 4, true>(P, grid, st) : launch_r<1, 4, false>(P, grid, st);
+  }
+  const dim3 grid((max_q_len + 2 * tile1 - 1) / (2 * tile1), y.Hkv, b.n_agents);
+  return y.sb_bf16 ? launch_r<2, 2, true>(P, grid, st) : launch_r<2, 2, false>(P, grid, st);
 }
 
 }  // namespace q4kv

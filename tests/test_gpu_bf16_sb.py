@@ -134,6 +134,7 @@ def test_latent_cache_fused_entry_is_refused_and_the_two_call_form_works(H):
     ("gqa128", [512, 200], 130, 0),
     ("gqa128", [300, 0], 70, 100),
     ("gqa256", [256, 10], 70, 128),
+    ("gqa256", [900, 0], 150, 0),
 ])
 def test_prefill_matches_oracle(H, name, prefix, chunk, window):
     lens = [n + chunk for n in prefix]

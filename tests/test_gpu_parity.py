@@ -648,9 +648,14 @@ def test_prefill_matches_oracle_and_chunking_is_invisible(H, name, prefix, chunk
     ((1, 8, 2, 128, 128, False), [700, 300], [200, 150], 96),            # sliding window across chunk edges
     ((1, 4, 4, 128, 128, False), [2500], [300], 0),                      # MHA (one query head per KV head)
     ((2, 6, 2, 128, 128, False), [100, 40], [65, 1], 0),                 # three query heads per KV head, a 1-token phase
+    ((1, 8, 4, 256, 256, False), [700, 0, 33], [150, 77, 130], 0),       # d = 256, two query heads per KV head
+    ((1, 8, 4, 256, 256, False), [1400, 300], [200, 150], 512),          # d = 256 under a sliding window
+    ((1, 4, 4, 256, 256, False), [900], [131], 0),                       # d = 256, one query head per KV head
+    ((1, 8, 2, 256, 256, False), [300, 40], [65, 1], 100),               # d = 256, four query heads per KV head
+    ((1, 6, 2, 256, 256, False), [300, 40], [65, 33], 0),                # d = 256, three query heads per KV head
 ])
 def test_prefill_tensor_core_path_ragged(H, spec_args, prefix, chunks, window):
-    """Ragged phases through the d=128 tensor-core prefill kernel: every row against the oracle."""
+    """Ragged phases through the tensor-core prefill kernels (d = 128 and d = 256): every row against the oracle."""
     lens = [p0 + c for p0, c in zip(prefix, chunks)]
     p = Pair(H, spec_args, lens, seed=43).fill()
     s = p.ospec
