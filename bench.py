@@ -7,7 +7,7 @@ agent, then decode attention of one query per agent over the whole Q4 cache.  On
 layers.  The metric is the achieved HBM bandwidth over the algorithmic bytes of the step (each
 needed Q4 row read once + q + out + new rows); agent-steps/s rides along.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4|5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4|5|6] [--impl reference]
 
 N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no collective.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
@@ -600,7 +600,7 @@ def main():
     }
     if rank == 0 and world == 1 and default_run and not args.no_all_configs:
         allc = {}
-        for idx in (2, 3, 4, 5):
+        for idx in (2, 3, 4, 5, 6):
             wi = synth.workload(idx)
             ri = measure(wi, args, local, None, full=False)
             units_i, roof_i = roofline_of(wi, ri)

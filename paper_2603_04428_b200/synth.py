@@ -126,7 +126,8 @@ class Workload:
 
 def workload(index: int) -> Workload:
     """The five benchmark configurations, 0-based, and (index 5) the per-head MLA cache of Section 3.6 at the sizes of
-    configuration 4: keys of 192 dims (3 groups), values of 128 (2 groups), 16 KV heads."""
+    configuration 4: keys of 192 dims (3 groups), values of 128 (2 groups), 16 KV heads; (index 6) a chunked-prefill
+    phase at d = 256."""
     seed = BASE_SEED + index
     if index == 0:
         return Workload("tiny_gqa_decode", 1, 8, 2, 128, 128, False, [1000, 700], 1,
@@ -147,4 +148,8 @@ def workload(index: int) -> Workload:
     if index == 5:
         return Workload("dsv2lite_perhead_mla_decode", 27, 16, 16, 192, 128, False, [16384] * 4, 1,
                         softmax_scale=1.0 / math.sqrt(192), seed=seed)
+    if index == 6:
+        # a d = 256 phase (Gemma-3-12B's head shape, global layers): what the exact-product prefill kernel does there
+        return Workload("gemma3_12b_shaped_global_prefill", 8, 16, 8, 256, 256, False, [4096] * 8, 512,
+                        softmax_scale=1.0 / math.sqrt(256), seed=seed, kind="prefill")
     raise IndexError(index)

@@ -676,6 +676,67 @@ def test_prefill_tensor_core_path_ragged(H, spec_args, prefix, chunks, window):
     assert p.dc.read_flags() == 0
 
 
+def test_interleaved_512_token_chunks_and_decoding_agents_in_one_batch(H):
+    """The scheduler's pattern of Section 3.4: prompts are prefilled in chunks of at most 512 tokens, the chunks of
+    different agents interleaved step by step, while another agent decodes one token per step -- every step is ONE
+    append call and ONE attention call over a ragged batch (chunk lengths 512, 188, 1 ...).  Every row must equal the
+    oracle's one-shot prefill of the whole prompt (the chunking is invisible), and the cache bytes its append."""
+    spec_args = (1, 8, 2, 128, 128, False)
+    prompts = [1700, 700, 0]                     # agent 2 has a cached context and decodes
+    cached = [0, 300, 900]                       # tokens already in the cache when the schedule starts
+    steps = 3
+    total = [cached[a] + (prompts[a] if prompts[a] else steps) for a in range(3)]
+    p = Pair(H, spec_args, total, seed=47)
+    s = p.ospec
+    data = [p.kv(0, a, total[a]) for a in range(3)]
+    qs = [p.q(20 + a, total[a] - cached[a]) for a in range(3)]       # one query row per new token
+    scale = 1.0 / math.sqrt(s.d_qk)
+    # the cached contexts
+    for a in range(3):
+        if cached[a]:
+            O.quantize_append(p.opool, 0, p.tabs[a:a + 1], [0], [0, cached[a]], f32(data[a][0][:cached[a]]), f32(data[a][1][:cached[a]]))
+    p.dc.append(0, [0, 0, 0], np.concatenate([[0], np.cumsum(cached)]).astype(np.int32),
+                np.concatenate([data[a][0][:cached[a]] for a in range(3)]), np.concatenate([data[a][1][:cached[a]] for a in range(3)]))
+    # oracle, one shot: each agent's new tokens as a single phase
+    for a in range(3):
+        O.quantize_append(p.opool, 0, p.tabs[a:a + 1], [cached[a]], [0, total[a] - cached[a]],
+                          f32(data[a][0][cached[a]:]), f32(data[a][1][cached[a]:]))
+    refs = []
+    for a in range(3):
+        n_new = total[a] - cached[a]
+        r, _ = O.prefill_attention(p.opool, 0, p.tabs[a:a + 1], [total[a]], [0, n_new], 0, f32(qs[a]), scale)
+        refs.append(r)
+    # the schedule: step t takes up to 512 prompt tokens of every prefilling agent and one token of the decoding one
+    done = [0, 0, 0]
+    for t in range(steps):
+        take = [min(512, prompts[a] - done[a]) if prompts[a] else 1 for a in range(3)]
+        assert any(take)
+        pos = [cached[a] + done[a] for a in range(3)]
+        offs = np.concatenate([[0], np.cumsum(take)]).astype(np.int32)
+        kb = np.concatenate([data[a][0][pos[a]:pos[a] + take[a]] for a in range(3)])
+        vb = np.concatenate([data[a][1][pos[a]:pos[a] + take[a]] for a in range(3)])
+        qb = np.concatenate([qs[a][done[a]:done[a] + take[a]] for a in range(3)])
+        p.dc.append(0, pos, offs, kb, vb)
+        lens = [pos[a] + take[a] for a in range(3)]
+        out, _ = p.dc.prefill(0, lens, offs, 0, qb, scale)
+        got = out.cpu().numpy()
+        for a in range(3):
+            if take[a]:
+                assert_attention_close(got[offs[a]:offs[a + 1]], refs[a][done[a]:done[a] + take[a]], f"step {t} agent {a}")
+        done = [done[a] + take[a] for a in range(3)]
+    assert done == [512 * steps, 700, steps]
+    # agent 0 still has 164 tokens left: a fourth step on its own
+    rest = prompts[0] - done[0]
+    if rest:
+        pos0 = cached[0] + done[0]
+        p.dc.append(0, [pos0], [0, rest], data[0][0][pos0:], data[0][1][pos0:], bt=p.dc.sub_batch(0, 1)[1])
+        t0, b0 = p.dc.sub_batch(0, 1)
+        out, _ = p.dc.prefill(0, [total[0]], [0, rest], 0, qs[0][done[0]:], scale, bt=b0)
+        assert_attention_close(out.cpu().numpy(), refs[0][done[0]:], "agent 0 tail")
+    p.lens = total
+    p.check_packed_equal()
+
+
 class QuietStartPair(Pair):
     """The first 300 keys of every agent are tiny, so every row's running maximum jumps far when the walk leaves them."""
 
