@@ -110,6 +110,9 @@ __device__ inline bool spin_until_ge(volatile int* word, int want, volatile int*
   *abort_flag = 1;
   return false;
 }
+__device__ inline void prefetch_l2_bulk(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ inline void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_u32(dst_smem)),
@@ -1142,7 +1145,18 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
         }
         __syncwarp();
       }
-      if (!waited) { grid_dependency_wait(); waited = true; }
+      if (!waited) {
+        // While the preceding kernel drains, ask L2 for the chunks of the first ring fill (more than that was measured
+        // and is no faster; the same prefetch in the MLA-latent kernel gains nothing).  A prefetch returns nothing
+        // to the kernel, and L2 is where the preceding kernel's writes land, so what the copies read after the wait
+        // is current whatever that kernel still writes.
+        if (lane < kSlots && next_k < planned) {
+          const uint32_t off = sm.src_off[next_k % kOffCap];
+          if (off != kOffBad) prefetch_l2_bulk(layer_base + (uint64_t)off * 16u, kChunkBytes);
+        }
+        grid_dependency_wait();
+        waited = true;
+      }
       // ---- issue: a short polling loop, left from time to time to plan further ----
       bool any_left = true;
       for (int it = 0; it < 64 && any_left; ++it) {
