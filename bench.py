@@ -543,13 +543,13 @@ def main():
                     help="decode step as a quantize-append launch plus an attention launch per layer instead of the "
                          "one-launch update-and-fetch")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="least duration of each timed region")
-    ap.add_argument("--op", default="step", choices=["step", "pack"],
+    ap.add_argument("--op", default="step", choices=["step", "pack", "unpack"],
                     help="step: the append + attention step of --workload; pack: q4kv_pack / q4kv_unpack / bulk append")
     ap.add_argument("--agents", type=int, default=0,
                     help="scaled variant of a uniform-length configuration: this many agents (named so in config.workload)")
     ap.add_argument("--layers", type=int, default=0, help="scaled variant: this many layers")
     args = ap.parse_args()
-    if args.op == "pack":
+    if args.op in ("pack", "unpack"):
         print(json.dumps(run_pack(args)))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
@@ -656,6 +656,18 @@ def run_pack(args):
             t = timed(g.replay)
             side.synchronize()
         return t
+    if args.op == "unpack":
+        # q4kv_unpack alone (pack and unpack are the same kernel by name: this is how a profiler tells them apart)
+        B.q4kv_pack(dc.spec, dc.pool, dc.n_blocks, dc.tables[0], n, dst, dc.flags)
+        t_unpack = timed_graph(lambda: B.q4kv_unpack(dc.spec, dst, n, dc.pool, dc.n_blocks, dc.tables[0], dc.flags))
+        ach = 2 * nbytes / t_unpack / 1e9
+        return {"metric": "q4_unpack_hbm_gbps", "value": ach, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": t_unpack * 1e3, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+                "config": {"workload": "unpack_llama31_8b_agent", "packed_bytes": nbytes},
+                "roofline": {"bound": "hbm", "kernel": "q4kv_unpack", "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
+                             "frac": ach / hbm_peak, "peak_kind": peak_kind, "avg_launch_us": t_unpack * 1e6,
+                             "traffic": NCU_TRAFFIC_BYTES.get("unpack")}, "gpu_launches": args.steps}
     t_pack = timed_graph(lambda: B.q4kv_pack(dc.spec, dc.pool, dc.n_blocks, dc.tables[0], n, dst, dc.flags))
     t_unpack = timed_graph(lambda: B.q4kv_unpack(dc.spec, dst, n, dc.pool, dc.n_blocks, dc.tables[0], dc.flags))
     # ---- warm restore: pinned host image -> chunked copies overlapping q4kv_unpack (Table "TTFT", warm rows) ----

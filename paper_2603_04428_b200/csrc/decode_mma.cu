@@ -388,6 +388,8 @@ struct Smem {
   int deposits[kMBufs];         // running count of deposits into each buffer
   int epilogues[kMBufs];        // number of completed epilogues of each buffer
   int next_chunk;               // claim counter
+  int epi_claim[kMBufs];        // uses of each deposit buffer whose epilogue has been taken (by a consumer or the planner)
+  int all_issued;               // set by the planner once every chunk of the CTA has been issued
   int fin_arrived;              // last segment: head warps whose record is written
   int fin_ticket;               // last segment: 0 until the ticket is drawn, then 1 (not the last) or 2 (combine the records)
   int abort_flag;
@@ -1070,7 +1072,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.full[s], 1); sm.released[s] = 0; sm.bad[s] = 0; sm.patched[s] = 0; }
     for (int i = 0; i < kQBufs; ++i) sm.q_tag[i] = 0;
-    for (int i = 0; i < kMBufs; ++i) { sm.deposits[i] = 0; sm.epilogues[i] = 0; }
+    for (int i = 0; i < kMBufs; ++i) { sm.deposits[i] = 0; sm.epilogues[i] = 0; sm.epi_claim[i] = 0; }
+    sm.all_issued = 0;
     sm.next_chunk = 0;
     sm.fin_arrived = 0; sm.fin_ticket = 0;
     sm.abort_flag = 0;
@@ -1108,7 +1111,24 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     // block tables are inputs that no kernel writes, so the first planning steps run while the preceding kernel drains;
     // the pool is read only after it.
     static_assert(kSlots <= 32 && kOffCap >= 2 * 32 + kSlots, "table ring: a step of entries ahead of every reader");
-    bool waited = false, bad_block = false, more = wk.next(seg);
+    // Once every chunk has been issued this warp has time to spare, and it takes the epilogues of the segments that
+    // complete from then on (all but the CTA's last): a consumer that leaves the stream for an epilogue (a few
+    // microseconds with the ticket and a pair's final combination) costs its CTA an extra round of chunks.  While
+    // chunks are still to be issued the consumers keep them, or the ring would run dry meanwhile.  A claim word per
+    // deposit buffer decides who runs one.  Segments complete in order, so a second walker names the next one.
+    // d = 128 only (5 agents x 4097 tokens: 20.2 -> 19.2 us per launch, 2 agents: 18.4 -> 15.9 us; 40 agents: 1.8 %
+    // slower): in the other instantiations the second copy of the epilogue's code slowed the chunk loop of long
+    // launches by 5-9 %, as one shared non-inlined copy did through its spills.
+    Walker wke = wk;
+    Segment sge;
+    int n_seg = 0, epi_idx = 0;
+    {
+      Walker w2 = wk;
+      Segment s2;
+      while (w2.next(s2)) ++n_seg;
+    }
+    wke.next(sge);
+    bool waited = false, bad_block = false, more = wk.next(seg), all_out = false;
     int tq_head = 0, tq_tail = 0;            // patch queue: entries tq_head .. tq_tail-1 (indices taken modulo kTailQ)
     int kb = 0;                              // chunks of `seg` already planned
     int planned = 0;                         // chunks of the CTA that have their table entry
@@ -1178,6 +1198,26 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
             idle = 0;
           }
         }
+        if (G == 2 && epi_idx < n_seg - 1) {
+          const int eb = epi_idx % kMBufs, euse = epi_idx / kMBufs;
+          if (*(volatile int*)&sm.deposits[eb] >= (euse + 1) * NW) {
+            int state = 0;                               // 1: a consumer has it, 2: this warp takes it
+            if (lane == 0) {
+              if (*(volatile int*)&sm.epi_claim[eb] > euse) state = 1;
+              else if (all_out) state = atomicCAS(&sm.epi_claim[eb], euse, euse + 1) == euse ? 2 : 1;
+            }
+            state = __shfl_sync(0xffffffffu, state, 0);
+            if (state == 2) {
+              __threadfence_block();
+              segment_epilogue<G, NW>(&sm.merge[eb][0][0][0], &sm.epilogues[eb], euse, P, sge, cta, rs.part, lane);
+            }
+            if (state != 0) {
+              wke.next(sge);
+              ++epi_idx;
+              idle = 0;
+            }
+          }
+        }
         const bool can = next_k < planned && *my_released >= round;
         if (can) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the consumer's reads and patches of the slot come first
@@ -1185,13 +1225,17 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
           next_k += kSlots;
           ++round;
         }
-        any_left = __any_sync(0xffffffffu, next_k < n_chunks) || tq_head < tq_tail;
+        if (!all_out && !__any_sync(0xffffffffu, next_k < n_chunks)) {
+          all_out = true;
+          if (lane == 0) *(volatile int*)&sm.all_issued = 1;
+        }
+        any_left = !all_out || tq_head < tq_tail || (G == 2 && epi_idx < n_seg - 1);
         if (__any_sync(0xffffffffu, can)) { idle = 0; continue; }
         if (more && tq_tail - tq_head < kTailQ && __all_sync(0xffffffffu, next_k >= planned)) break;   // plan further first
         ++idle;
         __nanosleep(200);
       }
-      if (!any_left) break;                  // every chunk has been issued
+      if (!any_left) break;                  // every chunk has been issued, every epilogue but the last is done
       if (idle > (kSpinLimit >> 2) || *(volatile int*)&sm.abort_flag) {
         if (lane == 0) { sm.abort_flag = 1; raise_flag(P.flags, Q4KV_FLAG_INTERNAL); }
         // giving up: each lane lets the last copy it issued into its slot land before the CTA lets go of shared memory
@@ -1321,6 +1365,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       return;
     }
     if (!last) return;
+    if (G == 2 && cur != n_seg - 1) {
+      // an earlier segment: the planner warp takes it if it has nothing left to issue
+      int mine = 0;
+      if (lane == 0 && !*(volatile int*)&sm.all_issued) mine = atomicCAS(&sm.epi_claim[b], use, use + 1) == use;
+      if (!__shfl_sync(0xffffffffu, mine, 0)) return;
+    }
     __threadfence_block();
     segment_epilogue<G, NW>(&sm.merge[b][0][0][0], &sm.epilogues[b], use, P, seg, cta, rs.part, lane);
   };
