@@ -828,16 +828,19 @@ __device__ __forceinline__ void segment_epilogue(const float* merge_buf, int* ep
   // ticket: the CTA whose record arrives last combines all records of the pair
   const uint32_t pair_u0 = seg.u0 - (uint32_t)(seg.c0 - seg.cf);
   const int c_first = part.cta_of(pair_u0), c_last = part.cta_of(pair_u0 + (uint32_t)seg.nc - 1u);
-  __threadfence();
+  // The warp's record stores are ordered before lane 0's release by the warp barrier, and the other lanes' record loads
+  // after its acquire by the second one: one acquire-release atomic takes the place of a fence on either side.
   __syncwarp();
   int final_merge = 0;
   if (lane == 0) {
-    final_merge = atomicAdd(&P.tickets[pair], 1) == c_last - c_first;
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(&P.tickets[pair]) : "memory");
+    final_merge = old == c_last - c_first;
     if (final_merge) P.tickets[pair] = 0;            // ready for the next call
   }
   final_merge = __shfl_sync(0xffffffffu, final_merge, 0);
   if (!final_merge) return;
-  __threadfence();
+  __syncwarp();
   const int R = c_last - c_first + 1;
   const float* base = P.partials + (size_t)(pair + c_first) * rstride;
   // The records sit in L2, a microsecond away: all heads travel together, and the first batch of record loads is issued
