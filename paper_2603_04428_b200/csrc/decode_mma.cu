@@ -1122,15 +1122,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     // d = 128 only (5 agents x 4097 tokens: 20.2 -> 19.2 us per launch, 2 agents: 18.4 -> 15.9 us; 40 agents: 1.8 %
     // slower): in the other instantiations the second copy of the epilogue's code slowed the chunk loop of long
     // launches by 5-9 %, as one shared non-inlined copy did through its spills.
+    // (A segment is the CTA's last when its chunks end the CTA's range: no count of the segments is needed.)
     Walker wke = wk;
     Segment sge;
-    int n_seg = 0, epi_idx = 0;
-    {
-      Walker w2 = wk;
-      Segment s2;
-      while (w2.next(s2)) ++n_seg;
-    }
-    wke.next(sge);
+    int epi_idx = 0;
+    bool epi_more = false, epi_started = false;          // sge names a segment that is not the CTA's last
     bool waited = false, bad_block = false, more = wk.next(seg), all_out = false;
     int tq_head = 0, tq_tail = 0;            // patch queue: entries tq_head .. tq_tail-1 (indices taken modulo kTailQ)
     int kb = 0;                              // chunks of `seg` already planned
@@ -1201,7 +1197,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
             idle = 0;
           }
         }
-        if (G == 2 && epi_idx < n_seg - 1) {
+        if (G == 2 && epi_more) {
           const int eb = epi_idx % kMBufs, euse = epi_idx / kMBufs;
           if (*(volatile int*)&sm.deposits[eb] >= (euse + 1) * NW) {
             int state = 0;                               // 1: a consumer has it, 2: this warp takes it
@@ -1215,7 +1211,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
               segment_epilogue<G, NW>(&sm.merge[eb][0][0][0], &sm.epilogues[eb], euse, P, sge, cta, rs.part, lane);
             }
             if (state != 0) {
-              wke.next(sge);
+              epi_more = wke.next(sge) && sge.k0 + (sge.c1 - sge.c0) < n_chunks;
               ++epi_idx;
               idle = 0;
             }
@@ -1228,11 +1224,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
           next_k += kSlots;
           ++round;
         }
+        if (G == 2 && !epi_started) {                    // the first segment is named here, after the first copies are out
+          epi_started = true;
+          epi_more = wke.next(sge) && sge.k0 + (sge.c1 - sge.c0) < n_chunks;
+        }
         if (!all_out && !__any_sync(0xffffffffu, next_k < n_chunks)) {
           all_out = true;
           if (lane == 0) *(volatile int*)&sm.all_issued = 1;
         }
-        any_left = !all_out || tq_head < tq_tail || (G == 2 && epi_idx < n_seg - 1);
+        any_left = !all_out || tq_head < tq_tail || (G == 2 && epi_more);
         if (__any_sync(0xffffffffu, can)) { idle = 0; continue; }
         if (more && tq_tail - tq_head < kTailQ && __all_sync(0xffffffffu, next_k >= planned)) break;   // plan further first
         ++idle;
@@ -1284,12 +1284,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     }
   }
 
-  int n_seg = 0;                // segments of this CTA: the last one's epilogue runs one warp per head
-  {
-    Walker w2 = wk;
-    Segment s2;
-    while (w2.next(s2)) ++n_seg;
-  }
   bool aborted = false, poisoned = false;
   int cur = -1;                 // index of the segment `seg` describes (-1: none yet)
   bool have_seg = false;        // this warp holds state for segment `cur`
@@ -1348,7 +1342,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     int last = 0;
     if (lane == 0) last = atomicAdd(&sm.deposits[b], 1) == (use + 1) * NW - 1;
     last = __shfl_sync(0xffffffffu, last, 0);
-    if (G == 4 && cur == n_seg - 1) {
+    const bool last_seg = seg.k0 + (seg.c1 - seg.c0) >= n_chunks;     // this segment's chunks end the CTA's range
+    if (G == 4 && last_seg) {
       // the CTA's last segment: nothing is left to stream, so the head warps wait for the last deposit and share the
       // epilogue; the other warps are done.  (d = 256 only: measured on the d-128 kernel the shared epilogue made the
       // 23.6 MB launch 1.2 us slower, on the d-256 kernel it makes every launch 1 us faster.)
@@ -1368,7 +1363,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
       return;
     }
     if (!last) return;
-    if (G == 2 && cur != n_seg - 1) {
+    if (G == 2 && !last_seg) {
       // an earlier segment: the planner warp takes it if it has nothing left to issue
       int mine = 0;
       if (lane == 0 && !*(volatile int*)&sm.all_issued) mine = atomicCAS(&sm.epi_claim[b], use, use + 1) == use;
