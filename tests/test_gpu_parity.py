@@ -289,6 +289,46 @@ def test_decode_long_contexts_wrap_the_ring(H, spec_args, lens, window):
     assert p.dc.read_flags() == 0
 
 
+@pytest.mark.parametrize("spec_args,n_agents,max_len,window,fused", [
+    ((1, 8, 2, 128, 128, False), 300, 200, 0, False),      # hundreds of short pairs: many segments per CTA
+    ((1, 8, 2, 128, 128, False), 300, 200, 0, True),
+    ((1, 4, 2, 256, 256, False), 150, 300, 64, True),
+    ((1, 4, 4, 192, 128, False), 120, 150, 0, True),
+    ((1, 8, 2, 128, 128, False), 40, 2500, 0, True),       # a few segments per CTA, pairs split over two or three CTAs
+])
+def test_decode_many_agents_many_segments_per_cta(H, spec_args, n_agents, max_len, window, fused):
+    """Every CTA walks several (agent, KV head) segments: deposit buffers and query buffers are reused, segment
+    epilogues run in the stream (by a consumer warp or, at d = 128, by the planner warp once all chunks are issued),
+    pairs that straddle CTAs go through records and tickets.  Twice in a row on one workspace."""
+    g = synth.rng(53, n_agents)
+    lens = [int(x) for x in g.integers(1, max_len + 1, size=n_agents)]
+    lens[3] = 0
+    p = Pair(H, spec_args, lens, seed=53, extra_tokens=1, spare_blocks=2).fill()
+    s = p.ospec
+    scale = 1.0 / math.sqrt(s.d_qk)
+    q = p.q(7, n_agents)
+    if fused:
+        kb = synth.kv_bf16(53, 500, n_agents, s.n_kv_heads, s.d_qk)
+        vb = synth.kv_bf16(53, 600, n_agents, s.n_kv_heads, s.d_v)
+        live = [a for a in range(n_agents) if lens[a] > 0]
+        offs = np.concatenate([[0], np.cumsum([1 if lens[a] > 0 else 0 for a in range(n_agents)])]).astype(np.int32)
+        O.quantize_append(p.opool, 0, p.tabs, lens, offs, f32(kb[live]), f32(vb[live]))
+        new_lens = [n + 1 if n > 0 else 0 for n in lens]
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, new_lens, window, f32(q), scale)
+        out, lse = p.dc.append_decode(0, new_lens, window, kb, vb, q, scale)
+        p.lens = new_lens
+    else:
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, lens, window, f32(q), scale)
+        out, lse = p.dc.decode(0, lens, window, q, scale)
+    assert_attention_close(out.cpu().numpy(), ref)
+    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    out2, lse2 = p.dc.decode(0, p.lens, window, q, scale)          # the workspace header was left at zero
+    assert_attention_close(out2.cpu().numpy(), ref, "second call")
+    assert p.dc.read_flags() == 0
+    if fused:
+        p.check_packed_equal()
+
+
 def test_decode_shorter_lengths_than_cached_and_zero_length(H):
     p = Pair(H, SPECS["gqa128"], [600, 300, 50], seed=32).fill()
     q = p.q(7, 3)
