@@ -992,22 +992,30 @@ __device__ __forceinline__ void last_segment_by_heads(const float* merge_buf, in
   // every head's record is written and fenced before one thread draws the ticket
   const uint32_t pair_u0 = seg.u0 - (uint32_t)(seg.c0 - seg.cf);
   const int c_first = part.cta_of(pair_u0), c_last = part.cta_of(pair_u0 + (uint32_t)seg.nc - 1u);
-  __threadfence();
+  // Ordering: each head warp's record stores come before its lane 0's arrival (warp barrier, then a CTA-scope
+  // fence); the last arrival draws the ticket with one acquire-release atomic at GPU scope, which publishes all the
+  // head warps' records and, if the ticket is the pair's last, makes the other CTAs' records readable; the answer
+  // reaches the other head warps through shared memory and a CTA-scope fence.
   __syncwarp();
   int state = 0;
   if (lane == 0) {
+    __threadfence_block();
     if (atomicAdd(fin_arrived, 1) == n_rep - 1) {
-      const int final_merge = atomicAdd(&P.tickets[pair], 1) == c_last - c_first;
+      __threadfence_block();
+      int old;
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(&P.tickets[pair]) : "memory");
+      const int final_merge = old == c_last - c_first;
       if (final_merge) P.tickets[pair] = 0;          // ready for the next call
       __threadfence_block();
       *(volatile int*)fin_ticket = 1 + final_merge;
     }
     for (uint32_t i = 0; i < (kSpinLimit << 4) && (state = *(volatile int*)fin_ticket) == 0; ++i)
       if ((i & 255u) == 255u && *abort_flag) break;
+    __threadfence_block();
   }
   state = __shfl_sync(0xffffffffu, state, 0);
   if (state != 2) return;
-  __threadfence();
+  __syncwarp();
   // this CTA drew the pair's last ticket: head h of all records, the loads of up to RB records in flight together
   const int R = c_last - c_first + 1;
   const float* base = P.partials + (size_t)(pair + c_first) * rstride + (size_t)h * kRecStride(Dv);
@@ -1343,10 +1351,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_mma_kernel(const __gr
     if (lane == 0) last = atomicAdd(&sm.deposits[b], 1) == (use + 1) * NW - 1;
     last = __shfl_sync(0xffffffffu, last, 0);
     const bool last_seg = seg.k0 + (seg.c1 - seg.c0) >= n_chunks;     // this segment's chunks end the CTA's range
-    if (G == 4 && last_seg) {
+    if (G != 3 && last_seg) {
       // the CTA's last segment: nothing is left to stream, so the head warps wait for the last deposit and share the
-      // epilogue; the other warps are done.  (d = 256 only: measured on the d-128 kernel the shared epilogue made the
-      // 23.6 MB launch 1.2 us slower, on the d-256 kernel it makes every launch 1 us faster.)
+      // epilogue; the other warps are done.  (Not in the d_qk 192 instantiation, where it measured 0.4 % slower.  On the
+      // d-128 kernel it cost 1.2 us while a consumer still ran the epilogues of earlier segments; since the planner
+      // warp takes those it saves 0.5 us per launch at 5 agents and 0.8 us at 2.)
       if (warp >= n_rep) return;
       {
         bool ok = false;
