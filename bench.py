@@ -220,8 +220,8 @@ class DeviceWorkload:
                                        [w.layer_window(l) for l in range(w.n_layers)], self.k_new, self.v_new, self.q,
                                        w.softmax_scale, self.out, B.OUT_F32, None, self.ws_layers, dc.flags)
 
-    def step(self):
-        for l in range(self.w.n_layers):
+    def step(self, l0=0, l1=None):
+        for l in range(l0, self.w.n_layers if l1 is None else l1):
             if self.fused:
                 self.fused_layer(l)
             else:
@@ -458,13 +458,45 @@ def measure(w, args, local, dist=None, full=True):
             hv = None if dw.v_new is None else dw.v_new.cpu().pin_memory()
             hout = torch.empty(dw.out.shape, dtype=dw.out.dtype).pin_memory()
 
+            # The step in two halves of the layers, so that the second half's inputs travel while the first half
+            # computes and the first half's results travel while the second computes: one CUDA graph over two streams
+            # (every input and every result still crosses the host link inside the step).
+            side = torch.cuda.Stream()
+            Lh = max(1, L // 2)
+            e2e_graph = None
+            if use_graph and L >= 2:
+                def half_in(a, b):
+                    dw.q[a:b].copy_(hq[a:b], non_blocking=True)
+                    dw.k_new[a:b].copy_(hk[a:b], non_blocking=True)
+                    if hv is not None:
+                        dw.v_new[a:b].copy_(hv[a:b], non_blocking=True)
+                e2e_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(e2e_graph, stream=stream):
+                    half_in(0, Lh)
+                    side.wait_stream(stream)                   # fork
+                    with torch.cuda.stream(side):
+                        half_in(Lh, L)
+                        in2 = torch.cuda.Event(); in2.record(side)
+                    dw.step(0, Lh)
+                    done1 = torch.cuda.Event(); done1.record(stream)
+                    with torch.cuda.stream(side):
+                        side.wait_event(done1)
+                        hout[0:Lh].copy_(dw.out[0:Lh], non_blocking=True)
+                    stream.wait_event(in2)
+                    dw.step(Lh, L)
+                    hout[Lh:L].copy_(dw.out[Lh:L], non_blocking=True)
+                    stream.wait_stream(side)                   # join
+
             def e2e_step():
-                dw.q.copy_(hq, non_blocking=True)
-                dw.k_new.copy_(hk, non_blocking=True)
-                if hv is not None:
-                    dw.v_new.copy_(hv, non_blocking=True)
-                run()
-                hout.copy_(dw.out, non_blocking=True)
+                if e2e_graph is not None:
+                    e2e_graph.replay()
+                else:
+                    dw.q.copy_(hq, non_blocking=True)
+                    dw.k_new.copy_(hk, non_blocking=True)
+                    if hv is not None:
+                        dw.v_new.copy_(hv, non_blocking=True)
+                    run()
+                    hout.copy_(dw.out, non_blocking=True)
                 stream.synchronize()
             for _ in range(2):
                 e2e_step()
