@@ -269,7 +269,7 @@ def test_decode_matches_oracle(H, name, lens, window):
 
 
 @pytest.mark.parametrize("spec_args,lens,window", [
-    ((1, 16, 8, 256, 256, False), [30000, 9000], 0),       # ~66 chunks per CTA through a 12-slot ring
+    ((1, 16, 8, 256, 256, False), [30000, 9000], 0),       # ~66 chunks per CTA through a 20-slot ring
     ((1, 32, 8, 128, 128, False), [40000, 23000], 0),      # ~106 chunks per CTA through a 32-slot ring
     ((1, 16, 8, 256, 256, False), [30000, 9000], 1024),
     ((1, 16, 16, 192, 128, False), [20000, 5000], 0),      # d_qk 192 / d_v 128, one query head per KV head
