@@ -449,17 +449,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   }
 }
 
-// grid: (16 heads, n_agents), 512 threads; combines the records of one (agent, head).  The records sit in L2 a
-// microsecond away, so nothing here is a chain of dependent loads: thread s fetches (m, l) of split s, the block
-// agrees on the weights, then four groups of 128 threads each take every fourth split with their loads issued
-// together, and the groups' sums meet in shared memory.
-constexpr int kMergeThreads = 512, kMaxSplits = 512;
+// grid: (16 heads, n_agents, 4 quarters of the value dims), 512 threads; combines the records of one (agent, head)
+// for 128 output dims.  The records sit in L2 a microsecond away, so nothing here is a chain of dependent loads: thread
+// s fetches (m, l) of split s, the block agrees on the weights, while sixteen groups of 32 threads each take every
+// sixteenth split with their loads issued together (up to 64 splits are in flight before the weights are known),
+// and the groups' sums meet in shared memory.  Four CTAs per (agent, head) rather than one: a quarter of the record
+// bytes per CTA and four times the SMs pulling them (4.1 -> see the profile).
+constexpr int kMergeThreads = 512, kMaxSplits = 512, kMergeGroups = kMergeThreads / 32, kMergeQuarters = 4;
 __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_splits, const float* __restrict__ records,
                                                                   void* __restrict__ out, int out_dtype,
                                                                   float* __restrict__ lse) {
   __shared__ float s_w[kMaxSplits];                      // weight of each split (0: empty)
   __shared__ float s_red[kMergeThreads / 32][2];
-  __shared__ float4 s_acc[3][128];
+  __shared__ float4 s_acc[kMergeGroups - 1][32];
   __shared__ float s_ml[2];
   const int h = blockIdx.x, a = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -467,14 +469,14 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
   if (h >= Hq) return;
   const float* rec = records + ((size_t)a * n_splits * kHeads + h) * kRecStride;
   const size_t step = (size_t)kHeads * kRecStride;       // between the splits of one head
-  // The record loads of the first 4 * kPre splits do not wait for the weights: they are issued first and overlap the
+  // The record loads of the first 16 * kPre splits do not wait for the weights: they are issued first and overlap the
   // round trip of the (m, l) loads (an empty split's data is whatever an earlier call left there; it is dropped below).
-  constexpr int kPre = 10;
-  const int grp = tid >> 7, d = 4 * (tid & 127);         // 128 threads x 4 consecutive dims per group
+  constexpr int kPre = 4;
+  const int grp = warp, d = (kDv / kMergeQuarters) * blockIdx.z + 4 * lane;   // 32 lanes x 4 consecutive dims per group
   float4 pre[kPre];
 #pragma unroll
   for (int u = 0; u < kPre; ++u) {
-    const int sp = grp + 4 * u;
+    const int sp = grp + kMergeGroups * u;
     pre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (sp < n_splits) {
       const float2 lo2 = *reinterpret_cast<const float2*>(rec + sp * step + d);       // records are 8-byte aligned
@@ -508,14 +510,14 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
   for (int u = 0; u < kPre; ++u) {
-    const int sp = grp + 4 * u;
+    const int sp = grp + kMergeGroups * u;
     const float wu = sp < n_splits ? s_w[sp] : 0.f;
     if (wu > 0.f) {                                      // an empty split's record holds no data
       acc.x = fmaf(wu, pre[u].x, acc.x); acc.y = fmaf(wu, pre[u].y, acc.y);
       acc.z = fmaf(wu, pre[u].z, acc.z); acc.w = fmaf(wu, pre[u].w, acc.w);
     }
   }
-  for (int sp = grp + 4 * kPre; sp < n_splits; sp += 4) {
+  for (int sp = grp + kMergeGroups * kPre; sp < n_splits; sp += kMergeGroups) {
     const float wu = s_w[sp];
     if (wu > 0.f) {
       const float2 lo2 = *reinterpret_cast<const float2*>(rec + sp * step + d);
@@ -524,13 +526,13 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
       acc.z = fmaf(wu, hi2.x, acc.z); acc.w = fmaf(wu, hi2.y, acc.w);
     }
   }
-  if (grp > 0) s_acc[grp - 1][tid & 127] = acc;
+  if (grp > 0) s_acc[grp - 1][lane] = acc;
   __syncthreads();
   if (grp > 0) return;
   const float Lsum = s_ml[1];
   const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
 #pragma unroll
-  for (int g = 0; g < 3; ++g) { const float4 o = s_acc[g][tid]; acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
+  for (int g = 0; g < kMergeGroups - 1; ++g) { const float4 o = s_acc[g][lane]; acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
   acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
   const size_t out_index = ((size_t)a * Hq + h) * kDv;
   if (out_dtype == Q4KV_OUT_BF16) {
@@ -542,7 +544,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_mla_kernel(int Hq, int n_
   } else {
     *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + out_index + d) = acc;
   }
-  if (tid == 0 && lse) lse[(size_t)a * Hq + h] = Lsum > 0.f ? (s_ml[0] + log2f(Lsum)) / kLog2e : -INFINITY;
+  if (tid == 0 && blockIdx.z == 0 && lse) lse[(size_t)a * Hq + h] = Lsum > 0.f ? (s_ml[0] + log2f(Lsum)) / kLog2e : -INFINITY;
 }
 
 struct MlaPlan { int n_splits, blocks_per_split; };
@@ -607,7 +609,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   e = cudaLaunchKernelEx(&cfg, decode_mla_kernel, P);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t mcfg = {};
-  mcfg.gridDim = dim3(kHeads, b.n_agents);
+  mcfg.gridDim = dim3(kHeads, b.n_agents, kMergeQuarters);
   mcfg.blockDim = dim3(kMergeThreads);
   mcfg.stream = st;
   mcfg.attrs = attr;
