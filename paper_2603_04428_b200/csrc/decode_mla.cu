@@ -164,6 +164,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
   __syncthreads();
   if (threadIdx.x < 2 && threadIdx.x < n_iter)           // the first two block-table entries, fetched towards the SM meanwhile
     asm volatile("prefetch.global.L1 [%0];" ::"l"(P.tables + (size_t)a * P.max_blocks + ((2 * (b0 + (int)threadIdx.x)) >> 3)) : "memory");
+  // While the preceding kernel drains, L2 is asked for the agent's query rows (a prefetch returns nothing to the kernel,
+  // so it may precede the wait; in a decode step they are what the preceding kernels have just written).
+  {
+    const int lines = n_rep * kD * 2 / 128;                // 128-byte lines of the agent's n_rep query rows
+    const uint16_t* qrows = P.q + (size_t)a * y.Hq * kD;
+    for (int i = threadIdx.x; i < lines; i += kThreads) asm volatile("prefetch.global.L2 [%0];" ::"l"(qrows + i * 64));
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the new token was appended by the preceding kernel
   volatile int* abort_flag = &sm.abort_flag;
 
