@@ -125,7 +125,7 @@ class DeviceWorkload:
     """All state of one workload resident on the GPU: the Q4 pool (filled by the library's own quantizer
     from seeded on-device N(0,1) bf16 values), block tables, per-layer q / new K,V, outputs."""
 
-    def __init__(self, w: synth.Workload, device_index: int, two_calls: bool = False):
+    def __init__(self, w: synth.Workload, device_index: int, two_calls: bool = False, exact_products: bool = False):
         import torch
         from paper_2603_04428_b200 import binding as B, harness as H
         self.torch, self.B, self.w = torch, B, w
@@ -134,7 +134,7 @@ class DeviceWorkload:
         self.n_blocks = w.blocks_needed() + 4
         tabs = synth.block_tables(w.seed, 99, w.lens, self.n_blocks, extra_tokens=w.new_tokens)
         self.dc = H.DeviceCache(L, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k, self.n_blocks, tabs,
-                                fill_byte=None)
+                                fill_byte=None, exact_products=exact_products)
         dc = self.dc
         g = torch.Generator(device="cuda")
         g.manual_seed(w.seed)
@@ -389,7 +389,8 @@ def measure(w, args, local, dist=None, full=True):
     region of at least half a second (median batch), the per-launch time of the attention kernel from a graph of the L
     attention calls, clocks sampled meanwhile; with full=True also the end-to-end step through host buffers."""
     import torch
-    dw = DeviceWorkload(w, local, two_calls=args.two_calls)
+    dw = DeviceWorkload(w, local, two_calls=args.two_calls or (args.exact_products and w.v_aliases_k),
+                        exact_products=args.exact_products)
     L = w.n_layers
     use_graph = not args.no_graph
     stream = torch.cuda.Stream()
@@ -576,6 +577,8 @@ def main():
                     help="decode step as a quantize-append launch plus an attention launch per layer instead of the "
                          "one-launch update-and-fetch")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="least duration of each timed region")
+    ap.add_argument("--exact-products", action="store_true",
+                    help="set q4kv_spec.exact_products: every call takes the kernels that multiply the 4-bit codes exactly")
     ap.add_argument("--op", default="step", choices=["step", "pack", "unpack"],
                     help="step: the append + attention step of --workload; pack: q4kv_pack / q4kv_unpack / bulk append")
     ap.add_argument("--agents", type=int, default=0,
@@ -586,7 +589,7 @@ def main():
         print(json.dumps(run_pack(args)))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
-    default_run = args.workload is None and args.agents == 0 and args.layers == 0
+    default_run = args.workload is None and args.agents == 0 and args.layers == 0 and not args.exact_products
     w = synth.workload(1 if args.workload is None else args.workload)
     if args.agents > 0 or args.layers > 0:
         # not one of the five configurations any more: the name says so, and no stored counter applies to it
@@ -596,6 +599,9 @@ def main():
         lens = [w.lens[0]] * args.agents if args.agents > 0 else w.lens
         layers = args.layers if args.layers > 0 else w.n_layers
         w = dataclasses.replace(w, lens=lens, n_layers=layers, name=f"{w.name}_scaled_{len(lens)}agents_{layers}layers")
+    if args.exact_products:
+        import dataclasses
+        w = dataclasses.replace(w, name=w.name + "_exact_products")       # other kernels: no stored counter applies
     if args.impl == "reference":
         run_reference(args, w)
         return
