@@ -81,6 +81,7 @@ def test_decode_long_context_wraps_the_ring(H):
 @pytest.mark.parametrize("name,lens,window", [
     ("gqa128", [1000, 700, 0, 255, 256, 257, 31, 32, 33], 0),
     ("gqa256", [1500, 41, 2049], 1024),
+    ("asym", [700, 33, 0, 256], 0),
 ])
 def test_update_and_fetch_in_one_launch(H, name, lens, window):
     steps = 3
@@ -190,3 +191,29 @@ def test_saved_image_names_bf16_and_restores(H, name, lens):
     with pytest.raises(B.Q4KVError):
         p3.dc.restore(0, p.dc.save(0, lens[0]).pin_memory(), staging_layers=1)
     assert p.dc.read_flags() == 0 and p2.dc.read_flags() == 0
+
+
+def test_layer_batched_entry_and_static_entry(H):
+    """The layer-batched entry and the entry without a caller workspace on a bfloat16 cache."""
+    from paper_2603_04428_b200 import binding as B
+    spec_args, lens = (3, 8, 2, 128, 128, False), [700, 33, 300]
+    p = Pair(H, spec_args, lens, seed=171, sb_dtype=1).fill()
+    s = p.ospec
+    L, A = s.n_layers, len(lens)
+    scale = 1.0 / math.sqrt(s.d_qk)
+    q_all = np.stack([p.q(80 + l, A) for l in range(L)])
+    out = torch.full((L, A, s.n_q_heads, s.d_v), float("nan"), device="cuda")
+    lse = torch.full((L, A, s.n_q_heads), float("nan"), device="cuda")
+    ws = torch.zeros(B.q4kv_workspace_bytes_layers(p.dc.spec, A, p.dc.bt.max_blocks * 256, L), dtype=torch.uint8, device="cuda")
+    lens_d = H.dev(np.asarray(lens, dtype=np.int32))
+    B.q4kv_decode_attention_layers(p.dc.spec, p.dc.pool, p.dc.n_blocks, 0, L, p.dc.bt, lens_d, 0, [0] * L, None, None,
+                                   H.bf16_dev(q_all), scale, out, B.OUT_F32, lse, ws, p.dc.flags)
+    out_s = torch.full((A, s.n_q_heads, s.d_v), float("nan"), device="cuda")
+    for l in range(L):
+        ref, lse_ref = O.decode_attention(p.opool, l, p.tabs, lens, 0, f32(q_all[l]), scale)
+        assert_attention_close(out[l].cpu().numpy(), ref, f"layer {l}")
+        assert_lse_close(lse[l].cpu().numpy(), lse_ref)
+        B.q4kv_decode_attention_static(p.dc.spec, p.dc.pool, p.dc.n_blocks, l, p.dc.bt, lens_d, 0, 0, H.bf16_dev(q_all[l]),
+                                       scale, out_s, B.OUT_F32, None, p.dc.flags)
+        assert_attention_close(out_s.cpu().numpy(), ref, f"static entry, layer {l}")
+    assert p.dc.read_flags() == 0
