@@ -389,8 +389,7 @@ def measure(w, args, local, dist=None, full=True):
     region of at least half a second (median batch), the per-launch time of the attention kernel from a graph of the L
     attention calls, clocks sampled meanwhile; with full=True also the end-to-end step through host buffers."""
     import torch
-    dw = DeviceWorkload(w, local, two_calls=args.two_calls or (args.exact_products and w.v_aliases_k),
-                        exact_products=args.exact_products)
+    dw = DeviceWorkload(w, local, two_calls=args.two_calls, exact_products=args.exact_products)
     L = w.n_layers
     use_graph = not args.no_graph
     stream = torch.cuda.Stream()
@@ -775,8 +774,8 @@ def fused_update_and_fetch(w):
     """Decode shapes that q4kv_append_decode_attention covers (one launch per layer for append + attention)."""
     if w.kind != "decode":
         return False
-    if w.v_aliases_k:      # the MLA-latent cache (at the usual softmax scales)
-        return (w.d_qk, w.d_v, w.n_kv_heads) == (576, 512, 1) and w.n_q_heads <= 16 and w.softmax_scale ** 2 * w.d_qk <= 4
+    if w.v_aliases_k:      # the MLA-latent cache
+        return (w.d_qk, w.d_v, w.n_kv_heads) == (576, 512, 1) and w.n_q_heads <= 16
     n_rep = w.n_q_heads // w.n_kv_heads
     return n_rep <= 4 and ((w.d_qk == w.d_v and w.d_qk in (128, 256)) or (w.d_qk, w.d_v) == (192, 128))
 

@@ -51,21 +51,7 @@ constexpr int kRecStride = kDv + 2;                      // acc[512], m, l
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLazy = 8.f;
 
-struct MlaParams {
-  Layout y;
-  const uint8_t* pool;
-  int n_blocks, layer, n_agents, max_blocks;
-  const int32_t* tables;
-  const int32_t* kv_lens;
-  int len_cap;
-  int window;
-  const uint16_t* q;          // bf16 [n_agents][Hq][576]
-  const uint16_t* k_new;      // bf16 [n_agents][576]: the row at position kv_len - 1, quantized and stored by this launch; or null
-  float scale_log2;
-  int n_splits, blocks_per_split;
-  float* records;             // [n_agents][n_splits][16][kRecStride]
-  int32_t* flags;
-};
+using MlaParams = MlaDecodeParams;
 
 struct MlaSmem {
   alignas(128) uint8_t khat[kStages][kTileBytes];        // [key 64][dim 576]: (key%8)*16 + (key/8)*9216 + (dim/8)*128
@@ -583,7 +569,8 @@ size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len)
 
 cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale, void* out,
-                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st, const void* k_new) {
+                              int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st, const void* k_new,
+                              bool on_codes) {
   if (b.n_agents <= 0) return cudaSuccess;
   MlaPlan plan = plan_mla(b.n_agents, max_kv_len, window);
   const MlaPlan full = plan_mla(b.n_agents, max_kv_len, 0);
@@ -593,27 +580,32 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.len_cap = max_kv_len; P.window = window;
   P.q = (const uint16_t*)q; P.k_new = (const uint16_t*)k_new; P.scale_log2 = scale * kLog2e; P.n_splits = plan.n_splits;
   P.blocks_per_split = plan.blocks_per_split; P.records = (float*)ws; P.flags = flags;
-  static bool configured[64] = {};
-  const size_t smem = sizeof(MlaSmem);
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(decode_mla_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
-  }
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(plan.n_splits, b.n_agents);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, decode_mla_kernel, P);
+  cudaError_t e;
+  if (on_codes) {
+    e = launch_mla_codes_kernel(P, st);
+  } else {
+    static bool configured[64] = {};
+    const size_t smem = sizeof(MlaSmem);
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+      e = cudaFuncSetAttribute(decode_mla_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.n_splits, b.n_agents);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, decode_mla_kernel, P);
+  }
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t mcfg = {};
   mcfg.gridDim = dim3(kHeads, b.n_agents, kMergeQuarters);

@@ -123,9 +123,9 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
   void* records = (uint8_t*)workspace + kWorkspaceHeaderBytes;
   cudaError_t e;
-  if (decode_mla_supported(y) && tiles_allowed(spec, softmax_scale))
+  if (decode_mla_supported(y))
     e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale, out, out_dtype,
-                          lse, records, status_flags, (cudaStream_t)stream);
+                          lse, records, status_flags, (cudaStream_t)stream, nullptr, !tiles_allowed(spec, softmax_scale));
   else if (decode_mma_supported(y) && decode_mma_fits(y, batch->n_agents, batch->max_blocks))
     e = launch_decode_mma(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, &window, 1, q, softmax_scale, out,
                           out_dtype, lse, workspace, status_flags, (cudaStream_t)stream);
@@ -157,12 +157,10 @@ int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_bl
   if (max_kv_len == 0 || max_kv_len > cap) max_kv_len = cap;
   const Layout y = make_layout(*spec, n_blocks);
   if (decode_mla_supported(y)) {
-    // the latent-cache kernel expands the keys into binary16 tiles (see q4kv_decode_attention)
-    if (!tiles_allowed(spec, softmax_scale)) return Q4KV_EUNSUPPORTED;
     if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, 0)) return Q4KV_EWORKSPACE;
     const cudaError_t e = launch_decode_mla(y, pool, n_blocks, layer, *batch, kv_lens, max_kv_len, window, q, softmax_scale,
                                             out, out_dtype, lse, (uint8_t*)workspace + kWorkspaceHeaderBytes, status_flags,
-                                            (cudaStream_t)stream, k_new);
+                                            (cudaStream_t)stream, k_new, !tiles_allowed(spec, softmax_scale));
     return e == cudaSuccess ? Q4KV_OK : Q4KV_ECUDA;
   }
   if (!decode_mma_supported(y) || !decode_mma_fits(y, batch->n_agents, batch->max_blocks)) return Q4KV_EUNSUPPORTED;

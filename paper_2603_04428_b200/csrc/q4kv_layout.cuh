@@ -155,12 +155,32 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
                                 const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
                                 float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
 
-// tcgen05 decode path for the MLA-latent cache (d_qk 576, d_v 512 aliasing K, one KV head, at most 16 query heads)
+// Decode on the MLA-latent cache (d_qk 576, d_v 512 aliasing K, one KV head, at most 16 query heads): a key-split
+// attention kernel -- on a binary16 tile of the dequantized keys, or, with on_codes, on the 4-bit codes themselves
+// (exact products; the only form for bfloat16 scales and biases) -- followed by the combination of the records.
 bool decode_mla_supported(const Layout& y);
 size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len);
 cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                               const int32_t* kv_lens, int max_kv_len, int window, const void* q, float scale, void* out,
                               int out_dtype, float* lse, void* ws, int32_t* flags, cudaStream_t st,
-                              const void* k_new = nullptr);   // k_new: update-and-fetch (the pool is written)
+                              const void* k_new = nullptr,    // k_new: update-and-fetch (the pool is written)
+                              bool on_codes = false);
+// what the two attention kernels receive
+struct MlaDecodeParams {
+  Layout y;
+  const uint8_t* pool;
+  int n_blocks, layer, n_agents, max_blocks;
+  const int32_t* tables;
+  const int32_t* kv_lens;
+  int len_cap;
+  int window;
+  const uint16_t* q;          // bf16 [n_agents][Hq][576]
+  const uint16_t* k_new;      // bf16 [n_agents][576]: the row at position kv_len - 1, quantized and stored by this launch; or null
+  float scale_log2;
+  int n_splits, blocks_per_split;
+  float* records;             // [n_agents][n_splits][16][514]: acc[512] (unnormalised, relative to m), m, l
+  int32_t* flags;
+};
+cudaError_t launch_mla_codes_kernel(const MlaDecodeParams& P, cudaStream_t st);   // grid (n_splits, n_agents)
 
 }  // namespace q4kv

@@ -109,24 +109,35 @@ def test_update_and_fetch_in_one_launch(H, name, lens, window):
     assert p.dc.read_flags() == 0
 
 
-def test_latent_cache_fused_entry_is_refused_and_the_two_call_form_works(H):
-    """The latent-cache kernel expands keys into binary16 tiles, which bfloat16 scales can overflow: the fused entry
-    says so; quantize-append followed by decode attention serves such a cache."""
-    from paper_2603_04428_b200 import binding as B
-    lens = [300, 64]
-    p = Pair(H, SPECS["mla"], lens, seed=140, extra_tokens=1, sb_dtype=1).fill()
+def test_latent_cache_update_and_fetch_runs_on_the_codes(H):
+    """A bfloat16 scale can lie outside binary16's range, so the latent-cache kernel that expands keys into binary16
+    tiles never serves such a cache: the kernel that multiplies the codes does, through both entries."""
+    lens = [300, 64, 1000]
+    steps = 2
+    p = Pair(H, SPECS["mla"], lens, seed=140, extra_tokens=steps, sb_dtype=1).fill()
     s = p.ospec
-    kb = synth.kv_bf16(140, 500, 2, s.n_kv_heads, s.d_qk)
-    q = p.q(70, 2)
-    new_lens = [n + 1 for n in lens]
-    with pytest.raises(B.Q4KVError):
-        p.dc.append_decode(0, new_lens, 0, kb, None, q, 1.0 / math.sqrt(192))
-    O.quantize_append(p.opool, 0, p.tabs, lens, [0, 1, 2], f32(kb), None)
-    p.dc.append(0, lens, [0, 1, 2], kb, None)
-    ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, new_lens, 0, f32(q), 1.0 / math.sqrt(192))
-    out, lse = p.dc.decode(0, new_lens, 0, q, 1.0 / math.sqrt(192))
-    assert_attention_close(out.cpu().numpy(), ref)
-    assert_lse_close(lse.cpu().numpy(), lse_ref)
+    A = len(lens)
+    cur = list(lens)
+    scale = 1.0 / math.sqrt(192)
+    for step in range(steps):
+        kb = synth.kv_bf16(140, 500 + step, A, s.n_kv_heads, s.d_qk)
+        q = p.q(70 + step, A)
+        new_lens = [n + 1 for n in cur]
+        O.quantize_append(p.opool, 0, p.tabs, cur, list(range(A + 1)), f32(kb), None)
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, new_lens, 0, f32(q), scale)
+        out, lse = p.dc.append_decode(0, new_lens, 0, kb, None, q, scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"step {step}")
+        assert_lse_close(lse.cpu().numpy(), lse_ref)
+        out, lse = p.dc.decode(0, new_lens, 0, q, scale)
+        assert_attention_close(out.cpu().numpy(), ref, f"two calls, step {step}")
+        cur = new_lens
+    for l in range(1, s.n_layers):                              # the other layers get the same rows through quantize-append
+        for step in range(steps):
+            kb = synth.kv_bf16(140, 500 + step, A, s.n_kv_heads, s.d_qk)
+            O.quantize_append(p.opool, l, p.tabs, [n + step for n in lens], list(range(A + 1)), f32(kb), None)
+            p.dc.append(l, [n + step for n in lens], list(range(A + 1)), kb, None)
+    p.lens = cur
+    p.check_packed_equal()
     assert p.dc.read_flags() == 0
 
 

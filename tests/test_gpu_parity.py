@@ -522,9 +522,45 @@ def test_decode_latent_cache_at_a_sharp_scale_takes_the_exact_kernel(H, window):
     assert p.dc.read_flags() == 0
 
 
+@pytest.mark.parametrize("lens,window,scale,exact", [
+    ([1000, 700, 0, 63, 64, 65, 129, 31, 32, 33], 0, 0.1, False),       # a sharp scale: 64-key block and chunk edges
+    ([2500, 300, 4000], 200, 1.0 / math.sqrt(192), True),               # exact products asked for, a window
+    ([9000, 1], 0, 0.1, True),                                          # many blocks per key share
+])
+def test_latent_cache_update_and_fetch_on_the_codes(H, lens, window, scale, exact):
+    """The latent-cache calls that may not round the cache (exact_products, or scale^2 * d_qk > 4) run on the kernel
+    that multiplies the 4-bit codes: update-and-fetch and the two-call form, pool bytes as quantize-append writes
+    them, and the result within the bound of the exact routes (2e-5 * M + 1e-5, M the largest dequantized magnitude)."""
+    steps = 2
+    p = Pair(H, SPECS["mla"], lens, seed=45, extra_tokens=steps, exact_products=exact).fill()
+    s = p.ospec
+    A = len(lens)
+    cur = list(lens)
+    live = [a for a in range(A) if lens[a] > 0]
+    for step in range(steps):
+        kb = synth.kv_bf16(45, 500 + step, A, s.n_kv_heads, s.d_qk)
+        q = p.q(70 + step, A)
+        new_lens = [n + 1 if lens[a] > 0 else 0 for a, n in enumerate(cur)]
+        offs = np.concatenate([[0], np.cumsum([1 if a in live else 0 for a in range(A)])]).astype(np.int32)
+        O.quantize_append(p.opool, 0, p.tabs, cur, offs, f32(kb[live]), None)
+        ref, lse_ref = O.decode_attention(p.opool, 0, p.tabs, new_lens, window, f32(q), scale)
+        out, lse = p.dc.append_decode(0, new_lens, window, kb, None, q, scale)
+        p.lens = new_lens
+        M = max_dequantized_magnitude(p, 0)
+        for what, (o, ls) in (("one launch", (out, lse)), ("two calls", p.dc.decode(0, new_lens, window, q, scale))):
+            assert_attention_close(o.cpu().numpy(), ref, f"{what}, step {step}")
+            assert_lse_close(ls.cpu().numpy(), lse_ref, what)
+            assert np.abs(o.cpu().numpy().astype(np.float64) - ref).max() <= 2e-5 * M + 1e-5, what
+        cur = new_lens
+    p.check_packed_equal()
+    assert p.dc.read_flags() == 0
+
+
 def max_dequantized_magnitude(p, layer):
     m = 0.0
     for a, n in enumerate(p.lens):
+        if n == 0:
+            continue
         K, V = O.gather_dequant(p.opool, layer, p.tabs[a], 0, n, 0)
         m = max(m, float(np.abs(K).max()), float(np.abs(V).max()))
     return m
