@@ -109,8 +109,9 @@ enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
  * dequantized values evaluated in float64).  Let M be the largest |code*scale + bias| among the
  * attended keys and values.
  *   - Kernels that multiply the 4-bit codes (decode with d_qk = d_v in {128, 256} or d_qk 192 / d_v 128
- *     and at most four query heads per KV head; prefill with d = 128 and exact_products = 1; the shape-agnostic
- *     kernels every other case falls back to): the products are exact, sums are float32, the
+ *     and at most four query heads per KV head; decode on the MLA-latent cache when the tile kernel
+ *     below is not allowed; prefill with d in {128, 256} when it is not; the shape-agnostic kernels
+ *     every other case falls back to): the products are exact, sums are float32, the
  *     probabilities enter the value product as a two-term binary16 pair or as float32.  Error
  *     at most 2e-5 * M + 1e-5, i.e. within 2e-3 for any cache with M <= 64.  (An absolute bound:
  *     the tensor-core kernels carry probability x scale in binary16, so contributions of groups
@@ -190,9 +191,8 @@ int q4kv_decode_attention(const q4kv_spec* spec, const void* pool, int32_t n_blo
  *                 (v_new is ignored, and may be NULL, when V aliases K)
  * All other arguments as in q4kv_decode_attention.  Covered specs: d_qk = d_v in {128, 256}, or d_qk 192
  * with d_v 128 (the per-head MLA cache of Section 3.6), with at most four query heads per KV head and V
- * not aliasing K; and the MLA-latent cache (V aliasing K,
- * d_qk 576, d_v 512, one KV head, at most 16 query heads) with exact_products == 0, binary16
- * scales and biases, and softmax_scale^2 * d_qk <= 4.
+ * not aliasing K; and the MLA-latent cache (V aliasing K, d_qk 576, d_v 512, one KV head, at most
+ * 16 query heads), on the kernel q4kv_decode_attention would take for the same spec and scale.
  * Anything else returns Q4KV_EUNSUPPORTED and the caller makes the two calls.  Two agents must
  * not share the block that is written. */
 int q4kv_append_decode_attention(const q4kv_spec* spec, void* pool, int32_t n_blocks, int32_t layer,
