@@ -15,6 +15,7 @@ N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no c
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import math
 import os
@@ -379,7 +380,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # fewer layers (the launch itself is the full-size one, so nothing is scaled); the config-3 figure is a global layer's
 # launch, the MLA figure the attention kernel without its merge launch (4.88 MB more when its records miss L2).
 NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23_991_723, "gemma3_12b_ragged_decode": 365_462_784,
-                     "dsv2lite_mla_decode": 21_440_640, "llama31_8b_chunked_prefill": 240_450_688,
+                     "dsv2lite_mla_decode": 21_440_640, "dsv2lite_mla_decode_exact_products": 21_446_656,
+                     "llama31_8b_chunked_prefill": 240_450_688,
                      "dsv2lite_perhead_mla_decode": 191_148_800, "gemma3_12b_shaped_global_prefill": 154_507_000,
                      "pack": 254_257_000, "unpack": 251_510_000, "append_8x1024": 33_606_912}
 
@@ -592,14 +594,12 @@ def main():
     w = synth.workload(1 if args.workload is None else args.workload)
     if args.agents > 0 or args.layers > 0:
         # not one of the five configurations any more: the name says so, and no stored counter applies to it
-        import dataclasses
         if args.agents > 0 and len(set(w.lens)) != 1:
             raise SystemExit("--agents scales configurations whose agents have one common length")
         lens = [w.lens[0]] * args.agents if args.agents > 0 else w.lens
         layers = args.layers if args.layers > 0 else w.n_layers
         w = dataclasses.replace(w, lens=lens, n_layers=layers, name=f"{w.name}_scaled_{len(lens)}agents_{layers}layers")
     if args.exact_products:
-        import dataclasses
         w = dataclasses.replace(w, name=w.name + "_exact_products")       # other kernels: no stored counter applies
     if args.impl == "reference":
         run_reference(args, w)
@@ -638,15 +638,23 @@ def main():
     }
     if rank == 0 and world == 1 and default_run and not args.no_all_configs:
         allc = {}
-        for idx in (2, 3, 4, 5, 6):
-            wi = synth.workload(idx)
-            ri = measure(wi, args, local, None, full=False)
+
+        def entry(wi, ai):
+            ri = measure(wi, ai, local, None, full=False)
             units_i, roof_i = roofline_of(wi, ri)
             mi, ui, di = metric_of(wi)
             allc[wi.name] = {"metric": mi, "value": units_i / ri["t_step"] / di, "unit": ui,
                              "ms_per_step": ri["t_step"] * 1e3, "agent_steps_per_s": wi.n_agents / ri["t_step"],
                              "append_avg_us": ri["app_s"] * 1e6, "roofline": roof_i, "config": config_of(wi, ri),
-                             "gpu_launches_per_step": dw_launches(wi, args.two_calls), "clocks": ri["clocks"]}
+                             "gpu_launches_per_step": dw_launches(wi, ai.two_calls), "clocks": ri["clocks"]}
+
+        for idx in (2, 3, 4, 5, 6):
+            entry(synth.workload(idx), args)
+        # the MLA-latent decode again with q4kv_spec.exact_products set: the kernel that multiplies the codes (also the
+        # route of bfloat16 caches and sharp softmax scales)
+        w3 = synth.workload(3)
+        entry(dataclasses.replace(w3, name=w3.name + "_exact_products"),
+              argparse.Namespace(**{**vars(args), "exact_products": True}))
         pk = run_pack(args)
         for name in ("pack", "unpack", "restore", "append_8x1024"):
             allc[name] = pk["kernels"][name]
