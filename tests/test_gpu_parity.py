@@ -415,10 +415,12 @@ def test_bf16_output_mode(H):
     ((1, 16, 1, 576, 512, True), [9000, 300], 1000),                 # a window that starts inside a 64-key block
     ((2, 8, 1, 576, 512, True), [2100], 0),                          # fewer than 16 heads, two layers
 ])
-def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
-    """The MLA-latent decode kernel: one binary16 tile per 64 keys serves as key and as value operand."""
+@pytest.mark.parametrize("exact", [False, True], ids=["tile", "codes"])
+def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window, exact):
+    """The MLA-latent decode kernels: one binary16 tile per 64 keys serves as key and as value operand; with
+    exact_products the 4-bit codes themselves do."""
     from paper_2603_04428_b200 import binding as B
-    p = Pair(H, spec_args, lens, seed=37).fill()
+    p = Pair(H, spec_args, lens, seed=37, exact_products=exact).fill()
     s = p.ospec
     q = p.q(7, len(lens))
     scale = 1.0 / math.sqrt(192)
@@ -443,6 +445,13 @@ def test_decode_mla_latent_tensor_memory_path(H, spec_args, lens, window):
             assert torch.all(bad[0] == 0) and torch.isneginf(lse_bad[0]).all()
         assert torch.allclose(bad[1:], out32[1:], atol=1e-5)
         p.dc.flags.zero_()
+    # a length beyond the block table is reported, and that agent's rows are zero
+    over = [p.tabs.shape[1] * 256 + 1] + list(lens[1:])
+    bad, lse_bad = p.dc.decode(0, over, window, q, scale)
+    assert p.dc.read_flags() & B.FLAG_BAD_LENGTH
+    assert torch.all(bad[0] == 0) and torch.isneginf(lse_bad[0]).all()
+    assert torch.allclose(bad[1:], out32[1:], atol=1e-5)
+    p.dc.flags.zero_()
 
 
 @pytest.mark.parametrize("name,lens,window", [
