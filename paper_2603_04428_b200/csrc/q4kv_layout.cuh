@@ -155,6 +155,13 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
                                 const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
                                 float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
 
+// tcgen05 prefill path for d_qk = d_v = 256 (1, 2 or 4 query heads per KV head): one 128-row tile per CTA, two score buffers
+bool prefill_umma256_supported(const Layout& y);
+cudaError_t launch_prefill_umma256(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                                   const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window,
+                                   const void* q, float scale, void* out, int out_dtype, float* lse, int32_t* flags,
+                                   cudaStream_t st);
+
 // Decode on the MLA-latent cache (d_qk 576, d_v 512 aliasing K, one KV head, at most 16 query heads): a key-split
 // attention kernel -- on a binary16 tile of the dequantized keys, or, with on_codes, on the 4-bit codes themselves
 // (exact products; the only form for bfloat16 scales and biases) -- followed by the combination of the records.
