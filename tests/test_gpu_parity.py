@@ -839,6 +839,11 @@ class QuietStartPair(Pair):
     ((1, 8, 2, 128, 128, False), [1500, 64], [129, 64], 0, 8.0),         # a sharp scale is routed to the exact-code kernel
     ((1, 6, 2, 128, 128, False), [700, 30], [100, 64], 0, 1.0),          # three query heads per KV head: exact-code kernel
     ((1, 4, 4, 128, 128, False), [0], [257], 0, 1.0),                    # no prefix at all: purely causal
+    ((1, 4, 2, 256, 256, False), [900, 5], [140, 70], 0, 1.0),           # d = 256 (one tile per CTA, two score buffers)
+    ((1, 8, 2, 256, 256, False), [3000], [200], 700, 1.0),               # d = 256, four heads per KV head, a window
+    ((1, 8, 2, 256, 256, False), [1500, 64], [129, 64], 0, 2.0),         # d = 256, the row maximum jumps by more than 2^8
+    ((1, 4, 4, 256, 256, False), [0], [257], 0, 1.0),                    # d = 256, no prefix, one head per KV head
+    ((1, 2, 1, 256, 256, False), [6000, 1], [300, 1], 0, 1.0),           # d = 256, ~100 blocks through the two-stage rings; one key
 ])
 def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
     """The tensor-memory prefill kernel: tile shapes for 1, 2 and 4 heads per KV head, key ranges that start
@@ -862,15 +867,16 @@ def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
 
 @pytest.mark.parametrize("gain,outlier_frac", [(8.0, 0.0), (1.0, 0.01)])
 @pytest.mark.parametrize("prefix,chunks", [([0, 40], [70, 30]), ([300], [64])])
-def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks):
+@pytest.mark.parametrize("d", [128, 256])
+def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks, d):
     """Rows that attend 1 to 64 keys of a cache with a gain of 8, or with 1 % of the channels carrying 8x the
     values, return value rows almost verbatim, so a single binary16 rounding of a dequantized value (half an ulp of
     2^-8 for magnitudes in [8, 16)) is visible.  With exact_products the usual bound holds; without it the
     binary16-tile kernel stays inside the bound the header states for it."""
-    spec_args = (1, 8, 2, 128, 128, False)
+    spec_args = (1, 8, 2, d, d, False)
     lens = [p0 + c for p0, c in zip(prefix, chunks)]
     q_offs = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
-    scale = 1.0 / math.sqrt(128)
+    scale = 1.0 / math.sqrt(d)
     for exact in (True, False):
         p = Pair(H, spec_args, lens, seed=48, gain=gain, outlier_frac=outlier_frac, exact_products=exact).fill()
         q = p.q(9, int(q_offs[-1]))
@@ -887,10 +893,11 @@ def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks
         assert p.dc.read_flags() == 0
 
 
-def test_prefill_bad_block_and_bad_length(H):
+@pytest.mark.parametrize("d", [128, 256])
+def test_prefill_bad_block_and_bad_length(H, d):
     from paper_2603_04428_b200 import binding as B
     lens = [600, 200]
-    p = Pair(H, (1, 8, 2, 128, 128, False), lens, seed=53).fill()
+    p = Pair(H, (1, 8, 2, d, d, False), lens, seed=53).fill()
     q_offs = [0, 100, 180]
     q = p.q(7, 180)
     good, _ = p.dc.prefill(0, lens, q_offs, 0, q, 0.1)
@@ -1068,12 +1075,14 @@ def test_full_size_decode_launches_match_the_oracle(H, index):
     assert p.dc.read_flags() == 0
 
 
-def test_full_size_prefill_launch_matches_the_oracle_on_sampled_rows(H):
-    """Configuration 5 as bench.py launches it, one layer: eight agents, 8192 cached + 1024 new tokens each.  The
-    library computes all 8192 x 32 output rows; the oracle checks 24 query rows per agent (all heads), spread over the
-    phase and including its first and last token, for two of the agents, and the appended cache bytes of all."""
-    w = synth.workload(4)
-    p = WorkloadPair(H, w, extra_tokens=w.new_tokens).fill(chunks=[8192])
+@pytest.mark.parametrize("index", [4, 6])
+def test_full_size_prefill_launch_matches_the_oracle_on_sampled_rows(H, index):
+    """Configuration 5 (and the d = 256 phase of bench workload 6) as bench.py launches it, one layer: eight agents,
+    8192 cached + 1024 new tokens each (4096 + 512 at d = 256).  The library computes every output row; the oracle
+    checks 24 query rows per agent (all heads), spread over the phase and including its first and last token, for two
+    of the agents, and the appended cache bytes of all."""
+    w = synth.workload(index)
+    p = WorkloadPair(H, w, extra_tokens=w.new_tokens).fill(chunks=[max(w.lens)])
     A, T = w.n_agents, w.new_tokens
     kb = synth.kv_bf16(w.seed, 501, A * T, w.n_kv_heads, w.d_qk)
     vb = synth.kv_bf16(w.seed, 502, A * T, w.n_kv_heads, w.d_v)
