@@ -460,33 +460,40 @@ def measure(w, args, local, dist=None, full=True):
             hv = None if dw.v_new is None else dw.v_new.cpu().pin_memory()
             hout = torch.empty(dw.out.shape, dtype=dw.out.dtype).pin_memory()
 
-            # The step in two halves of the layers, so that the second half's inputs travel while the first half
-            # computes and the first half's results travel while the second computes: one CUDA graph over two streams
-            # (every input and every result still crosses the host link inside the step).
+            # The step in four runs of layers, so that a run's inputs travel while the runs before it compute and its
+            # results travel while the runs after it compute: one CUDA graph over two streams (every input and every
+            # result still crosses the host link inside the step).
             side = torch.cuda.Stream()
-            Lh = max(1, L // 2)
+            n_seg = 4 if L >= 8 else (2 if L >= 2 else 1)
+            cuts = [L * i // n_seg for i in range(n_seg + 1)]
             e2e_graph = None
-            if use_graph and L >= 2:
-                def half_in(a, b):
+            if use_graph and n_seg >= 2:
+                def run_in(a, b):
                     dw.q[a:b].copy_(hq[a:b], non_blocking=True)
                     dw.k_new[a:b].copy_(hk[a:b], non_blocking=True)
                     if hv is not None:
                         dw.v_new[a:b].copy_(hv[a:b], non_blocking=True)
                 e2e_graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(e2e_graph, stream=stream):
-                    half_in(0, Lh)
+                    run_in(cuts[0], cuts[1])
                     side.wait_stream(stream)                   # fork
+                    arrived = [None]
                     with torch.cuda.stream(side):
-                        half_in(Lh, L)
-                        in2 = torch.cuda.Event(); in2.record(side)
-                    dw.step(0, Lh)
-                    done1 = torch.cuda.Event(); done1.record(stream)
-                    with torch.cuda.stream(side):
-                        side.wait_event(done1)
-                        hout[0:Lh].copy_(dw.out[0:Lh], non_blocking=True)
-                    stream.wait_event(in2)
-                    dw.step(Lh, L)
-                    hout[Lh:L].copy_(dw.out[Lh:L], non_blocking=True)
+                        for i in range(1, n_seg):
+                            run_in(cuts[i], cuts[i + 1])
+                            ev = torch.cuda.Event(); ev.record(side)
+                            arrived.append(ev)
+                    for i in range(n_seg):
+                        if arrived[i] is not None:
+                            stream.wait_event(arrived[i])
+                        dw.step(cuts[i], cuts[i + 1])
+                        if i + 1 < n_seg:
+                            done = torch.cuda.Event(); done.record(stream)
+                            with torch.cuda.stream(side):
+                                side.wait_event(done)
+                                hout[cuts[i]:cuts[i + 1]].copy_(dw.out[cuts[i]:cuts[i + 1]], non_blocking=True)
+                        else:
+                            hout[cuts[i]:cuts[i + 1]].copy_(dw.out[cuts[i]:cuts[i + 1]], non_blocking=True)
                     stream.wait_stream(side)                   # join
 
             def e2e_step():
