@@ -916,6 +916,33 @@ def test_prefill_bad_block_and_bad_length(H, d):
 
 
 
+def test_tensor_memory_prefill_and_latent_decode_repeat_bit_for_bit(H):
+    """The kernels whose warps hand tiles to one another through mbarriers (tensor-memory prefill at d = 128 and 256,
+    latent-cache decode on tiles and on codes) have a fixed order of arithmetic: sixty launches in a row on the same
+    inputs return the same bits, which a missed hand-off (a tile read before it is complete) would not."""
+    for spec_args, prefix, chunk in (((1, 8, 2, 128, 128, False), [1800, 300], 200),
+                                     ((1, 8, 4, 256, 256, False), [1800, 300], 200)):
+        lens = [n + chunk for n in prefix]
+        p = Pair(H, spec_args, lens, seed=91).fill()
+        q_offs = [0, chunk, 2 * chunk]
+        q = H.bf16_dev(p.q(7, 2 * chunk))
+        scale = 1.0 / math.sqrt(spec_args[3])
+        first, lse0 = p.dc.prefill(0, lens, q_offs, 0, q, scale)
+        for _ in range(60):
+            out, lse = p.dc.prefill(0, lens, q_offs, 0, q, scale)
+            assert torch.equal(out, first) and torch.equal(lse, lse0)
+        assert p.dc.read_flags() == 0
+    for exact in (False, True):
+        lens = [5000, 700, 64]
+        p = Pair(H, SPECS["mla"], lens, seed=92, exact_products=exact).fill()
+        q = H.bf16_dev(p.q(7, len(lens)))
+        first, lse0 = p.dc.decode(0, lens, 0, q, 1.0 / math.sqrt(192))
+        for _ in range(60):
+            out, lse = p.dc.decode(0, lens, 0, q, 1.0 / math.sqrt(192))
+            assert torch.equal(out, first) and torch.equal(lse, lse0)
+        assert p.dc.read_flags() == 0
+
+
 # ---- persisted container and warm restore --------------------------------------------------------
 @pytest.mark.parametrize("name,lens", [("gqa128", [700, 33]), ("mla", [300, 256]), ("asym", [17, 513])])
 def test_saved_file_image_equals_the_oracles_and_restores_into_other_blocks(H, name, lens, tmp_path):
