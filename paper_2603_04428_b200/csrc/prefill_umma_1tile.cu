@@ -1,27 +1,29 @@
-// q4kv_prefill_attention, tcgen05 path for d_qk = d_v = 256 (1, 2 or 4 query heads per KV head): the
+// q4kv_prefill_attention, tcgen05 path with one query tile per CTA, for the head shapes whose
+// accumulator leaves no room for two: d_qk = d_v = 256 (the sliding-window model of Section 3.6) and
+// d_qk 192 / d_v 128 (the per-head MLA cache of Section 3.6); 1, 2 or 4 query heads per KV head.  The
 // queries of a new phase over the cached Q4 prefix plus the causal new tokens, read from the Q4
-// cache in place (Sections 3.4 "chunked prefill" and 3.5 "cross-phase context injection"; GQA and
-// the sliding-window layers of Section 3.6, whose model has this head dimension).
+// cache in place (Sections 3.4 "chunked prefill" and 3.5 "cross-phase context injection").
 //
 // The d = 128 kernel's structure with one 128-row tile per CTA: at d = 256 a tile's accumulator
-// alone is 256 of the 512 tensor-memory columns, so two tiles do not fit.  What the second tile gave
-// there -- its MMAs run while the first tile's softmax does -- comes here from two score buffers:
+// alone is 256 of the 512 tensor-memory columns, and at 192 / 128 the queries of two tiles would not
+// fit beside the accumulators.  What the second tile gave there -- its MMAs run while the first
+// tile's softmax does -- comes here from two score buffers:
 //   * A CTA owns 128 score rows (128 / n_rep consecutive queries x the n_rep heads of one KV head)
-//     and walks the keys 64 at a time (two 32-token chunks, one bulk copy of 18432 bytes).
-//   * Eight "dequantize" warps turn each raw block into binary16 tiles K^ [64 keys][256 dims] and
-//     V^ [256 dims][64 keys] in shared memory (two stages each), in the core-matrix order a K-major
+//     and walks the keys 64 at a time (two 32-token chunks, one bulk copy).
+//   * Eight "dequantize" warps turn each raw block into binary16 tiles K^ [64 keys][d_qk] and
+//     V^ [d_v][64 keys] in shared memory (two stages each), in the core-matrix order a K-major
 //     tcgen05 operand wants: x^ = c * s + b in one binary16 fma per pair of codes, each value rounded
 //     once to 11 significant bits.  A packed word becomes one 16-byte row of a core matrix; the order
 //     of the eight elements inside a row (0,4,1,5,2,6,3,7) is absorbed by storing the queries, and
 //     the key rows, in the same order.
-//   * One thread issues the MMAs: S_b = Q K^T (M 128, N 64, K 256: 16 instructions) into score buffer
-//     b = block % 2, with Q resident in tensor memory as packed binary16 (each bf16 row scaled by a
-//     power of two, so nothing is rounded), and O += P_b V^ (M 128, N 256, K 64: 4 instructions) with
-//     P_b read from tensor memory too, where it overlays S_b.  The scores of block j + 1 are issued
-//     before the probabilities of block j exist, so the tensor pipe works through the softmax.
-//     Tensor memory: O 256 columns, S 2 x 64, Q 128.
-//   * Eight softmax warps, two threads per score row (each takes 32 of the 64 scores and 128 of the
-//     256 accumulator columns): mask, online softmax with a lazily updated reference maximum, P_b as
+//   * One thread issues the MMAs: S_b = Q K^T (M 128, N 64, K d_qk: d_qk / 16 instructions) into score
+//     buffer b = block % 2, with Q resident in tensor memory as packed binary16 (each bf16 row scaled
+//     by a power of two, so nothing is rounded), and O += P_b V^ (M 128, N d_v, K 64: 4 instructions)
+//     with P_b read from tensor memory too, where it overlays S_b.  The scores of block j + 1 are
+//     issued before the probabilities of block j exist, so the tensor pipe works through the softmax.
+//     Tensor memory: O d_v columns, S 2 x 64, Q d_qk / 2.
+//   * Eight softmax warps, two threads per score row (each takes 32 of the 64 scores and half of the
+//     accumulator columns): mask, online softmax with a lazily updated reference maximum, P_b as
 //     packed binary16.
 //   * One warp streams the raw blocks through a three-slot ring with bulk asynchronous copies.
 // All hand-offs are mbarriers; every wait is bounded and a wait that runs out raises
@@ -35,17 +37,22 @@ namespace {
 
 using namespace tc;
 
-constexpr int kD = 256;
 constexpr int kSoftmaxWarps = 8, kDequantWarps = 8;
 constexpr int kMmaWarp = kSoftmaxWarps + kDequantWarps, kLoadWarp = kMmaWarp + 1;
 constexpr int kThreads = (kLoadWarp + 1) * 32;           // 576
 constexpr int kStages = 2;                               // K^ tiles, and V^ tiles, in flight
 constexpr int kRawSlots = 3;                             // raw 64-key blocks in flight
-constexpr int kChunkBytes = 9216;                        // d = 256: [Kc 4096 | Ksb 512 | Vc 4096 | Vsb 512]
-constexpr int kOffKsb = 4096, kOffVc = 4608, kOffVsb = 8704;
-constexpr int kRawBytes = 2 * kChunkBytes;
-constexpr int kTileBytes = 64 * kD * 2;                  // one binary16 tile: 32768
-constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;  // tensor-memory columns (256, 2 x 64, 128)
+constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;  // tensor-memory columns (d_v <= 256, 2 x 64, d_qk / 2 <= 128)
+// G, Gv: groups of 64 along the key and value head dims
+template <int G, int Gv>
+struct Shape {
+  static constexpr int D = 64 * G, Dv = 64 * Gv;
+  static constexpr int kOffKsb = 16 * D, kOffVc = kOffKsb + 128 * G, kOffVsb = kOffVc + 16 * Dv;
+  static constexpr int kChunkBytes = kOffVsb + 128 * Gv; // [Kc | Ksb | Vc | Vsb]: 9216 at 256 / 256, 5760 at 192 / 128
+  static constexpr int kRawBytes = 2 * kChunkBytes;
+  static constexpr int kTileK = 64 * D * 2, kTileV = Dv * 64 * 2;   // binary16 tiles
+  static constexpr int kSboK = (D / 8) * 128;            // bytes between 8-key groups of K^
+};
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLazy = 8.f;                             // rescale when the row maximum grew by more than this (log2)
 
@@ -57,7 +64,7 @@ struct UmmaParams {
   const int32_t* kv_lens;
   const int32_t* q_offs;
   int window;
-  const uint16_t* q;          // bf16 [total_q][Hq][256]
+  const uint16_t* q;          // bf16 [total_q][Hq][d_qk]
   float scale_log2;
   void* out;
   int out_dtype;
@@ -65,10 +72,12 @@ struct UmmaParams {
   int32_t* flags;
 };
 
+template <int G, int Gv>
 struct UmmaSmem {
-  alignas(128) uint8_t khat[kStages][kTileBytes];        // [key 64][dim 256]: (n%8)*16 + (n/8)*4096 + (k/8)*128
-  alignas(128) uint8_t vhat[kStages][kTileBytes];        // [dim 256][key 64]: (n%8)*16 + (n/8)*1024 + (k/8)*128
-  alignas(128) uint8_t raw[kRawSlots][kRawBytes];
+  using Sh = Shape<G, Gv>;
+  alignas(128) uint8_t khat[kStages][Sh::kTileK];        // [key 64][dim d_qk]: (n%8)*16 + (n/8)*kSboK + (k/8)*128
+  alignas(128) uint8_t vhat[kStages][Sh::kTileV];        // [dim d_v][key 64]: (n%8)*16 + (n/8)*1024 + (k/8)*128
+  alignas(128) uint8_t raw[kRawSlots][Sh::kRawBytes];
   alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots];
   uint64_t k_full[kStages], v_full[kStages], k_free[kStages], v_free[kStages];
   uint64_t s_full[2], p_full[2], o_done, q_ready, drain;
@@ -110,9 +119,13 @@ __device__ inline uint32_t f32x2_to_h2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-__global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __grid_constant__ UmmaParams P) {
+template <int G, int Gv>
+__global__ void __launch_bounds__(kThreads, 1) prefill_umma_1tile_kernel(const __grid_constant__ UmmaParams P) {
+  using Sh = Shape<G, Gv>;
+  constexpr int kD = Sh::D, kDv = Sh::Dv, kChunkBytes = Sh::kChunkBytes, kRawBytes = Sh::kRawBytes;
+  constexpr int kOffKsb = Sh::kOffKsb, kOffVc = Sh::kOffVc, kOffVsb = Sh::kOffVsb;
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  UmmaSmem& sm = *reinterpret_cast<UmmaSmem*>(smem_raw);
+  UmmaSmem<G, Gv>& sm = *reinterpret_cast<UmmaSmem<G, Gv>*>(smem_raw);
 
   const Layout& y = P.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -192,18 +205,25 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
     }
   } else if (warp >= kSoftmaxWarps && warp < kMmaWarp) {
     // =============================== dequantize warps ==========================================
+    // 256 threads.  At 256 / 256 a thread takes one of the two 16-byte key pieces of a token row (kj) and one value
+    // piece, in both chunks of the block; at 192 / 128 a token row is a 16-byte and an 8-byte key piece and there are
+    // half as many value pieces, and a thread works on one chunk of the block (c1).
     const int x = threadIdx.x - kSoftmaxWarps * 32;      // 0..255
-    // K: one 16-byte piece of token tau = 4 kg + ki per chunk: words 16 kj + kt + 4 m, m = 0..3 (groups 2 kj, 2 kj + 1).
-    // The eight lanes of a shared-memory phase read eight different 16-byte columns and write eight different rows.
-    const int ki = x & 3, kg = 2 * ((x >> 3) & 3) + ((x >> 2) & 1), kt = (ki + (x >> 5)) & 3, kj = x >> 7;
+    const int x7 = x & 127, c1 = x >> 7;
+    // K: token tau = 4 kg + ki of a chunk, piece kt of its lane group.  The eight lanes of a shared-memory phase read
+    // eight different 16-byte columns and write eight different rows.
+    const int ki = x & 3, kg = 2 * ((x >> 3) & 3) + ((x >> 2) & 1), kt = (ki + (x7 >> 5)) & 3, kj = G == 4 ? c1 : 0;
     const int ktau = 4 * kg + ki;
-    const int k_read = ki * 1024 + kj * 512 + kg * 64 + kt * 16;
-    const int k_sb = kOffKsb + ((((ktau & 3) * 4 + (ktau >> 3)) * 2 + ((ktau >> 2) & 1)) * 4 + 2 * kj) * 4;
+    const int k_read = ki * (256 * G) + kj * 512 + kg * 64 + kt * 16;       // 16-byte piece: words 16 kj + kt + 4 m, m = 0..3
+    const int k_read2 = ki * (256 * G) + 512 + kg * 32 + kt * 8;            // G = 3: the 8-byte piece, words 16 + kt, 20 + kt
+    const int k_tok = ((ktau & 3) * 4 + (ktau >> 3)) * 2 + ((ktau >> 2) & 1);   // the token's place among the (scale, bias) rows
+    const int k_sb = kOffKsb + (k_tok * G + 2 * kj) * 4;
     const int k_row = 8 * (ktau >> 3) + slot_of(ktau & 7);       // row of the token inside its chunk's 32 rows
     // V: one 16-byte piece (dims 32 vq + 8 k + vr, k = 0..3) of token octet vo per chunk.
-    const int vr = x & 7, vq = ((x >> 3) & 3) + 4 * (x >> 7), vo = ((vr >> 1) + (x >> 5)) & 3;
+    const int vr = x & 7, vq = ((x >> 3) & 3) + (Gv == 4 ? 4 * c1 : 0), vo = ((vr >> 1) + (x7 >> 5)) & 3;
     const int v_read = kOffVc + ((vq * 8 + vr) * 4 + vo) * 16;
-    const int v_sb = kOffVsb + vo * 32 + (vq >> 1) * 4;          // + i * 128 + e * 16: token 8 vo + 4 e + i, group vq / 2
+    const int v_sb = kOffVsb + (vo * 2 * Gv + (vq >> 1)) * 4;    // + (i * 8 + e) * Gv * 4: token 8 vo + 4 e + i, group vq / 2
+    constexpr int kChunksPerThread = G == 4 ? 2 : 1;
     for (int j = 0; j < n_iter; ++j) {
       const int s = j % kStages, r = j % kRawSlots;
       if (j >= kStages && !mbar_wait(&sm.k_free[s], (uint32_t)(j / kStages - 1), abort_flag)) break;
@@ -211,33 +231,45 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
       const bool bad = sm.bad[r] != 0;
       const int pos_base = (it0 + j) * 64;
 #pragma unroll
-      for (int ci = 0; ci < 2; ++ci) {
+      for (int cc = 0; cc < kChunksPerThread; ++cc) {
+        const int ci = G == 4 ? cc : c1;
         const uint8_t* chunk = sm.raw[r] + ci * kChunkBytes;
-        const uint4 kw = *reinterpret_cast<const uint4*>(chunk + k_read);
-        uint2 sb = *reinterpret_cast<const uint2*>(chunk + k_sb);          // (scale, bias) of groups 2 kj and 2 kj + 1
-        if (bad || pos_base + ci * 32 + ktau >= kv_len) sb = make_uint2(0u, 0u);   // stale bytes past the end
-        const uint32_t s0 = __byte_perm(sb.x, sb.x, 0x1010), b0 = __byte_perm(sb.x, sb.x, 0x3232);
-        const uint32_t s1 = __byte_perm(sb.y, sb.y, 0x1010), b1 = __byte_perm(sb.y, sb.y, 0x3232);
+        const bool dead = bad || pos_base + ci * 32 + ktau >= kv_len;      // stale bytes past the end
         const int n = ci * 32 + k_row;
-        uint8_t* dst = sm.khat[s] + (n & 7) * 16 + (n >> 3) * 4096 + (16 * kj + kt) * 128;
+        uint8_t* dst = sm.khat[s] + (n & 7) * 16 + (n >> 3) * Sh::kSboK + (16 * kj + kt) * 128;
+        const uint4 kw = *reinterpret_cast<const uint4*>(chunk + k_read);
+        uint32_t e0 = *reinterpret_cast<const uint32_t*>(chunk + k_sb);       // (scale, bias) of groups 2 kj and 2 kj + 1
+        uint32_t e1 = *reinterpret_cast<const uint32_t*>(chunk + k_sb + 4);
+        if (dead) { e0 = 0u; e1 = 0u; }
+        const uint32_t s0 = __byte_perm(e0, e0, 0x1010), b0 = __byte_perm(e0, e0, 0x3232);
+        const uint32_t s1 = __byte_perm(e1, e1, 0x1010), b1 = __byte_perm(e1, e1, 0x3232);
         *reinterpret_cast<uint4*>(dst + 0 * 512) = dequant8(kw.x, s0, b0, s0, b0, s0, b0, s0, b0);
         *reinterpret_cast<uint4*>(dst + 1 * 512) = dequant8(kw.y, s0, b0, s0, b0, s0, b0, s0, b0);
         *reinterpret_cast<uint4*>(dst + 2 * 512) = dequant8(kw.z, s1, b1, s1, b1, s1, b1, s1, b1);
         *reinterpret_cast<uint4*>(dst + 3 * 512) = dequant8(kw.w, s1, b1, s1, b1, s1, b1, s1, b1);
+        if (G == 3) {
+          const uint2 kw2 = *reinterpret_cast<const uint2*>(chunk + k_read2);
+          uint32_t e2 = *reinterpret_cast<const uint32_t*>(chunk + k_sb + 8);  // group 2
+          if (dead) e2 = 0u;
+          const uint32_t s2 = __byte_perm(e2, e2, 0x1010), b2 = __byte_perm(e2, e2, 0x3232);
+          *reinterpret_cast<uint4*>(dst + 4 * 512) = dequant8(kw2.x, s2, b2, s2, b2, s2, b2, s2, b2);
+          *reinterpret_cast<uint4*>(dst + 5 * 512) = dequant8(kw2.y, s2, b2, s2, b2, s2, b2, s2, b2);
+        }
       }
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.k_full[s]);
       if (j >= kStages && !mbar_wait(&sm.v_free[s], (uint32_t)(j / kStages - 1), abort_flag)) break;
 #pragma unroll
-      for (int ci = 0; ci < 2; ++ci) {
+      for (int cc = 0; cc < kChunksPerThread; ++cc) {
+        const int ci = G == 4 ? cc : c1;
         const uint8_t* chunk = sm.raw[r] + ci * kChunkBytes;
         const uint4 vw = *reinterpret_cast<const uint4*>(chunk + v_read);
         uint32_t sp[4], bp[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          uint32_t e0 = *reinterpret_cast<const uint32_t*>(chunk + v_sb + i * 128);
-          uint32_t e1 = *reinterpret_cast<const uint32_t*>(chunk + v_sb + i * 128 + 16);
+          uint32_t e0 = *reinterpret_cast<const uint32_t*>(chunk + v_sb + i * 32 * Gv);
+          uint32_t e1 = *reinterpret_cast<const uint32_t*>(chunk + v_sb + i * 32 * Gv + 4 * Gv);
           const int pos = pos_base + ci * 32 + 8 * vo + i;
           if (bad || pos >= kv_len) e0 = 0u;
           if (bad || pos + 4 >= kv_len) e1 = 0u;
@@ -259,12 +291,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
     // The whole warp runs this code, so that operands are computed once for the warp, and one elected
     // lane (always the same) issues the MMAs and the commits.
     if (n_iter > 0) {
-      constexpr uint32_t kIdescS = idesc_f16(128, 64), kIdescO = idesc_f16(128, 256);
+      constexpr uint32_t kIdescS = idesc_f16(128, 64), kIdescO = idesc_f16(128, kDv);
       auto issue_qk = [&](int b, int s) {                // S_b = Q K^T; afterwards the K^ stage is free
         const uint32_t kb = smem_u32(sm.khat[s]);
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k) {
-          const uint64_t bd = smem_desc(kb + 256 * k, 128, 4096);
+          const uint64_t bd = smem_desc(kb + 256 * k, 128, Sh::kSboK);
           if (elect_one()) mma_f16_ts(tb + kColS + 64 * b, tb + kColQ + 8 * k, bd, kIdescS, k > 0);
         }
         if (elect_one()) { commit(&sm.s_full[b]); commit(&sm.k_free[s]); }
@@ -323,12 +355,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
     {
       // ---- stage this thread's half of the query row: bf16 -> binary16 times a power of two, element order
       //      (0,4,1,5,2,6,3,7) inside every eight ----
-      const uint16_t* qrow = P.q + ((size_t)(q0 + (valid ? i : 0)) * y.Hq + (size_t)hk * n_rep + h) * kD + 128 * half;
-      uint32_t qa[64];
+      constexpr int kQWords = kD / 4;                    // packed binary16 words of this thread's half row: 64 or 48
+      const uint16_t* qrow = P.q + ((size_t)(q0 + (valid ? i : 0)) * y.Hq + (size_t)hk * n_rep + h) * kD + (kD / 2) * half;
+      uint32_t qa[kQWords];
       float mx = 0.f;
       if (valid) {
 #pragma unroll
-        for (int w = 0; w < 16; ++w) {
+        for (int w = 0; w < kQWords / 4; ++w) {
           const uint4 v = *reinterpret_cast<const uint4*>(qrow + 8 * w);
           qa[4 * w] = v.x; qa[4 * w + 1] = v.y; qa[4 * w + 2] = v.z; qa[4 * w + 3] = v.w;
           mx = fmaxf(mx, fmaxf(fmaxf(fabsf(__uint_as_float(v.x << 16)), fabsf(__uint_as_float(v.x & 0xffff0000u))),
@@ -338,7 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
         }
       } else {
 #pragma unroll
-        for (int w = 0; w < 64; ++w) qa[w] = 0u;
+        for (int w = 0; w < kQWords; ++w) qa[w] = 0u;
       }
       sm.xchg[1][half][row] = mx;                        // slot 1: block 0 of the loop below writes slot 0
       tile_barrier();
@@ -349,7 +382,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
       const float sf = __uint_as_float((uint32_t)(127 + 8 - ex) << 23);      // 256 <= max |q| * sf < 512
       kappa = P.scale_log2 * __uint_as_float((uint32_t)(127 - 8 + ex) << 23);
 #pragma unroll
-      for (int w = 0; w < 16; ++w) {
+      for (int w = 0; w < kQWords / 4; ++w) {
         // elements 8w..8w+7 arrive as bf16 pairs (0,1) (2,3) (4,5) (6,7); columns hold (0,4) (1,5) (2,6) (3,7)
         const uint32_t u01 = qa[4 * w], u23 = qa[4 * w + 1], u45 = qa[4 * w + 2], u67 = qa[4 * w + 3];
         const float x0 = __uint_as_float(u01 << 16) * sf, x1 = __uint_as_float(u01 & 0xffff0000u) * sf;
@@ -359,8 +392,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
         qa[4 * w] = f32x2_to_h2(x0, x4); qa[4 * w + 1] = f32x2_to_h2(x1, x5);
         qa[4 * w + 2] = f32x2_to_h2(x2, x6); qa[4 * w + 3] = f32x2_to_h2(x3, x7);
       }
-      tmem_st32(lane_addr + kColQ + 64 * half, qa);
-      tmem_st32(lane_addr + kColQ + 64 * half + 32, qa + 32);
+      // 32-column stores start at multiples of 32 columns, 16-column stores at multiples of 16
+      if (kQWords == 64) {
+        tmem_st32(lane_addr + kColQ + 64 * half, qa);
+        tmem_st32(lane_addr + kColQ + 64 * half + 32, qa + 32);
+      } else if (half == 0) {
+        tmem_st32(lane_addr + kColQ, qa);
+        tmem_st16(lane_addr + kColQ + 32, qa + 32);
+      } else {
+        tmem_st16(lane_addr + kColQ + 48, qa);
+        tmem_st32(lane_addr + kColQ + 64, qa + 16);
+      }
       wait_st();
       fence_before_sync();
       mbar_arrive(&sm.q_ready);
@@ -421,13 +463,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
           fence_after_sync();
           const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;           // m_ref = -inf: 0
 #pragma unroll 1
-          for (int part = 0; part < 4; ++part) {
+          for (int part = 0; part < kDv / 64; ++part) {
             uint32_t orow[32];
-            tmem_ld32(lane_addr + kColO + 128 * half + 32 * part, orow);
+            tmem_ld32(lane_addr + kColO + (kDv / 2) * half + 32 * part, orow);
             wait_ld();
 #pragma unroll
             for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * f);
-            tmem_st32(lane_addr + kColO + 128 * half + 32 * part, orow);
+            tmem_st32(lane_addr + kColO + (kDv / 2) * half + 32 * part, orow);
           }
           if (grow) l *= f;
         }
@@ -452,12 +494,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
     if (ok) fence_after_sync();
     const bool zero = !ok || n_iter == 0 || sm.poisoned != 0 || l <= 0.f;
     const float inv = zero ? 0.f : 1.f / l;
-    const size_t orow_index = ((size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h) * kD + 128 * half;
+    const size_t orow_index = ((size_t)(q0 + i) * y.Hq + (size_t)hk * n_rep + h) * kDv + (kDv / 2) * half;
 #pragma unroll 1
-    for (int part = 0; part < 4; ++part) {
+    for (int part = 0; part < kDv / 64; ++part) {
       uint32_t orow[32];
       if (ok && n_iter > 0) {
-        tmem_ld32(lane_addr + kColO + 128 * half + 32 * part, orow);
+        tmem_ld32(lane_addr + kColO + (kDv / 2) * half + 32 * part, orow);
         wait_ld();
       }
       if (i >= q_len) continue;
@@ -508,32 +550,27 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma256_kernel(const __gr
 
 }  // namespace
 
-bool prefill_umma256_supported(const Layout& y) {
-  return !y.alias && y.D == kD && y.Dv == kD && (y.n_rep == 1 || y.n_rep == 2 || y.n_rep == 4);
+bool prefill_umma_1tile_supported(const Layout& y) {
+  const bool shape = (y.D == 256 && y.Dv == 256) || (y.D == 192 && y.Dv == 128);
+  return !y.alias && shape && (y.n_rep == 1 || y.n_rep == 2 || y.n_rep == 4);
 }
 
-cudaError_t launch_prefill_umma256(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
-                                   const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window,
-                                   const void* q, float scale, void* out, int out_dtype, float* lse, int32_t* flags,
-                                   cudaStream_t st) {
-  if (b.n_agents <= 0 || max_q_len <= 0) return cudaSuccess;
-  UmmaParams P;
-  P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
-  P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.q_offs = q_offs; P.window = window;
-  P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
+namespace {
+template <int G, int Gv>
+cudaError_t launch_shape(const UmmaParams& P, int max_q_len, cudaStream_t st) {
   static bool configured[64] = {};
-  const size_t smem = sizeof(UmmaSmem);
+  const size_t smem = sizeof(UmmaSmem<G, Gv>);
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(prefill_umma256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(prefill_umma_1tile_kernel<G, Gv>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  const int cta_q = 128 / y.n_rep;
+  const int cta_q = 128 / P.y.n_rep;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((max_q_len + cta_q - 1) / cta_q, y.Hkv, b.n_agents);
+  cfg.gridDim = dim3((max_q_len + cta_q - 1) / cta_q, P.y.Hkv, P.n_agents);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
@@ -542,7 +579,20 @@ cudaError_t launch_prefill_umma256(const Layout& y, const void* pool, int n_bloc
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, prefill_umma256_kernel, P);
+  return cudaLaunchKernelEx(&cfg, prefill_umma_1tile_kernel<G, Gv>, P);
+}
+}  // namespace
+
+cudaError_t launch_prefill_umma_1tile(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+                                      const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window,
+                                      const void* q, float scale, void* out, int out_dtype, float* lse, int32_t* flags,
+                                      cudaStream_t st) {
+  if (b.n_agents <= 0 || max_q_len <= 0) return cudaSuccess;
+  UmmaParams P;
+  P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
+  P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.q_offs = q_offs; P.window = window;
+  P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
+  return y.D == 256 ? launch_shape<4, 4>(P, max_q_len, st) : launch_shape<3, 2>(P, max_q_len, st);
 }
 
 }  // namespace q4kv

@@ -234,9 +234,9 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale))
     e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                             out_dtype, lse, status_flags, (cudaStream_t)stream);
-  else if (prefill_umma256_supported(y) && tiles_allowed(spec, softmax_scale))
-    e = launch_prefill_umma256(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale,
-                               out, out_dtype, lse, status_flags, (cudaStream_t)stream);
+  else if (prefill_umma_1tile_supported(y) && tiles_allowed(spec, softmax_scale))
+    e = launch_prefill_umma_1tile(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale,
+                                  out, out_dtype, lse, status_flags, (cudaStream_t)stream);
   else if (prefill_mma_supported(y))
     e = launch_prefill_mma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                            out_dtype, lse, status_flags, (cudaStream_t)stream);

@@ -155,9 +155,10 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
                                 const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window, const void* q,
                                 float scale, void* out, int out_dtype, float* lse, int32_t* flags, cudaStream_t st);
 
-// tcgen05 prefill path for d_qk = d_v = 256 (1, 2 or 4 query heads per KV head): one 128-row tile per CTA, two score buffers
-bool prefill_umma256_supported(const Layout& y);
-cudaError_t launch_prefill_umma256(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
+// tcgen05 prefill path for d_qk = d_v = 256 and for d_qk 192 / d_v 128 (1, 2 or 4 query heads per KV head): one 128-row
+// tile per CTA, two score buffers
+bool prefill_umma_1tile_supported(const Layout& y);
+cudaError_t launch_prefill_umma_1tile(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
                                    const int32_t* kv_lens, const int32_t* q_offs, int max_q_len, int window,
                                    const void* q, float scale, void* out, int out_dtype, float* lse, int32_t* flags,
                                    cudaStream_t st);

@@ -705,6 +705,8 @@ def test_layer_batched_decode_equals_the_oracle_layer_by_layer(H, spec_args, len
     ("gqa128", [512, 200], 130, 0),
     ("gqa256", [256, 10], 70, 128),
     ("mla", [200], 33, 0),
+    ("asym", [300, 70], 40, 0),
+    ("asym", [300, 70], 40, 50),
 ])
 def test_prefill_matches_oracle_and_chunking_is_invisible(H, name, prefix, chunk, window):
     lens = [n + chunk for n in prefix]
@@ -844,6 +846,10 @@ class QuietStartPair(Pair):
     ((1, 8, 2, 256, 256, False), [1500, 64], [129, 64], 0, 2.0),         # d = 256, the row maximum jumps by more than 2^8
     ((1, 4, 4, 256, 256, False), [0], [257], 0, 1.0),                    # d = 256, no prefix, one head per KV head
     ((1, 2, 1, 256, 256, False), [6000, 1], [300, 1], 0, 1.0),           # d = 256, ~100 blocks through the two-stage rings; one key
+    ((1, 4, 4, 192, 128, False), [900, 5], [140, 70], 0, 1.0),           # d_qk 192 / d_v 128 (the same one-tile kernel), one head per KV head
+    ((1, 8, 2, 192, 128, False), [3000], [200], 700, 1.0),               # 192 / 128, four heads per KV head, a window
+    ((1, 4, 2, 192, 128, False), [1500, 64], [129, 64], 0, 2.0),         # 192 / 128, the row maximum jumps by more than 2^8
+    ((1, 16, 16, 192, 128, False), [0, 33, 5000], [257, 31, 100], 0, 1.0),   # 192 / 128, sixteen KV heads, no prefix, a long prefix
 ])
 def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
     """The tensor-memory prefill kernel: tile shapes for 1, 2 and 4 heads per KV head, key ranges that start
@@ -867,13 +873,13 @@ def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
 
 @pytest.mark.parametrize("gain,outlier_frac", [(8.0, 0.0), (1.0, 0.01)])
 @pytest.mark.parametrize("prefix,chunks", [([0, 40], [70, 30]), ([300], [64])])
-@pytest.mark.parametrize("d", [128, 256])
+@pytest.mark.parametrize("d", [128, 256, 192])
 def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks, d):
     """Rows that attend 1 to 64 keys of a cache with a gain of 8, or with 1 % of the channels carrying 8x the
     values, return value rows almost verbatim, so a single binary16 rounding of a dequantized value (half an ulp of
     2^-8 for magnitudes in [8, 16)) is visible.  With exact_products the usual bound holds; without it the
     binary16-tile kernel stays inside the bound the header states for it."""
-    spec_args = (1, 8, 2, d, d, False)
+    spec_args = (1, 8, 2, d, 128 if d == 192 else d, False)
     lens = [p0 + c for p0, c in zip(prefix, chunks)]
     q_offs = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
     scale = 1.0 / math.sqrt(d)
@@ -893,11 +899,11 @@ def test_prefill_on_large_magnitude_caches(H, gain, outlier_frac, prefix, chunks
         assert p.dc.read_flags() == 0
 
 
-@pytest.mark.parametrize("d", [128, 256])
+@pytest.mark.parametrize("d", [128, 256, 192])
 def test_prefill_bad_block_and_bad_length(H, d):
     from paper_2603_04428_b200 import binding as B
     lens = [600, 200]
-    p = Pair(H, (1, 8, 2, d, d, False), lens, seed=53).fill()
+    p = Pair(H, (1, 8, 2, d, 128 if d == 192 else d, False), lens, seed=53).fill()
     q_offs = [0, 100, 180]
     q = p.q(7, 180)
     good, _ = p.dc.prefill(0, lens, q_offs, 0, q, 0.1)
@@ -921,7 +927,8 @@ def test_tensor_memory_prefill_and_latent_decode_repeat_bit_for_bit(H):
     latent-cache decode on tiles and on codes) have a fixed order of arithmetic: sixty launches in a row on the same
     inputs return the same bits, which a missed hand-off (a tile read before it is complete) would not."""
     for spec_args, prefix, chunk in (((1, 8, 2, 128, 128, False), [1800, 300], 200),
-                                     ((1, 8, 4, 256, 256, False), [1800, 300], 200)):
+                                     ((1, 8, 4, 256, 256, False), [1800, 300], 200),
+                                     ((1, 8, 8, 192, 128, False), [1800, 300], 200)):
         lens = [n + chunk for n in prefix]
         p = Pair(H, spec_args, lens, seed=91).fill()
         q_offs = [0, chunk, 2 * chunk]
