@@ -7,7 +7,7 @@ agent, then decode attention of one query per agent over the whole Q4 cache.  On
 layers.  The metric is the achieved HBM bandwidth over the algorithmic bytes of the step (each
 needed Q4 row read once + q + out + new rows); agent-steps/s rides along.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4|5|6] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4|5|6|7] [--impl reference]
 
 N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no collective.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
@@ -383,6 +383,7 @@ NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23_991_723, "gemma3_12b_ragged_decode"
                      "dsv2lite_mla_decode": 21_440_640, "dsv2lite_mla_decode_exact_products": 21_446_656,
                      "llama31_8b_chunked_prefill": 240_450_688,
                      "dsv2lite_perhead_mla_decode": 191_148_800, "gemma3_12b_shaped_global_prefill": 151_449_472,
+                     "dsv2lite_perhead_mla_prefill": 146_757_504,
                      "pack": 254_257_000, "unpack": 251_510_000, "append_8x1024": 33_606_912}
 
 
@@ -655,7 +656,7 @@ def main():
                              "append_avg_us": ri["app_s"] * 1e6, "roofline": roof_i, "config": config_of(wi, ri),
                              "gpu_launches_per_step": dw_launches(wi, ai.two_calls), "clocks": ri["clocks"]}
 
-        for idx in (2, 3, 4, 5, 6):
+        for idx in (2, 3, 4, 5, 6, 7):
             entry(synth.workload(idx), args)
         # the MLA-latent decode again with q4kv_spec.exact_products set: the kernel that multiplies the codes (also the
         # route of bfloat16 caches and sharp softmax scales)

@@ -116,7 +116,7 @@ enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
  *     at most 2e-5 * M + 1e-5, i.e. within 2e-3 for any cache with M <= 64.  (An absolute bound:
  *     the tensor-core kernels carry probability x scale in binary16, so contributions of groups
  *     whose scale is below 2^-24 vanish; only bfloat16 caches can hold such scales.)
- *   - Kernels that expand the cache into binary16 tiles (prefill with d_qk = d_v in {128, 256} and 1, 2 or 4
+ *   - Kernels that expand the cache into binary16 tiles (prefill with d_qk = d_v in {128, 256} or d_qk 192 / d_v 128 and 1, 2 or 4
  *     query heads per KV head; decode on the MLA-latent cache: V aliasing K, d_qk 576, d_v 512, one
  *     KV head, at most 16 query heads) round every dequantized value once to binary16, a relative
  *     error of 2^-11 at most, and the probabilities likewise.  They are chosen only when

@@ -127,7 +127,7 @@ class Workload:
 def workload(index: int) -> Workload:
     """The five benchmark configurations, 0-based, and (index 5) the per-head MLA cache of Section 3.6 at the sizes of
     configuration 4: keys of 192 dims (3 groups), values of 128 (2 groups), 16 KV heads; (index 6) a chunked-prefill
-    phase at d = 256."""
+    phase at d = 256; (index 7) a chunked-prefill phase on the per-head MLA cache."""
     seed = BASE_SEED + index
     if index == 0:
         return Workload("tiny_gqa_decode", 1, 8, 2, 128, 128, False, [1000, 700], 1,
@@ -149,7 +149,11 @@ def workload(index: int) -> Workload:
         return Workload("dsv2lite_perhead_mla_decode", 27, 16, 16, 192, 128, False, [16384] * 4, 1,
                         softmax_scale=1.0 / math.sqrt(192), seed=seed)
     if index == 6:
-        # a d = 256 phase (Gemma-3-12B's head shape, global layers): what the exact-product prefill kernel does there
+        # a d = 256 phase (Gemma-3-12B's head shape, global layers)
         return Workload("gemma3_12b_shaped_global_prefill", 8, 16, 8, 256, 256, False, [4096] * 8, 512,
                         softmax_scale=1.0 / math.sqrt(256), seed=seed, kind="prefill")
+    if index == 7:
+        # a phase on the per-head MLA cache (d_qk 192 / d_v 128, 16 KV heads, one query head each)
+        return Workload("dsv2lite_perhead_mla_prefill", 8, 16, 16, 192, 128, False, [4096] * 8, 512,
+                        softmax_scale=1.0 / math.sqrt(192), seed=seed, kind="prefill")
     raise IndexError(index)
