@@ -850,6 +850,9 @@ class QuietStartPair(Pair):
     ((1, 8, 2, 192, 128, False), [3000], [200], 700, 1.0),               # 192 / 128, four heads per KV head, a window
     ((1, 4, 2, 192, 128, False), [1500, 64], [129, 64], 0, 2.0),         # 192 / 128, the row maximum jumps by more than 2^8
     ((1, 16, 16, 192, 128, False), [0, 33, 5000], [257, 31, 100], 0, 1.0),   # 192 / 128, sixteen KV heads, no prefix, a long prefix
+    ((1, 2, 2, 256, 256, False), [30000], [64], 0, 1.0),                 # d = 256: 470 blocks, every ring wraps hundreds of times
+    ((1, 2, 2, 192, 128, False), [20000, 300], [100, 10], 0, 1.0),       # 192 / 128: 314 blocks
+    ((1, 4, 1, 128, 128, False), [30000], [64], 0, 1.0),                 # d = 128 (two tiles, one of them empty): 470 blocks
 ])
 def test_prefill_tcgen05_path(H, spec_args, prefix, chunks, window, scale_mul):
     """The tensor-memory prefill kernel: tile shapes for 1, 2 and 4 heads per KV head, key ranges that start
