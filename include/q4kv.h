@@ -101,7 +101,10 @@ enum {
 enum {
   Q4KV_FLAG_BAD_BLOCK = 1,   /* a block id outside [0, n_blocks)                                    */
   Q4KV_FLAG_BAD_LENGTH = 2,  /* a length or position negative or beyond max_blocks*256              */
-  Q4KV_FLAG_INTERNAL = 4     /* a bounded wait inside a kernel ran out (the output is not valid)    */
+  Q4KV_FLAG_INTERNAL = 4,    /* a bounded wait inside a kernel ran out (the output is not valid)    */
+  Q4KV_FLAG_SB_RANGE = 8     /* a bfloat16 scale or bias beyond binary16's largest number met a kernel that
+                                expands the cache into binary16 tiles: the call's output is not valid;
+                                set exact_products and call again                                    */
 };
 enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
 

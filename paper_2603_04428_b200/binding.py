@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libq4kv.so")
 
 OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA = 0, -1, -2, -3, -4
-FLAG_BAD_BLOCK, FLAG_BAD_LENGTH = 1, 2
+FLAG_BAD_BLOCK, FLAG_BAD_LENGTH, FLAG_INTERNAL, FLAG_SB_RANGE = 1, 2, 4, 8
 OUT_F32, OUT_BF16 = 0, 1
 
 EXPORTS = [

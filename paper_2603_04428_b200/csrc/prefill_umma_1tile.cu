@@ -78,7 +78,7 @@ struct UmmaSmem {
   alignas(128) uint8_t khat[kStages][Sh::kTileK];        // [key 64][dim d_qk]: (n%8)*16 + (n/8)*kSboK + (k/8)*128
   alignas(128) uint8_t vhat[kStages][Sh::kTileV];        // [dim d_v][key 64]: (n%8)*16 + (n/8)*1024 + (k/8)*128
   alignas(128) uint8_t raw[kRawSlots][Sh::kRawBytes];
-  alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots];
+  alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots], sb_done[kRawSlots];
   uint64_t k_full[kStages], v_full[kStages], k_free[kStages], v_free[kStages];
   uint64_t s_full[2], p_full[2], o_done, q_ready, drain;
   uint32_t tmem_base;
@@ -118,8 +118,15 @@ __device__ inline uint32_t f32x2_to_h2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
+// A bfloat16 (scale, bias) pair as a binary16 pair: exact while the magnitude is a binary16 normal number (bfloat16
+// has 8 significant bits), within 2^-25 below that; a magnitude beyond binary16's largest number is reported.
+__device__ inline uint32_t bf16_pair_to_h2(uint32_t u, bool& overflow) {
+  const uint32_t h = f32x2_to_h2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+  overflow |= (((h & 0x7C007C00u) + 0x04000400u) & 0x80008000u) != 0u;     // an exponent field of all ones
+  return h;
+}
 
-template <int G, int Gv>
+template <int G, int Gv, bool kBf>
 __global__ void __launch_bounds__(kThreads, 1) prefill_umma_1tile_kernel(const __grid_constant__ UmmaParams P) {
   using Sh = Shape<G, Gv>;
   constexpr int kD = Sh::D, kDv = Sh::Dv, kChunkBytes = Sh::kChunkBytes, kRawBytes = Sh::kRawBytes;
@@ -150,7 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_1tile_kernel(const _
 
   if (threadIdx.x == 0) {
     if (bad_len) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
-    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); mbar_init(&sm.raw_free[s], kDequantWarps); sm.bad[s] = 0; }
+    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); mbar_init(&sm.raw_free[s], kDequantWarps); mbar_init(&sm.sb_done[s], kDequantWarps); sm.bad[s] = 0; }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.k_full[s], kDequantWarps); mbar_init(&sm.v_full[s], kDequantWarps);
       mbar_init(&sm.k_free[s], 1); mbar_init(&sm.v_free[s], 1);
@@ -230,6 +237,26 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_1tile_kernel(const _
       if (!mbar_wait(&sm.raw_full[r], (uint32_t)(j / kRawSlots), abort_flag)) break;
       const bool bad = sm.bad[r] != 0;
       const int pos_base = (it0 + j) * 64;
+      if (kBf) {
+        // bfloat16 scales and biases become binary16 in place, once per block (the tiles are binary16); only the
+        // tokens below the agent's length count for the range report (bytes past the end are whatever was there)
+        constexpr int kSbWords = 32 * (G + Gv);          // per chunk: Ksb then Vsb
+        bool overflow = false;
+        for (int w = x; w < 2 * kSbWords; w += kDequantWarps * 32) {
+          const int ci = w / kSbWords, o = w - ci * kSbWords;
+          const bool is_k = o < 32 * G;
+          const int row = is_k ? o / G : (o - 32 * G) / Gv;               // (i * 4 + tid) * 2 + e: token 8 tid + 4 e + i
+          const int tau = 8 * ((row >> 1) & 3) + 4 * (row & 1) + (row >> 3);
+          uint32_t* at = reinterpret_cast<uint32_t*>(sm.raw[r] + ci * kChunkBytes + (is_k ? kOffKsb + 4 * o : kOffVsb + 4 * (o - 32 * G)));
+          bool over = false;
+          *at = bf16_pair_to_h2(*at, over);
+          overflow |= over && pos_base + ci * 32 + tau < kv_len;
+        }
+        if (overflow && !bad) raise_flag(P.flags, Q4KV_FLAG_SB_RANGE);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.sb_done[r]);
+        if (!mbar_wait(&sm.sb_done[r], (uint32_t)(j / kRawSlots), abort_flag)) break;
+      }
 #pragma unroll
       for (int cc = 0; cc < kChunksPerThread; ++cc) {
         const int ci = G == 4 ? cc : c1;
@@ -556,7 +583,7 @@ bool prefill_umma_1tile_supported(const Layout& y) {
 }
 
 namespace {
-template <int G, int Gv>
+template <int G, int Gv, bool kBf>
 cudaError_t launch_shape(const UmmaParams& P, int max_q_len, cudaStream_t st) {
   static bool configured[64] = {};
   const size_t smem = sizeof(UmmaSmem<G, Gv>);
@@ -564,7 +591,7 @@ cudaError_t launch_shape(const UmmaParams& P, int max_q_len, cudaStream_t st) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(prefill_umma_1tile_kernel<G, Gv>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(prefill_umma_1tile_kernel<G, Gv, kBf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -579,7 +606,7 @@ cudaError_t launch_shape(const UmmaParams& P, int max_q_len, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, prefill_umma_1tile_kernel<G, Gv>, P);
+  return cudaLaunchKernelEx(&cfg, prefill_umma_1tile_kernel<G, Gv, kBf>, P);
 }
 }  // namespace
 
@@ -592,7 +619,8 @@ cudaError_t launch_prefill_umma_1tile(const Layout& y, const void* pool, int n_b
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.q_offs = q_offs; P.window = window;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
-  return y.D == 256 ? launch_shape<4, 4>(P, max_q_len, st) : launch_shape<3, 2>(P, max_q_len, st);
+  if (y.D == 256) return y.sb_bf16 ? launch_shape<4, 4, true>(P, max_q_len, st) : launch_shape<4, 4, false>(P, max_q_len, st);
+  return y.sb_bf16 ? launch_shape<3, 2, true>(P, max_q_len, st) : launch_shape<3, 2, false>(P, max_q_len, st);
 }
 
 }  // namespace q4kv

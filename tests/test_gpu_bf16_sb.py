@@ -147,6 +147,8 @@ def test_latent_cache_update_and_fetch_runs_on_the_codes(H):
     ("gqa128", [300, 0], 70, 100),
     ("gqa256", [256, 10], 70, 128),
     ("gqa256", [900, 0], 150, 0),
+    ("asym", [900, 0, 63], 150, 0),
+    ("asym", [300, 70], 40, 50),
 ])
 def test_prefill_matches_oracle(H, name, prefix, chunk, window):
     lens = [n + chunk for n in prefix]
@@ -228,3 +230,35 @@ def test_layer_batched_entry_and_static_entry(H):
                                        scale, out_s, B.OUT_F32, None, p.dc.flags)
         assert_attention_close(out_s.cpu().numpy(), ref, f"static entry, layer {l}")
     assert p.dc.read_flags() == 0
+
+
+TILE_KERNELS_TAKE_BF16 = ("gqa256", "asym")
+
+
+@pytest.mark.parametrize("name", TILE_KERNELS_TAKE_BF16)
+def test_a_scale_beyond_binary16_is_reported_by_the_tile_kernels(H, name):
+    """The library's own quantizer never produces a scale or bias beyond binary16's largest number (its inputs are
+    bounded by it, and the header asks the same of caches persisted elsewhere), but nothing stops a foreign file from
+    holding one.  Such a scale (here 2^20, planted in the oracle's pool and carried to the device through pack /
+    unpack) cannot enter a binary16 tile: the kernels that build such tiles raise Q4KV_FLAG_SB_RANGE rather than
+    return a wrong result silently; the same planted value past the agent's length is not looked at."""
+    from paper_2603_04428_b200 import binding as B
+    lens = [300, 64]
+    chunk = 40
+    p = Pair(H, SPECS[name], [n + chunk for n in lens], seed=150, sb_dtype=1).fill()
+    s = p.ospec
+    q_offs = [chunk * a for a in range(len(lens) + 1)]
+    q = p.q(7, chunk * len(lens))
+    scale = 1.0 / math.sqrt(s.d_qk)
+    good, _ = p.dc.prefill(0, p.lens, q_offs, 0, q, scale)
+    assert p.dc.read_flags() == 0
+    blk = int(p.tabs[0][1])                            # agent 0's second block holds tokens 256 .. 339
+    for tok, expect in ((340 - 256 + 3, False), (17, True)):     # past the length: ignored; inside: reported
+        p.opool.Vs[0, blk, 0, tok, 0] = 0x4980         # 2^20 as bfloat16
+        p.dc.unpack(0, 512, O.pack(p.opool, p.tabs[0], 512))
+        out, _ = p.dc.prefill(0, p.lens, q_offs, 0, q, scale)
+        flags = p.dc.read_flags()
+        assert bool(flags & B.FLAG_SB_RANGE) == expect and (flags & ~B.FLAG_SB_RANGE) == 0
+        if not expect:
+            assert torch.equal(out, good)
+        p.dc.flags.zero_()
