@@ -68,7 +68,7 @@ struct UmmaSmem {
   alignas(128) uint8_t khat[kStages][kTileBytes];        // [key 64][dim 128]: (n%8)*16 + (n/8)*2048 + (k/8)*128
   alignas(128) uint8_t vhat[kStages][kTileBytes];        // [dim 128][key 64]: (n%8)*16 + (n/8)*1024 + (k/8)*128
   alignas(128) uint8_t raw[kRawSlots][kRawBytes];
-  alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots];
+  alignas(8) uint64_t raw_full[kRawSlots], raw_free[kRawSlots], sb_done[kRawSlots];
   uint64_t k_full[kStages], v_full[kStages], kv_free[kStages];
   uint64_t s_full[2], p_full[2], o_done[2], q_ready, drain;
   uint32_t tmem_base;
@@ -108,7 +108,15 @@ __device__ inline uint32_t f32x2_to_h2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
+// A bfloat16 (scale, bias) pair as a binary16 pair: exact while the magnitude is a binary16 normal number (bfloat16
+// has 8 significant bits), within 2^-25 below that; a magnitude beyond binary16's largest number is reported.
+__device__ inline uint32_t bf16_pair_to_h2(uint32_t u, bool& overflow) {
+  const uint32_t h = f32x2_to_h2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+  overflow |= (((h & 0x7C007C00u) + 0x04000400u) & 0x80008000u) != 0u;     // an exponent field of all ones
+  return h;
+}
 
+template <bool kBf>
 __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_constant__ UmmaParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   UmmaSmem& sm = *reinterpret_cast<UmmaSmem*>(smem_raw);
@@ -136,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
 
   if (threadIdx.x == 0) {
     if (bad_len) raise_flag(P.flags, Q4KV_FLAG_BAD_LENGTH);
-    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); mbar_init(&sm.raw_free[s], kDequantWarps); sm.bad[s] = 0; }
+    for (int s = 0; s < kRawSlots; ++s) { mbar_init(&sm.raw_full[s], 1); mbar_init(&sm.raw_free[s], kDequantWarps); mbar_init(&sm.sb_done[s], kDequantWarps); sm.bad[s] = 0; }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.k_full[s], kDequantWarps); mbar_init(&sm.v_full[s], kDequantWarps); mbar_init(&sm.kv_free[s], 1);
     }
@@ -207,6 +215,24 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
       if (!mbar_wait(&sm.raw_full[r], (uint32_t)(j / kRawSlots), abort_flag)) break;
       const bool bad = sm.bad[r] != 0;
       const int pos_base = (it0 + j) * 64;
+      if (kBf) {
+        // bfloat16 scales and biases become binary16 in place, once per block (the tiles are binary16); only the
+        // tokens below the agent's length count for the range report (bytes past the end are whatever was there)
+        bool overflow = false;
+        for (int w = x; w < 256; w += kDequantWarps * 32) {              // per chunk: 64 words of Ksb, 64 of Vsb
+          const int ci = w >> 7, o = w & 127;
+          const int row = (o & 63) >> 1;                                 // (i * 4 + tid) * 2 + e: token 8 tid + 4 e + i
+          const int tau = 8 * ((row >> 1) & 3) + 4 * (row & 1) + (row >> 3);
+          uint32_t* at = reinterpret_cast<uint32_t*>(sm.raw[r] + ci * kChunkBytes + (o < 64 ? 2048 + 4 * o : 4352 + 4 * (o - 64)));
+          bool over = false;
+          *at = bf16_pair_to_h2(*at, over);
+          overflow |= over && pos_base + ci * 32 + tau < kv_len;
+        }
+        if (overflow && !bad) raise_flag(P.flags, Q4KV_FLAG_SB_RANGE);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.sb_done[r]);
+        if (!mbar_wait(&sm.sb_done[r], (uint32_t)(j / kRawSlots), abort_flag)) break;
+      }
 #pragma unroll
       for (int ci = 0; ci < 2; ++ci) {
         const uint8_t* chunk = sm.raw[r] + ci * kChunkBytes;
@@ -513,15 +539,17 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
   P.y = y; P.pool = (const uint8_t*)pool; P.n_blocks = n_blocks; P.layer = layer; P.n_agents = b.n_agents;
   P.max_blocks = b.max_blocks; P.tables = b.block_tables; P.kv_lens = kv_lens; P.q_offs = q_offs; P.window = window;
   P.q = (const uint16_t*)q; P.scale_log2 = scale * kLog2e; P.out = out; P.out_dtype = out_dtype; P.lse = lse; P.flags = flags;
-  static bool configured[64] = {};
+  static bool configured[64][2] = {};
   const size_t smem = sizeof(UmmaSmem);
+  const int bf = y.sb_bf16 ? 1 : 0;
+  void (*kernel)(const UmmaParams) = bf ? prefill_umma_kernel<true> : prefill_umma_kernel<false>;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
-    e = cudaFuncSetAttribute(prefill_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (dev < 0 || dev >= 64 || !configured[dev][bf]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev][bf] = true;
   }
   const int cta_q = 2 * (128 / y.n_rep);
   cudaLaunchConfig_t cfg = {};
@@ -534,7 +562,7 @@ cudaError_t launch_prefill_umma(const Layout& y, const void* pool, int n_blocks,
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, prefill_umma_kernel, P);
+  return cudaLaunchKernelEx(&cfg, kernel, P);
 }
 
 }  // namespace q4kv

@@ -231,7 +231,7 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
   cudaError_t e;
-  if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale))
+  if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale, true))
     e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                             out_dtype, lse, status_flags, (cudaStream_t)stream);
   else if (prefill_umma_1tile_supported(y) && tiles_allowed(spec, softmax_scale, true))

@@ -232,7 +232,7 @@ def test_layer_batched_entry_and_static_entry(H):
     assert p.dc.read_flags() == 0
 
 
-TILE_KERNELS_TAKE_BF16 = ("gqa256", "asym")
+TILE_KERNELS_TAKE_BF16 = ("gqa128", "gqa256", "asym")
 
 
 @pytest.mark.parametrize("name", TILE_KERNELS_TAKE_BF16)
