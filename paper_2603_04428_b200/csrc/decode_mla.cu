@@ -95,6 +95,13 @@ __device__ inline uint32_t f32x2_to_h2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
+// A bfloat16 (scale, bias) pair as a binary16 pair: exact while the magnitude is a binary16 normal number (bfloat16
+// has 8 significant bits), within 2^-25 below that; a magnitude beyond binary16's largest number is reported.
+__device__ inline uint32_t bf16_pair_to_h2(uint32_t u, bool& overflow) {
+  const uint32_t h = f32x2_to_h2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+  overflow |= (((h & 0x7C007C00u) + 0x04000400u) & 0x80008000u) != 0u;     // an exponent field of all ones
+  return h;
+}
 __device__ inline void compute_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }   // the eight compute warps
 // four 8x8 b16 matrices; lane l supplies the address of row l % 8 of matrix l / 8; register i <- matrix i,
 // thread (g, t) of the warp receiving the elements (row g, columns 2t, 2t+1)
@@ -113,6 +120,7 @@ __device__ inline void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+template <bool kBf>
 __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_constant__ MlaParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   MlaSmem& sm = *reinterpret_cast<MlaSmem*>(smem_raw);
@@ -199,7 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[e] = 0.f;
       }
-      const QuantOut qo = quantize_eight(x, false);             // eight lanes per group of 64; 72 words = 9 whole groups
+      const QuantOut qo = quantize_eight(x, kBf);             // eight lanes per group of 64; 72 words = 9 whole groups
       if (w < kD / 8) {
         sm.new_words[w] = qo.word;
         if ((w & 7) == 0) sm.new_sb[w >> 3] = *reinterpret_cast<const uint32_t*>(&qo.sb);
@@ -297,6 +305,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_mla_kernel(const __grid_co
         uint8_t* dst = const_cast<uint8_t*>(head_block(P.pool, y, P.layer, blk, 0)) + (size_t)(c & 7) * kChunkBytes + at;
         *reinterpret_cast<uint32_t*>(dst) = val;
       }
+      compute_barrier();
+    }
+    if (kBf) {
+      // bfloat16 scales and biases become binary16 in place, once per block (the tile is binary16); only the tokens
+      // below the agent's length count for the range report (bytes past the end are whatever was there)
+      bool overflow = false;
+      for (int w = tq; w < 2 * 288; w += kThreads) {     // per chunk: 32 tokens x 9 groups
+        const int cw = w >= 288 ? 1 : 0, o = w - 288 * cw;
+        const int row = o / 9;                           // (i * 4 + tid) * 2 + e: token 8 tid + 4 e + i
+        const int tok = 8 * ((row >> 1) & 3) + 4 * (row & 1) + (row >> 3);
+        uint32_t* at = reinterpret_cast<uint32_t*>(sm.raw[r] + cw * kChunkBytes + 9216 + 4 * o);
+        bool over = false;
+        *at = bf16_pair_to_h2(*at, over);
+        overflow |= over && (b0 + j) * 64 + cw * 32 + tok < n;
+      }
+      if (overflow && sm.bad[r] == 0) raise_flag(P.flags, Q4KV_FLAG_SB_RANGE);
       compute_barrier();
     }
     {
@@ -587,15 +611,17 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
   if (on_codes) {
     e = launch_mla_codes_kernel(P, st);
   } else {
-    static bool configured[64] = {};
+    static bool configured[64][2] = {};
     const size_t smem = sizeof(MlaSmem);
+    const int bf = y.sb_bf16 ? 1 : 0;
+    void (*kernel)(const MlaParams) = bf ? decode_mla_kernel<true> : decode_mla_kernel<false>;
     int dev = 0;
     e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-      e = cudaFuncSetAttribute(decode_mla_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (dev < 0 || dev >= 64 || !configured[dev][bf]) {
+      e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      if (dev >= 0 && dev < 64) configured[dev] = true;
+      if (dev >= 0 && dev < 64) configured[dev][bf] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.n_splits, b.n_agents);
@@ -604,7 +630,7 @@ cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, i
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, decode_mla_kernel, P);
+    e = cudaLaunchKernelEx(&cfg, kernel, P);
   }
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t mcfg = {};

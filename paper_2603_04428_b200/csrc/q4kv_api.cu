@@ -44,11 +44,11 @@ size_t workspace_need(const Layout& y, int n_agents, int max_kv_len, int total_q
 
 // The kernels that expand the cache into binary16 tiles round each dequantized element once; they are taken only when
 // the spec allows it and the softmax scale is at most 2 / sqrt(d_qk) (the error a rounded key leaves in a score grows
-// with the scale).  Everything else multiplies the codes exactly.  A bfloat16 scale or bias can lie outside binary16's
-// range, so those caches never take the tile kernels.
-bool tiles_allowed(const q4kv_spec* s, float softmax_scale, bool converts_bf16 = false) {
-  return s->exact_products == 0 && (s->sb_dtype == 0 || converts_bf16) && softmax_scale > 0.f &&
-         softmax_scale * softmax_scale * (float)s->d_qk <= 4.f;
+// with the scale).  Everything else multiplies the codes exactly.  Bfloat16 scales and biases are converted to binary16
+// once per key block by those kernels (exact for every magnitude a cache written by this library can hold; a magnitude
+// beyond binary16's largest number, which only a foreign cache can hold, raises Q4KV_FLAG_SB_RANGE).
+bool tiles_allowed(const q4kv_spec* s, float softmax_scale) {
+  return s->exact_products == 0 && softmax_scale > 0.f && softmax_scale * softmax_scale * (float)s->d_qk <= 4.f;
 }
 
 }  // namespace
@@ -231,10 +231,10 @@ int q4kv_prefill_attention(const q4kv_spec* spec, const void* pool, int32_t n_bl
   const Layout y = make_layout(*spec, n_blocks);
   if (workspace_bytes < workspace_need(y, batch->n_agents, max_kv_len, total_q)) return Q4KV_EWORKSPACE;
   cudaError_t e;
-  if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale, true))
+  if (prefill_umma_supported(y) && tiles_allowed(spec, softmax_scale))
     e = launch_prefill_umma(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale, out,
                             out_dtype, lse, status_flags, (cudaStream_t)stream);
-  else if (prefill_umma_1tile_supported(y) && tiles_allowed(spec, softmax_scale, true))
+  else if (prefill_umma_1tile_supported(y) && tiles_allowed(spec, softmax_scale))
     e = launch_prefill_umma_1tile(y, pool, n_blocks, layer, *batch, kv_lens, q_offs, max_q_len, window, q, softmax_scale,
                                   out, out_dtype, lse, status_flags, (cudaStream_t)stream);
   else if (prefill_mma_supported(y))

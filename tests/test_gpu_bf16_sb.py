@@ -109,9 +109,9 @@ def test_update_and_fetch_in_one_launch(H, name, lens, window):
     assert p.dc.read_flags() == 0
 
 
-def test_latent_cache_update_and_fetch_runs_on_the_codes(H):
-    """A bfloat16 scale can lie outside binary16's range, so the latent-cache kernel that expands keys into binary16
-    tiles never serves such a cache: the kernel that multiplies the codes does, through both entries."""
+def test_latent_cache_update_and_fetch(H):
+    """A bfloat16 latent cache through both entries: the step's new row quantized with bfloat16 scale and bias by the
+    attention kernel itself, pool bytes as quantize-append writes them."""
     lens = [300, 64, 1000]
     steps = 2
     p = Pair(H, SPECS["mla"], lens, seed=140, extra_tokens=steps, sb_dtype=1).fill()
@@ -232,10 +232,7 @@ def test_layer_batched_entry_and_static_entry(H):
     assert p.dc.read_flags() == 0
 
 
-TILE_KERNELS_TAKE_BF16 = ("gqa128", "gqa256", "asym")
-
-
-@pytest.mark.parametrize("name", TILE_KERNELS_TAKE_BF16)
+@pytest.mark.parametrize("name", ["gqa128", "gqa256", "asym", "mla"])
 def test_a_scale_beyond_binary16_is_reported_by_the_tile_kernels(H, name):
     """The library's own quantizer never produces a scale or bias beyond binary16's largest number (its inputs are
     bounded by it, and the header asks the same of caches persisted elsewhere), but nothing stops a foreign file from
@@ -247,16 +244,23 @@ def test_a_scale_beyond_binary16_is_reported_by_the_tile_kernels(H, name):
     chunk = 40
     p = Pair(H, SPECS[name], [n + chunk for n in lens], seed=150, sb_dtype=1).fill()
     s = p.ospec
+    latent = bool(s.v_aliases_k)
     q_offs = [chunk * a for a in range(len(lens) + 1)]
-    q = p.q(7, chunk * len(lens))
-    scale = 1.0 / math.sqrt(s.d_qk)
-    good, _ = p.dc.prefill(0, p.lens, q_offs, 0, q, scale)
+    q = p.q(7, len(lens) if latent else chunk * len(lens))
+    scale = 1.0 / math.sqrt(192 if latent else s.d_qk)
+
+    def attend():
+        if latent:
+            return p.dc.decode(0, p.lens, 0, q, scale)[0]
+        return p.dc.prefill(0, p.lens, q_offs, 0, q, scale)[0]
+
+    good = attend()
     assert p.dc.read_flags() == 0
     blk = int(p.tabs[0][1])                            # agent 0's second block holds tokens 256 .. 339
     for tok, expect in ((340 - 256 + 3, False), (17, True)):     # past the length: ignored; inside: reported
-        p.opool.Vs[0, blk, 0, tok, 0] = 0x4980         # 2^20 as bfloat16
+        (p.opool.Ks if latent else p.opool.Vs)[0, blk, 0, tok, 0] = 0x4980     # 2^20 as bfloat16
         p.dc.unpack(0, 512, O.pack(p.opool, p.tabs[0], 512))
-        out, _ = p.dc.prefill(0, p.lens, q_offs, 0, q, scale)
+        out = attend()
         flags = p.dc.read_flags()
         assert bool(flags & B.FLAG_SB_RANGE) == expect and (flags & ~B.FLAG_SB_RANGE) == 0
         if not expect:
