@@ -126,7 +126,8 @@ class DeviceWorkload:
     """All state of one workload resident on the GPU: the Q4 pool (filled by the library's own quantizer
     from seeded on-device N(0,1) bf16 values), block tables, per-layer q / new K,V, outputs."""
 
-    def __init__(self, w: synth.Workload, device_index: int, two_calls: bool = False, exact_products: bool = False):
+    def __init__(self, w: synth.Workload, device_index: int, two_calls: bool = False, exact_products: bool = False,
+                 sb_dtype: int = 0):
         import torch
         from paper_2603_04428_b200 import binding as B, harness as H
         self.torch, self.B, self.w = torch, B, w
@@ -135,7 +136,7 @@ class DeviceWorkload:
         self.n_blocks = w.blocks_needed() + 4
         tabs = synth.block_tables(w.seed, 99, w.lens, self.n_blocks, extra_tokens=w.new_tokens)
         self.dc = H.DeviceCache(L, w.n_q_heads, w.n_kv_heads, w.d_qk, w.d_v, w.v_aliases_k, self.n_blocks, tabs,
-                                fill_byte=None, exact_products=exact_products)
+                                fill_byte=None, exact_products=exact_products, sb_dtype=sb_dtype)
         dc = self.dc
         g = torch.Generator(device="cuda")
         g.manual_seed(w.seed)
@@ -392,7 +393,8 @@ def measure(w, args, local, dist=None, full=True):
     region of at least half a second (median batch), the per-launch time of the attention kernel from a graph of the L
     attention calls, clocks sampled meanwhile; with full=True also the end-to-end step through host buffers."""
     import torch
-    dw = DeviceWorkload(w, local, two_calls=args.two_calls, exact_products=args.exact_products)
+    dw = DeviceWorkload(w, local, two_calls=args.two_calls, exact_products=args.exact_products,
+                        sb_dtype=1 if args.sb_bf16 else 0)
     L = w.n_layers
     use_graph = not args.no_graph
     stream = torch.cuda.Stream()
@@ -586,6 +588,8 @@ def main():
                     help="decode step as a quantize-append launch plus an attention launch per layer instead of the "
                          "one-launch update-and-fetch")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="least duration of each timed region")
+    ap.add_argument("--sb-bf16", action="store_true",
+                    help="bfloat16 scales and biases in the cache (q4kv_spec.sb_dtype = 1) instead of binary16")
     ap.add_argument("--exact-products", action="store_true",
                     help="set q4kv_spec.exact_products: every call takes the kernels that multiply the 4-bit codes exactly")
     ap.add_argument("--op", default="step", choices=["step", "pack", "unpack"],
@@ -598,7 +602,8 @@ def main():
         print(json.dumps(run_pack(args)))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "q4kv" else args.warmup
-    default_run = args.workload is None and args.agents == 0 and args.layers == 0 and not args.exact_products
+    default_run = (args.workload is None and args.agents == 0 and args.layers == 0 and not args.exact_products
+                   and not args.sb_bf16)
     w = synth.workload(1 if args.workload is None else args.workload)
     if args.agents > 0 or args.layers > 0:
         # not one of the five configurations any more: the name says so, and no stored counter applies to it
@@ -609,6 +614,8 @@ def main():
         w = dataclasses.replace(w, lens=lens, n_layers=layers, name=f"{w.name}_scaled_{len(lens)}agents_{layers}layers")
     if args.exact_products:
         w = dataclasses.replace(w, name=w.name + "_exact_products")       # other kernels: no stored counter applies
+    if args.sb_bf16:
+        w = dataclasses.replace(w, name=w.name + "_bf16_scale_bias")
     if args.impl == "reference":
         run_reference(args, w)
         return
