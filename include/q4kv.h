@@ -75,9 +75,9 @@ typedef struct {
                             (shared latent of MLA in absorbed form); requires d_v <= d_qk           */
   int32_t group;         /* quantization group, must be 64                                          */
   int32_t block_tokens;  /* tokens per pool block, must be 256                                      */
-  int32_t sb_dtype;      /* scale/bias type: 0 = binary16, 1 = bfloat16.  A bfloat16 cache is always
-                            attended by the kernels that multiply the codes exactly (as with
-                            exact_products = 1): its scales can lie outside binary16's range          */
+  int32_t sb_dtype;      /* scale/bias type: 0 = binary16, 1 = bfloat16.  Both take the same kernels; those
+                            that work in binary16 convert a bfloat16 scale or bias first (see "Accuracy"
+                            and Q4KV_FLAG_SB_RANGE)                                                  */
   int32_t exact_products;/* 0: attention kernels may expand the cache into binary16 tiles (one rounding
                             of every dequantized value, see "Accuracy" below); 1: always multiply the
                             4-bit codes exactly.  Ignored by append, pack and unpack.               */
@@ -123,9 +123,16 @@ enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
  *     query heads per KV head; decode on the MLA-latent cache: V aliasing K, d_qk 576, d_v 512, one
  *     KV head, at most 16 query heads) round every dequantized value once to binary16, a relative
  *     error of 2^-11 at most, and the probabilities likewise.  They are chosen only when
- *     exact_products == 0, sb_dtype == 0 and softmax_scale <= 2/sqrt(d_qk).  Their error is at most
+ *     exact_products == 0 and softmax_scale <= 2/sqrt(d_qk).  Their error is at most
  *     2^-10 * M * (1 + softmax_scale * ||q||_1 * M): the value and probability roundings, plus what
- *     the rounded keys do to the softmax weights.  On caches of unit-variance values (M about 5) the
+ *     the rounded keys do to the softmax weights.  A bfloat16 scale or bias enters as the binary16
+ *     number of the same value: exact for magnitudes in [2^-14, 65504] (a bfloat16 number has 8
+ *     significant bits), off by at most 2^-25 below that, so for bfloat16 caches add 2^-20 to the
+ *     bound; a magnitude above 65504 raises Q4KV_FLAG_SB_RANGE.  The quantizer of this library never
+ *     writes such a value (its inputs are bf16 numbers of magnitude at most 65504: the bias is then
+ *     the group's minimum itself and the scale at most 8734); a cache persisted elsewhere should keep
+ *     |code * scale + bias| <= 65504 as well: no tensor-core kernel here, exact or not, carries
+ *     probability x scale beyond binary16's range.  On caches of unit-variance values (M about 5) the
  *     roundings average out over the attended keys and the measured error is below 3e-4; a cache
  *     with outlier channels or a gain (M >= 8) needs exact_products = 1 to stay within 2e-3. */
 
