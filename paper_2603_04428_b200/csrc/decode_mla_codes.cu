@@ -1,7 +1,7 @@
 // q4kv_decode_attention for the MLA-latent cache, on the 4-bit codes (d_qk = 576 = 512 latent + 64 rope,
 // d_v = 512, V aliases the first 512 dims of K, one shared KV head, up to 16 query heads): the route of
-// calls that ask for exact products, of caches with bfloat16 scales and biases, and of sharp softmax
-// scales (Section 3.4 "Batched Quantized Inference"; the MLA cache of Section 3.6).
+// calls that ask for exact products and of sharp softmax scales, for either scale / bias type
+// (Section 3.4 "Batched Quantized Inference"; the MLA cache of Section 3.6).
 //
 // Every key serves all 16 heads and is both key and value, and both products run on the codes
 // themselves (mma.sync m16n8k16 f16; a nibble masked in place in a 16-bit lane is the binary16

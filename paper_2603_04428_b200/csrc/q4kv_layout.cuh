@@ -165,7 +165,7 @@ cudaError_t launch_prefill_umma_1tile(const Layout& y, const void* pool, int n_b
 
 // Decode on the MLA-latent cache (d_qk 576, d_v 512 aliasing K, one KV head, at most 16 query heads): a key-split
 // attention kernel -- on a binary16 tile of the dequantized keys, or, with on_codes, on the 4-bit codes themselves
-// (exact products; the only form for bfloat16 scales and biases) -- followed by the combination of the records.
+// (exact products) -- followed by the combination of the records.
 bool decode_mla_supported(const Layout& y);
 size_t decode_mla_workspace_bytes(const Layout& y, int n_agents, int max_kv_len);
 cudaError_t launch_decode_mla(const Layout& y, const void* pool, int n_blocks, int layer, const q4kv_batch& b,
