@@ -670,6 +670,11 @@ def main():
         w3 = synth.workload(3)
         entry(dataclasses.replace(w3, name=w3.name + "_exact_products"),
               argparse.Namespace(**{**vars(args), "exact_products": True}))
+        # caches with bfloat16 scales and biases (q4kv_spec.sb_dtype = 1) on the two binary16-tile routes
+        for idx in (3, 4):
+            wi = synth.workload(idx)
+            entry(dataclasses.replace(wi, name=wi.name + "_bf16_scale_bias"),
+                  argparse.Namespace(**{**vars(args), "sb_bf16": True}))
         pk = run_pack(args)
         for name in ("pack", "unpack", "restore", "append_8x1024"):
             allc[name] = pk["kernels"][name]
