@@ -103,8 +103,9 @@ enum {
   Q4KV_FLAG_BAD_LENGTH = 2,  /* a length or position negative or beyond max_blocks*256              */
   Q4KV_FLAG_INTERNAL = 4,    /* a bounded wait inside a kernel ran out (the output is not valid)    */
   Q4KV_FLAG_SB_RANGE = 8     /* a bfloat16 scale or bias beyond binary16's largest number met a kernel that
-                                expands the cache into binary16 tiles: the call's output is not valid;
-                                set exact_products and call again                                    */
+                                expands the cache into binary16 tiles: the call's output is not valid
+                                (such a cache lies outside what the tensor-core kernels carry, see
+                                "Accuracy"; this library's quantizer never writes one)               */
 };
 enum { Q4KV_OUT_F32 = 0, Q4KV_OUT_BF16 = 1 };
 
