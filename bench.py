@@ -381,8 +381,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # fewer layers (the launch itself is the full-size one, so nothing is scaled); the config-3 figure is a global layer's
 # launch, the MLA figure the attention kernel without its merge launch (4.88 MB more when its records miss L2).
 NCU_TRAFFIC_BYTES = {"llama31_8b_decode": 23_991_723, "gemma3_12b_ragged_decode": 365_462_784,
-                     "dsv2lite_mla_decode": 21_440_640, "dsv2lite_mla_decode_exact_products": 21_446_656,
-                     "llama31_8b_chunked_prefill": 240_450_688,
+                     "dsv2lite_mla_decode": 21_440_512, "dsv2lite_mla_decode_exact_products": 21_446_656,
+                     "llama31_8b_chunked_prefill": 241_124_480,
                      "dsv2lite_perhead_mla_decode": 191_148_800, "gemma3_12b_shaped_global_prefill": 151_449_472,
                      "dsv2lite_perhead_mla_prefill": 146_757_504,
                      "pack": 254_257_000, "unpack": 251_510_000, "append_8x1024": 33_606_912}
